@@ -1,0 +1,229 @@
+"""CPU oracle for the speculative-decoding verify step.  TEST INFRASTRUCTURE ONLY.
+
+A thin ctypes wrapper around ``spx_oracle.c`` (plain C, float64 arithmetic, OpenMP over
+independent items).  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
+import this package; the CUDA library and its Python binding never do, and the two share no
+code.  See the header of ``spx_oracle.c`` for what each function follows and how it is pinned.
+
+All tensors are CPU ``torch`` tensors (bf16 or fp32 for data, int32 for indices); outputs are
+float64 / int32 CPU tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "spx_oracle.c")
+_LIB_PATH = os.path.join(_HERE, "libspx_oracle.so")
+
+BF16, F32 = 0, 1
+OK, ERR_ARG, ERR_LEN, ERR_PAGE, ERR_TOKEN, ERR_ALLOC = 0, 1, 2, 3, 4, 5
+FLAG_DEGENERATE = 1
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (-O2, OpenMP).  Returns the library path."""
+    if force or not os.path.exists(_LIB_PATH) or os.path.getmtime(_LIB_PATH) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-Wall", "-o", _LIB_PATH,
+               _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB_PATH
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB_PATH)
+        c = ctypes
+        lib.oracle_num_threads.restype = c.c_int
+        lib.oracle_verify_attention.restype = c.c_int
+        lib.oracle_verify_attention.argtypes = [
+            c.c_int32, c.c_int32, c.c_int32, c.c_int32, c.c_int32, c.c_int64, c.c_int32, c.c_int32,
+            c.c_double, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int64, c.c_int64, c.c_int64,
+            c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int32, c.c_void_p, c.c_void_p]
+        lib.oracle_softmax_row.restype = None
+        lib.oracle_softmax_row.argtypes = [c.c_void_p, c.c_int32, c.c_int64, c.c_int64, c.c_void_p]
+        lib.oracle_residual.restype = c.c_double
+        lib.oracle_residual.argtypes = [c.c_void_p, c.c_void_p, c.c_int64, c.c_void_p]
+        lib.oracle_inverse_cdf.restype = c.c_int64
+        lib.oracle_inverse_cdf.argtypes = [c.c_void_p, c.c_int64, c.c_double, c.c_double,
+                                           c.c_void_p, c.c_void_p]
+        lib.oracle_rejection_sample.restype = c.c_int
+        lib.oracle_rejection_sample.argtypes = [
+            c.c_int32, c.c_int64, c.c_int64, c.c_int32, c.c_void_p, c.c_void_p, c.c_void_p,
+            c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+            c.c_void_p, c.c_void_p, c.c_void_p]
+        lib.oracle_emit_cdf.restype = c.c_double
+        lib.oracle_emit_cdf.argtypes = [c.c_int32, c.c_int32, c.c_int64, c.c_int64, c.c_int32,
+                                        c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+        lib.oracle_verify_step.restype = c.c_int
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError(f"oracle accepts bf16 or fp32 data, got {t.dtype}")
+
+
+def _cpu(t: torch.Tensor, dtype=None) -> torch.Tensor:
+    assert t.device.type == "cpu", "oracle inputs must be host tensors"
+    if dtype is not None:
+        assert t.dtype == dtype, (t.dtype, dtype)
+    return t
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+class OracleError(RuntimeError):
+    def __init__(self, code: int):
+        super().__init__(f"oracle returned error code {code}")
+        self.code = code
+
+
+def verify_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
+                     kv_strides: Sequence[int], block_table: torch.Tensor, seq_lens: torch.Tensor,
+                     q_indptr: torch.Tensor, num_kv_heads: int, page_size: int, num_pages: int,
+                     sm_scale: float = 0.0, req_list: Optional[Sequence[int]] = None):
+    """Attention of every request's k+1 query rows over its paged cache, in float64.
+
+    ``q`` is [TQ, Hq, D]; ``k_cache``/``v_cache`` are pools addressed by
+    ``kv_strides = (page, head, token)`` element strides with D contiguous.  Returns
+    ``(out [TQ,Hq,D] float64, lse [TQ,Hq] float64)``; with ``req_list`` only those requests'
+    rows are computed (the rest stay NaN).
+    """
+    lib = _load()
+    q = _cpu(q).contiguous()
+    dt = _dtype_code(q)
+    assert _dtype_code(k_cache) == dt and _dtype_code(v_cache) == dt
+    TQ, Hq, D = q.shape
+    B = seq_lens.numel()
+    bt = _cpu(block_table, torch.int32).contiguous()
+    sl = _cpu(seq_lens, torch.int32).contiguous()
+    qi = _cpu(q_indptr, torch.int32).contiguous()
+    out = torch.full((TQ, Hq, D), float("nan"), dtype=torch.float64)
+    lse = torch.full((TQ, Hq), float("nan"), dtype=torch.float64)
+    rl = None
+    n_rl = 0
+    if req_list is not None:
+        rl = torch.tensor(list(req_list), dtype=torch.int32)
+        n_rl = rl.numel()
+    st = lib.oracle_verify_attention(
+        B, Hq, num_kv_heads, D, page_size, num_pages, bt.shape[1] if bt.dim() == 2 else 0, dt,
+        float(sm_scale), _ptr(q), _ptr(k_cache), _ptr(v_cache), int(kv_strides[0]),
+        int(kv_strides[1]), int(kv_strides[2]), _ptr(bt), _ptr(sl), _ptr(qi), _ptr(rl), n_rl,
+        _ptr(out), _ptr(lse))
+    if st != OK:
+        raise OracleError(st)
+    return out, lse
+
+
+def softmax_row(logits_row: torch.Tensor) -> torch.Tensor:
+    """Step 1 of the sampling rule: float64 softmax of one stored logits row."""
+    lib = _load()
+    row = _cpu(logits_row).contiguous()
+    p = torch.empty(row.numel(), dtype=torch.float64)
+    lib.oracle_softmax_row(_ptr(row), _dtype_code(row), 0, row.numel(), _ptr(p))
+    return p
+
+
+def residual(p: torch.Tensor, q: torch.Tensor):
+    """Step 3: r = max(0, p - q) and its mass R."""
+    lib = _load()
+    p = _cpu(p, torch.float64).contiguous()
+    q = _cpu(q, torch.float64).contiguous()
+    r = torch.empty_like(p)
+    R = lib.oracle_residual(_ptr(p), _ptr(q), p.numel(), _ptr(r))
+    return r, float(R)
+
+
+def inverse_cdf(r: torch.Tensor, R: float, s: float) -> int:
+    """Steps 3/4: the first token whose inclusive cumulative mass exceeds s*R."""
+    lib = _load()
+    r = _cpu(r, torch.float64).contiguous()
+    return int(lib.oracle_inverse_cdf(_ptr(r), r.numel(), float(R), float(s), None, None))
+
+
+@dataclass
+class SampleResult:
+    accepted_len: torch.Tensor   # [B] int32
+    out_tokens: torch.Tensor     # [TQ] int32
+    rho: torch.Tensor            # [TD] float64, NaN for drafts after the first rejection
+    resid_mass: torch.Tensor     # [B] float64
+    cdf_lo: torch.Tensor         # [B] float64
+    cdf_hi: torch.Tensor         # [B] float64
+    flags: torch.Tensor          # [B] int32
+    status: int                  # OK or ERR_TOKEN
+
+
+def rejection_sample(target_logits: torch.Tensor, draft_logits: torch.Tensor,
+                     draft_ids: torch.Tensor, q_indptr: torch.Tensor, u_accept: torch.Tensor,
+                     u_sample: torch.Tensor, vocab: Optional[int] = None) -> SampleResult:
+    """Speculative rejection sampling for the whole batch, in float64, one request at a time."""
+    lib = _load()
+    tl = _cpu(target_logits)
+    dl = _cpu(draft_logits)
+    assert tl.dim() == 2 and tl.stride(1) == 1
+    dt = _dtype_code(tl)
+    row_stride = tl.stride(0)
+    V = int(vocab if vocab is not None else tl.shape[1])
+    if dl.numel() > 0:
+        assert dl.dim() == 2 and dl.stride(1) == 1 and dl.stride(0) == row_stride
+        assert _dtype_code(dl) == dt
+    qi = _cpu(q_indptr, torch.int32).contiguous()
+    B = qi.numel() - 1
+    TQ = int(qi[-1])
+    TD = TQ - B
+    ids = _cpu(draft_ids, torch.int32).contiguous()
+    ua = _cpu(u_accept, torch.float32).contiguous()
+    us = _cpu(u_sample, torch.float32).contiguous()
+    assert ids.numel() == TD and ua.numel() == TD and us.numel() == B
+    res = SampleResult(
+        accepted_len=torch.empty(B, dtype=torch.int32),
+        out_tokens=torch.empty(TQ, dtype=torch.int32),
+        rho=torch.empty(TD, dtype=torch.float64),
+        resid_mass=torch.empty(B, dtype=torch.float64),
+        cdf_lo=torch.empty(B, dtype=torch.float64),
+        cdf_hi=torch.empty(B, dtype=torch.float64),
+        flags=torch.empty(B, dtype=torch.int32),
+        status=OK)
+    st = lib.oracle_rejection_sample(
+        B, V, row_stride, dt, _ptr(tl), _ptr(dl), _ptr(ids), _ptr(qi), _ptr(ua), _ptr(us),
+        _ptr(res.accepted_len), _ptr(res.out_tokens), _ptr(res.rho), _ptr(res.resid_mass),
+        _ptr(res.cdf_lo), _ptr(res.cdf_hi), _ptr(res.flags))
+    if st not in (OK, ERR_TOKEN):
+        raise OracleError(st)
+    res.status = st
+    return res
+
+
+def emit_cdf(r: int, n: int, target_logits: torch.Tensor, draft_logits: torch.Tensor,
+             q_indptr: torch.Tensor, vocab: Optional[int] = None):
+    """Inclusive cumulative distribution request ``r``'s emitted token was drawn from, and R."""
+    lib = _load()
+    tl = _cpu(target_logits)
+    dl = _cpu(draft_logits)
+    V = int(vocab if vocab is not None else tl.shape[1])
+    qi = _cpu(q_indptr, torch.int32).contiguous()
+    cdf = torch.empty(V, dtype=torch.float64)
+    R = lib.oracle_emit_cdf(int(r), int(n), V, tl.stride(0), _dtype_code(tl), _ptr(tl), _ptr(dl),
+                            _ptr(qi), _ptr(cdf))
+    return cdf, float(R)

@@ -1,0 +1,437 @@
+/*
+ * CPU oracle for the speculative-decoding verify step.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is a plain, slow, float64 restatement of what the verify step computes.  It is
+ * used by the tests, by the smoke check and by the benchmark's CPU-baseline leg, and by
+ * nothing else: the CUDA library never links, loads or calls it, and it shares no code,
+ * header, table or helper with the CUDA path.
+ *
+ * What it follows.  The paper (Section 2, "Speculative decoding"; Section 4,
+ * "Self-speculation and parallel scheduling") states only that a draft proposes several
+ * tokens and the base model verifies them jointly against one shared, paged KV cache; it
+ * prints no formula for either half.  The two halves are therefore written out from their
+ * standard definitions:
+ *
+ *   (A) attention  - textbook scaled-dot-product attention with a causal mask among the
+ *       k+1 new positions, keys and values addressed through a block table (paged cache);
+ *   (B) speculative sampling - the rule of the speculative-decoding work the paper cites in
+ *       Section 2: accept draft x_i with probability min(1, p_i(x_i)/q_i(x_i)); at the
+ *       first rejection draw from the normalised residual max(0, p - q); if every draft is
+ *       accepted draw one bonus token from the target distribution.
+ *
+ * Every input value (bf16 or fp32) is widened exactly to double; all arithmetic is double.
+ * There is no tiling, no online softmax, no fusion: two plain passes per softmax and a
+ * sequential cumulative sum for the inverse CDF, so that each loop can be checked against
+ * the definition by eye.  OpenMP is used only across independent (request, position, head)
+ * or row items; it never changes the order of any floating-point sum.
+ *
+ * Pins (tests/test_oracle_*.py): brute-force numpy float64 attention on tiny inputs,
+ * weights-sum-to-one, causal and page-placement invariance, closed forms (K = 0 gives the
+ * mean of V and LSE = log n; one token gives V[0]), a needle key, GQA head duplication; for
+ * sampling a chi-square test of the output law against the target distribution on a
+ * 16-token vocabulary, the identity min(p,q) + (1-beta) r/R = p, closed-form acceptance
+ * rates, special cases, and interval-arithmetic brute force on tiny vocabularies.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORACLE_BF16 = 0, ORACLE_F32 = 1 };
+
+enum {
+  ORACLE_OK = 0,
+  ORACLE_ERR_ARG = 1,      /* bad scalar argument                                   */
+  ORACLE_ERR_LEN = 2,      /* some L_r < k_r + 1                                     */
+  ORACLE_ERR_PAGE = 3,     /* a needed block-table entry is outside [0, num_pages)   */
+  ORACLE_ERR_TOKEN = 4,    /* a draft token id is outside [0, V)                     */
+  ORACLE_ERR_ALLOC = 5
+};
+
+/* Bit flags written per request by the sampler. */
+enum { ORACLE_FLAG_DEGENERATE = 1 /* residual mass R == 0, target row used instead */ };
+
+static inline double widen(const void *base, int dtype, int64_t idx) {
+  if (dtype == ORACLE_F32) return (double)((const float *)base)[idx];
+  /* bf16 is the upper 16 bits of an IEEE binary32 */
+  uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16;
+  float f;
+  memcpy(&f, &bits, sizeof f);
+  return (double)f;
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* (A) attention                                                                         */
+/* ------------------------------------------------------------------------------------ */
+
+/*
+ * For request r with k_r = q_indptr[r+1]-q_indptr[r]-1 drafts and L_r = seq_lens[r] cached
+ * tokens (the k_r+1 new positions included), query j in [0,k_r], q-head h, kv-head
+ * g = h / (Hq/Hkv), pos = L_r-(k_r+1)+j:
+ *
+ *   s_t   = scale * sum_d Q[qi,h,d] K[t,g,d]         t = 0..pos
+ *   w_t   = exp(s_t - max_t s_t) / sum_t exp(s_t - max)
+ *   O     = sum_t w_t V[t,g,:]
+ *   LSE   = max + log sum_t exp(s_t - max)
+ *
+ * Token t of request r lives in page block_table[r][t / P], slot t % P; element
+ * (page, g, slot, d) of a pool is at page*stride_page + g*stride_head + slot*stride_token + d.
+ *
+ * req_list (may be NULL) restricts the computation to the listed requests; rows of other
+ * requests in out/lse are left untouched.  out is [TQ,Hq,D] double, lse [TQ,Hq] double
+ * (lse may be NULL).
+ */
+int oracle_verify_attention(int32_t batch, int32_t Hq, int32_t Hkv, int32_t D, int32_t P,
+                            int64_t num_pages, int32_t max_pages_per_req, int32_t dtype,
+                            double sm_scale, const void *q, const void *k_cache,
+                            const void *v_cache, int64_t stride_page, int64_t stride_head,
+                            int64_t stride_token, const int32_t *block_table,
+                            const int32_t *seq_lens, const int32_t *q_indptr,
+                            const int32_t *req_list, int32_t n_req_list, double *out,
+                            double *lse) {
+  if (batch < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || D <= 0 || P <= 0) return ORACLE_ERR_ARG;
+  if (dtype != ORACLE_BF16 && dtype != ORACLE_F32) return ORACLE_ERR_ARG;
+  const int G = Hq / Hkv;
+  const double scale = (sm_scale == 0.0) ? 1.0 / sqrt((double)D) : sm_scale;
+  const int n_req = req_list ? n_req_list : batch;
+
+  /* validate first, so that the parallel part below has no early exits */
+  for (int ri = 0; ri < n_req; ++ri) {
+    const int r = req_list ? req_list[ri] : ri;
+    if (r < 0 || r >= batch) return ORACLE_ERR_ARG;
+    const int m = q_indptr[r + 1] - q_indptr[r];
+    const int L = seq_lens[r];
+    if (m < 1 || L < m) return ORACLE_ERR_LEN;
+    const int n_pages = (L + P - 1) / P;
+    if (n_pages > max_pages_per_req) return ORACLE_ERR_PAGE;
+    for (int pg = 0; pg < n_pages; ++pg) {
+      const int32_t phys = block_table[(int64_t)r * max_pages_per_req + pg];
+      if (phys < 0 || phys >= num_pages) return ORACLE_ERR_PAGE;
+    }
+  }
+
+  /* flatten (request, position, head) so that OpenMP can balance ragged lengths */
+  int64_t n_items = 0;
+  for (int ri = 0; ri < n_req; ++ri) {
+    const int r = req_list ? req_list[ri] : ri;
+    n_items += (int64_t)(q_indptr[r + 1] - q_indptr[r]) * Hq;
+  }
+  int32_t *item_r = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_items > 0 ? n_items : 1));
+  int32_t *item_j = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_items > 0 ? n_items : 1));
+  int32_t *item_h = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_items > 0 ? n_items : 1));
+  if (!item_r || !item_j || !item_h) { free(item_r); free(item_j); free(item_h); return ORACLE_ERR_ALLOC; }
+  {
+    int64_t it = 0;
+    for (int ri = 0; ri < n_req; ++ri) {
+      const int r = req_list ? req_list[ri] : ri;
+      const int m = q_indptr[r + 1] - q_indptr[r];
+      for (int j = 0; j < m; ++j)
+        for (int h = 0; h < Hq; ++h) { item_r[it] = r; item_j[it] = j; item_h[it] = h; ++it; }
+    }
+  }
+
+  int alloc_failed = 0;
+#pragma omp parallel
+  {
+    double *s = NULL;
+    int64_t s_cap = 0;
+    double *qrow = (double *)malloc(sizeof(double) * (size_t)D);
+    double *acc = (double *)malloc(sizeof(double) * (size_t)D);
+    if (!qrow || !acc) {
+#pragma omp atomic write
+      alloc_failed = 1;
+    }
+#pragma omp for schedule(dynamic, 1)
+    for (int64_t it = 0; it < n_items; ++it) {
+      if (alloc_failed) continue;
+      const int r = item_r[it], j = item_j[it], h = item_h[it];
+      const int g = h / G;
+      const int m = q_indptr[r + 1] - q_indptr[r];
+      const int L = seq_lens[r];
+      const int pos = L - m + j;               /* last visible token index */
+      const int64_t qi = (int64_t)q_indptr[r] + j;
+      const int32_t *bt = block_table + (int64_t)r * max_pages_per_req;
+      if (pos + 1 > s_cap) {
+        free(s);
+        s_cap = pos + 1;
+        s = (double *)malloc(sizeof(double) * (size_t)s_cap);
+        if (!s) {
+#pragma omp atomic write
+          alloc_failed = 1;
+          s_cap = 0;
+          continue;
+        }
+      }
+      for (int d = 0; d < D; ++d) qrow[d] = widen(q, dtype, (qi * Hq + h) * D + d);
+
+      /* pass 1: scores and their maximum */
+      double mx = -INFINITY;
+      for (int t = 0; t <= pos; ++t) {
+        const int64_t base = (int64_t)bt[t / P] * stride_page + (int64_t)g * stride_head +
+                             (int64_t)(t % P) * stride_token;
+        double dot = 0.0;
+        for (int d = 0; d < D; ++d) dot += qrow[d] * widen(k_cache, dtype, base + d);
+        s[t] = scale * dot;
+        if (s[t] > mx) mx = s[t];
+      }
+      /* pass 2: normaliser */
+      double denom = 0.0;
+      for (int t = 0; t <= pos; ++t) denom += exp(s[t] - mx);
+      /* weighted sum of values */
+      for (int d = 0; d < D; ++d) acc[d] = 0.0;
+      for (int t = 0; t <= pos; ++t) {
+        const double w = exp(s[t] - mx) / denom;
+        const int64_t base = (int64_t)bt[t / P] * stride_page + (int64_t)g * stride_head +
+                             (int64_t)(t % P) * stride_token;
+        for (int d = 0; d < D; ++d) acc[d] += w * widen(v_cache, dtype, base + d);
+      }
+      for (int d = 0; d < D; ++d) out[(qi * Hq + h) * D + d] = acc[d];
+      if (lse) lse[qi * Hq + h] = mx + log(denom);
+    }
+    free(s); free(qrow); free(acc);
+  }
+  free(item_r); free(item_j); free(item_h);
+  return alloc_failed ? ORACLE_ERR_ALLOC : ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* (B) speculative rejection sampling                                                    */
+/* ------------------------------------------------------------------------------------ */
+
+/* Step 1: p = softmax(row) over the full vocabulary at temperature 1, max subtracted. */
+void oracle_softmax_row(const void *logits, int32_t dtype, int64_t row_offset, int64_t V,
+                        double *p) {
+  double mx = -INFINITY;
+  for (int64_t v = 0; v < V; ++v) {
+    const double x = widen(logits, dtype, row_offset + v);
+    if (x > mx) mx = x;
+  }
+  double denom = 0.0;
+  for (int64_t v = 0; v < V; ++v) {
+    p[v] = exp(widen(logits, dtype, row_offset + v) - mx);
+    denom += p[v];
+  }
+  for (int64_t v = 0; v < V; ++v) p[v] /= denom;
+}
+
+/* Step 3 (first half): r(v) = max(0, p(v) - q(v)); returns R = sum_v r(v), ascending v. */
+double oracle_residual(const double *p, const double *q, int64_t V, double *r) {
+  double R = 0.0;
+  for (int64_t v = 0; v < V; ++v) {
+    const double d = p[v] - q[v];
+    r[v] = d > 0.0 ? d : 0.0;
+    R += r[v];
+  }
+  return R;
+}
+
+/*
+ * Steps 3/4 (second half): y = min{ v : sum_{w<=v} r(w) > s*R }.  If rounding leaves no such
+ * v, y is the largest v with r(v) > 0.  Bins of zero width are never selected because the
+ * inequality is strict and the cumulative sum does not move across them.  cdf_lo/cdf_hi (may
+ * be NULL) receive the exclusive/inclusive cumulative sums at y.  Returns -1 only if every
+ * r(v) is zero.
+ */
+int64_t oracle_inverse_cdf(const double *r, int64_t V, double R, double s, double *cdf_lo,
+                           double *cdf_hi) {
+  const double target = s * R;
+  double cum = 0.0;
+  int64_t last_pos = -1;
+  double last_lo = 0.0, last_hi = 0.0;
+  for (int64_t v = 0; v < V; ++v) {
+    const double before = cum;
+    cum += r[v];
+    if (r[v] > 0.0) { last_pos = v; last_lo = before; last_hi = cum; }
+    if (cum > target) {
+      if (cdf_lo) *cdf_lo = before;
+      if (cdf_hi) *cdf_hi = cum;
+      return v;
+    }
+  }
+  if (cdf_lo) *cdf_lo = last_lo;
+  if (cdf_hi) *cdf_hi = last_hi;
+  return last_pos;
+}
+
+/* Inclusive cumulative sum of r, ascending v, written to cdf[0..V).  For near-tie accounting. */
+void oracle_cumsum(const double *r, int64_t V, double *cdf) {
+  double cum = 0.0;
+  for (int64_t v = 0; v < V; ++v) { cum += r[v]; cdf[v] = cum; }
+}
+
+/*
+ * One request.  T_i = target row q_indptr[r]+i (i = 0..k), D_i = draft row q_indptr[r]-r+i
+ * (i = 0..k-1), x_i = draft_ids[q_indptr[r]-r+i], a_i = u_accept[same], s = u_sample[r].
+ * Scratch p, q, res each hold V doubles.
+ */
+static int sample_one(int r, int32_t dtype, int64_t V, int64_t row_stride,
+                      const void *target_logits, const void *draft_logits,
+                      const int32_t *draft_ids, const int32_t *q_indptr, const float *u_accept,
+                      const float *u_sample, int32_t *accepted_len, int32_t *out_tokens,
+                      double *rho_out, double *resid_mass, double *cdf_lo, double *cdf_hi,
+                      int32_t *flags, double *p, double *q, double *res) {
+  const int64_t t0 = q_indptr[r];          /* first target row / first output slot */
+  const int64_t d0 = (int64_t)q_indptr[r] - r; /* first draft row */
+  const int k = q_indptr[r + 1] - q_indptr[r] - 1;
+  int n = k;
+  int bad_token = 0;
+  if (flags) flags[r] = 0;
+  for (int i = 0; i < k && !bad_token; ++i)
+    if (draft_ids[d0 + i] < 0 || draft_ids[d0 + i] >= V) bad_token = 1;
+  if (bad_token) {
+    accepted_len[r] = 0;
+    for (int i = 0; i <= k; ++i) out_tokens[t0 + i] = -1;
+    if (rho_out) for (int i = 0; i < k; ++i) rho_out[d0 + i] = NAN;
+    if (resid_mass) resid_mass[r] = NAN;
+    if (cdf_lo) cdf_lo[r] = NAN;
+    if (cdf_hi) cdf_hi[r] = NAN;
+    return ORACLE_ERR_TOKEN;
+  }
+  if (rho_out) for (int i = 0; i < k; ++i) rho_out[d0 + i] = NAN; /* rows after n: not consulted */
+
+  /* step 2: sequential accept tests */
+  for (int i = 0; i < k; ++i) {
+    const int64_t x = draft_ids[d0 + i];
+    oracle_softmax_row(target_logits, dtype, (t0 + i) * row_stride, V, p);
+    oracle_softmax_row(draft_logits, dtype, (d0 + i) * row_stride, V, q);
+    const double rho = (q[x] == 0.0) ? INFINITY : p[x] / q[x];
+    if (rho_out) rho_out[d0 + i] = rho;
+    if (!((double)u_accept[d0 + i] < rho)) { n = i; break; }
+  }
+
+  double R, lo = 0.0, hi = 0.0;
+  int64_t y;
+  if (n < k) {
+    /* step 3: p, q still hold rows n */
+    R = oracle_residual(p, q, V, res);
+    if (R == 0.0) {
+      if (flags) flags[r] |= ORACLE_FLAG_DEGENERATE;
+      R = 0.0;
+      for (int64_t v = 0; v < V; ++v) { res[v] = p[v]; R += p[v]; }
+    }
+    y = oracle_inverse_cdf(res, V, R, (double)u_sample[r], &lo, &hi);
+  } else {
+    /* step 4: bonus token from target row k */
+    oracle_softmax_row(target_logits, dtype, (t0 + k) * row_stride, V, p);
+    R = 0.0;
+    for (int64_t v = 0; v < V; ++v) R += p[v];
+    y = oracle_inverse_cdf(p, V, R, (double)u_sample[r], &lo, &hi);
+  }
+
+  /* step 5 */
+  accepted_len[r] = n;
+  for (int i = 0; i < n; ++i) out_tokens[t0 + i] = draft_ids[d0 + i];
+  out_tokens[t0 + n] = (int32_t)y;
+  for (int i = n + 1; i <= k; ++i) out_tokens[t0 + i] = -1;
+  if (resid_mass) resid_mass[r] = R;
+  if (cdf_lo) cdf_lo[r] = lo;
+  if (cdf_hi) cdf_hi[r] = hi;
+  return ORACLE_OK;
+}
+
+/*
+ * Whole batch.  Outputs accepted_len [B], out_tokens [TQ]; optional diagnostics: rho [TD]
+ * (p/q per consulted draft, NaN for drafts after the first rejection), resid_mass [B] (the R
+ * used), cdf_lo/cdf_hi [B] (cumulative sums bracketing the emitted token), flags [B].
+ * Returns ORACLE_ERR_TOKEN if some request carried an invalid draft id (that request emits
+ * n = 0 and -1 tokens; the others are unaffected).
+ */
+int oracle_rejection_sample(int32_t batch, int64_t V, int64_t row_stride, int32_t dtype,
+                            const void *target_logits, const void *draft_logits,
+                            const int32_t *draft_ids, const int32_t *q_indptr,
+                            const float *u_accept, const float *u_sample,
+                            int32_t *accepted_len, int32_t *out_tokens, double *rho_out,
+                            double *resid_mass, double *cdf_lo, double *cdf_hi, int32_t *flags) {
+  if (batch < 0 || V <= 0 || row_stride < V) return ORACLE_ERR_ARG;
+  if (dtype != ORACLE_BF16 && dtype != ORACLE_F32) return ORACLE_ERR_ARG;
+  for (int r = 0; r < batch; ++r)
+    if (q_indptr[r + 1] - q_indptr[r] < 1) return ORACLE_ERR_ARG;
+  int status = ORACLE_OK;
+#pragma omp parallel
+  {
+    double *p = (double *)malloc(sizeof(double) * (size_t)V);
+    double *q = (double *)malloc(sizeof(double) * (size_t)V);
+    double *res = (double *)malloc(sizeof(double) * (size_t)V);
+    if (!p || !q || !res) {
+#pragma omp atomic write
+      status = ORACLE_ERR_ALLOC;
+    }
+#pragma omp for schedule(dynamic, 1)
+    for (int r = 0; r < batch; ++r) {
+      if (!p || !q || !res) continue;
+      const int st = sample_one(r, dtype, V, row_stride, target_logits, draft_logits, draft_ids,
+                                q_indptr, u_accept, u_sample, accepted_len, out_tokens, rho_out,
+                                resid_mass, cdf_lo, cdf_hi, flags, p, q, res);
+      if (st != ORACLE_OK) {
+#pragma omp atomic write
+        status = st;
+      }
+    }
+    free(p); free(q); free(res);
+  }
+  return status;
+}
+
+/*
+ * The distribution the emitted token of request r was drawn from, as the oracle computed it:
+ * cdf[0..V) = inclusive cumulative sum of the residual at row n (n < k) or of the target
+ * row k (n == k).  n is passed in (the oracle's accepted_len[r]).  Returns R.
+ */
+double oracle_emit_cdf(int32_t r, int32_t n, int64_t V, int64_t row_stride, int32_t dtype,
+                       const void *target_logits, const void *draft_logits,
+                       const int32_t *q_indptr, double *cdf) {
+  const int64_t t0 = q_indptr[r];
+  const int64_t d0 = (int64_t)q_indptr[r] - r;
+  const int k = q_indptr[r + 1] - q_indptr[r] - 1;
+  double *p = (double *)malloc(sizeof(double) * (size_t)V);
+  double *q = (double *)malloc(sizeof(double) * (size_t)V);
+  double R = NAN;
+  if (p && q) {
+    oracle_softmax_row(target_logits, dtype, (t0 + n) * row_stride, V, p);
+    if (n < k) {
+      oracle_softmax_row(draft_logits, dtype, (d0 + n) * row_stride, V, q);
+      R = oracle_residual(p, q, V, q);
+      if (R == 0.0) { R = 0.0; for (int64_t v = 0; v < V; ++v) { q[v] = p[v]; R += p[v]; } }
+      oracle_cumsum(q, V, cdf);
+    } else {
+      R = 0.0;
+      for (int64_t v = 0; v < V; ++v) R += p[v];
+      oracle_cumsum(p, V, cdf);
+    }
+  }
+  free(p); free(q);
+  return R;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* (C) the whole step: the two halves are independent given their inputs                  */
+/* ------------------------------------------------------------------------------------ */
+int oracle_verify_step(int32_t batch, int32_t Hq, int32_t Hkv, int32_t D, int32_t P,
+                       int64_t num_pages, int32_t max_pages_per_req, int32_t kv_dtype,
+                       double sm_scale, const void *q, const void *k_cache, const void *v_cache,
+                       int64_t stride_page, int64_t stride_head, int64_t stride_token,
+                       const int32_t *block_table, const int32_t *seq_lens,
+                       const int32_t *q_indptr, double *out, double *lse, int64_t V,
+                       int64_t row_stride, int32_t logits_dtype, const void *target_logits,
+                       const void *draft_logits, const int32_t *draft_ids, const float *u_accept,
+                       const float *u_sample, int32_t *accepted_len, int32_t *out_tokens) {
+  const int sa = oracle_verify_attention(batch, Hq, Hkv, D, P, num_pages, max_pages_per_req,
+                                         kv_dtype, sm_scale, q, k_cache, v_cache, stride_page,
+                                         stride_head, stride_token, block_table, seq_lens,
+                                         q_indptr, NULL, 0, out, lse);
+  if (sa != ORACLE_OK) return sa;
+  return oracle_rejection_sample(batch, V, row_stride, logits_dtype, target_logits, draft_logits,
+                                 draft_ids, q_indptr, u_accept, u_sample, accepted_len,
+                                 out_tokens, NULL, NULL, NULL, NULL, NULL);
+}
