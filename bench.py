@@ -1,0 +1,336 @@
+#!/usr/bin/env python
+"""Benchmark of the speculative-decoding verify step (one step = attention + rejection sampling
+for one batch of synthetic requests).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload I] [--impl reference]
+
+Prints ONE JSON line.  `value` is verified tokens per second (sum over requests of accepted+1,
+per step, over all GPUs) with inputs resident in HBM; `e2e` is the same metric through the
+host-buffer entry point with host<->device copies inside the timed region; `roofline` is the
+verify-attention kernel (the kernel that streams the KV cache) against the measured HBM copy
+bandwidth; `cpu_baseline` is the float64 CPU oracle timed on a bounded sample of the same
+workload.  With N > 1 (under torchrun) every rank runs an independent replica of the workload on
+its own GPU (the path has no exchange step), times are the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import spx_workloads as W  # noqa: E402
+
+METRIC = "verified_tokens_per_s"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one verify-attention launch, from the ncu
+# captures summarised under profiles/ (None until captured for that workload).
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if visible:
+                entry = visible.split(",")[index]
+                phys = int(entry) if entry.isdigit() else None
+            self.h = (pynvml.nvmlDeviceGetHandleByIndex(phys) if phys is not None
+                      else pynvml.nvmlDeviceGetHandleByUUID(entry))
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _poll(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while True:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            if self._stop.wait(0.002):
+                break
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._poll, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+        return {
+            "sm_mhz": statistics.median(self.samples) if self.samples else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": sorted(self.reasons),
+            "samples": len(self.samples),
+        }
+
+
+def sub_batch(b_cpu: W.VerifyBatch, n_req: int) -> W.VerifyBatch:
+    """The first n_req requests of a host batch (KV pools shared, not copied)."""
+    import dataclasses
+    qi = b_cpu.q_indptr.tolist()
+    tq, td = qi[n_req], qi[n_req] - n_req
+    return dataclasses.replace(
+        b_cpu, q=b_cpu.q[:tq], block_table=b_cpu.block_table[:n_req], seq_lens=b_cpu.seq_lens[:n_req],
+        q_indptr=b_cpu.q_indptr[:n_req + 1], target_logits=b_cpu.target_logits[:tq],
+        draft_logits=b_cpu.draft_logits[:td], draft_ids=b_cpu.draft_ids[:td], u_accept=b_cpu.u_accept[:td],
+        u_sample=b_cpu.u_sample[:n_req], seq_lens_host=b_cpu.seq_lens_host[:n_req], k_host=b_cpu.k_host[:n_req])
+
+
+def oracle_sample_size(spec: W.WorkloadSpec) -> int:
+    """Requests in the CPU-baseline sample: about 10-30 s of float64 work on ~8-32 cores."""
+    return {0: 4, 1: 16, 2: 16, 3: 1, 4: 16}.get(spec.index, min(spec.batch, 8))
+
+
+def time_oracle(b_cpu: W.VerifyBatch, n_req: int):
+    """One oracle pass over the sample.  Returns (seconds, verified tokens, threads)."""
+    import oracle
+    sb = sub_batch(b_cpu, n_req)
+    s = sb.spec
+    t0 = time.perf_counter()
+    oracle.verify_attention(sb.q, sb.k_cache, sb.v_cache, sb.kv_strides, sb.block_table, sb.seq_lens, sb.q_indptr,
+                            s.num_kv_heads, s.page_size, sb.num_pages)
+    res = oracle.rejection_sample(sb.target_logits, sb.draft_logits, sb.draft_ids, sb.q_indptr, sb.u_accept,
+                                  sb.u_sample)
+    dt = time.perf_counter() - t0
+    return dt, int(res.accepted_len.sum()) + n_req, oracle.num_threads()
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    spec = W.CONFIGS[args.workload]
+    b_cpu = W.generate(spec, device="cpu")
+    n_req = oracle_sample_size(spec)
+    for _ in range(args.warmup):
+        time_oracle(b_cpu, n_req)
+    total_t, tokens, threads = 0.0, 0, 1
+    for _ in range(args.steps):
+        dt, tok, threads = time_oracle(b_cpu, n_req)
+        total_t += dt
+        tokens += tok
+    value = tokens / total_t
+    sample = f"first {n_req} of {spec.batch} requests per step (attention + sampling, float64)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": spec.name, "batch": spec.batch, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", type=int, default=1, help="index into the five named workloads (default: Llama-3-8B shape)")
+    ap.add_argument("--impl", default="spx", choices=["spx", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps == 2000:
+            args.steps, args.warmup = 3, 1
+        run_reference(args)
+        return
+
+    import paper_2609_34370_b200 as spx
+    from paper_2609_34370_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the verify step has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    warmup = max(args.warmup, 3)
+
+    spec = W.CONFIGS[args.workload]
+    b = W.generate(spec, device=dev, seed=spec.seed + 1000 * rank)
+    out = torch.empty_like(b.q)
+    lse = torch.empty(b.q.shape[:2], dtype=torch.float32, device=dev)
+    acc = torch.empty(b.batch, dtype=torch.int32, device=dev)
+    tok = torch.empty(b.total_q, dtype=torch.int32, device=dev)
+    a = binding.make_attn_args(b.q, b.k_cache, b.v_cache, b.kv_strides, b.block_table, b.seq_lens, b.q_indptr,
+                               spec.num_kv_heads, spec.page_size, b.num_pages, out, lse, max_q_len=max(b.k_host) + 1)
+    s = binding.make_sample_args(b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample,
+                                 acc, tok)
+    ws = spx.Workspace.allocate(spx.workspace_size(a, s), dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    for _ in range(warmup):
+        spx.verify_step(a, s, ws, dev)
+    torch.cuda.synchronize()
+    launches_per_step = spx.last_launch_count()
+    tokens_per_step = int(acc.sum().item()) + b.batch
+    if int(ws.status.item()) != 0:
+        raise SystemExit(f"device status {int(ws.status.item())} after warm-up")
+
+    # per-step event pairs around the verify-attention kernel (handles must exist before use)
+    k_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                for _ in range(args.steps)]
+    for e0, e1 in k_events:
+        e0.record()
+        e1.record()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    clocks = ClockSampler(local)
+    barrier()
+    torch.cuda.synchronize()
+    clocks.start()
+    ev0.record()
+    for e0, e1 in k_events:
+        spx.set_timing_events(e0, e1)
+        spx.verify_step(a, s, ws, dev)
+    ev1.record()
+    torch.cuda.synchronize()
+    clock_info = clocks.stop()
+    spx.set_timing_events(None, None)
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    attn_ms = [e0.elapsed_time(e1) for e0, e1 in k_events]
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    toks = torch.tensor([tokens_per_step], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
+    ms_total = float(t.item())
+    value = float(toks.item()) * args.steps / (ms_total * 1e-3)
+    ms_per_step = ms_total / args.steps
+
+    # ---- end to end through the host-buffer entry point (every rank, max time) ----
+    b_host = None
+    e2e = None
+    try:
+        b_host = b.to("cpu")
+        pin = {n: getattr(b_host, n).pin_memory() for n in W.VerifyBatch._TENSORS}
+        out_h = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+        acc_h = torch.empty(acc.shape, dtype=torch.int32).pin_memory()
+        tok_h = torch.empty(tok.shape, dtype=torch.int32).pin_memory()
+        st_h = torch.zeros(1, dtype=torch.int32).pin_memory()
+        ah = binding.make_attn_args(pin["q"], pin["k_cache"], pin["v_cache"], b.kv_strides, pin["block_table"],
+                                    pin["seq_lens"], pin["q_indptr"], spec.num_kv_heads, spec.page_size, b.num_pages,
+                                    out_h, None, max_q_len=max(b.k_host) + 1)
+        sh = binding.make_sample_args(pin["target_logits"], pin["draft_logits"], pin["draft_ids"], pin["q_indptr"],
+                                      pin["u_accept"], pin["u_sample"], acc_h, tok_h)
+        pool_elems = b.k_cache.numel()
+        arena = torch.empty(spx.host_step_arena_size(ah, sh, pool_elems), dtype=torch.uint8, device=dev)
+        for _ in range(2):
+            spx.verify_step_host(ah, sh, pool_elems, arena, st_h, dev)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(args.e2e_steps):
+            spx.verify_step_host(ah, sh, pool_elems, arena, st_h, dev)
+        e1.record()
+        torch.cuda.synchronize()
+        te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        assert int(st_h.item()) == 0 and torch.equal(acc_h, acc.cpu()) and torch.equal(tok_h, tok.cpu())
+        h2d = sum(pin[n].numel() * pin[n].element_size() for n in W.VerifyBatch._TENSORS)
+        d2h = out_h.numel() * out_h.element_size() + acc_h.numel() * 4 + tok_h.numel() * 4 + 4
+        e2e = {"value": float(toks.item()) * args.e2e_steps / (float(te.item()) * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
+        del arena, pin
+    except Exception as exc:  # reported, never hidden
+        e2e = {"value": None, "unit": UNIT, "error": repr(exc)}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    kv_bytes, logit_bytes = b.kv_bytes(), b.logits_bytes()
+    attn_avg_ms = sum(attn_ms) / len(attn_ms)
+    achieved = kv_bytes / (attn_avg_ms * 1e-3) / 1e9
+    step_gbs = (kv_bytes + logit_bytes) / (ms_per_step * 1e-3) / 1e9
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": spec.dtype, "data": "synthetic",
+        "config": {"workload": spec.name, "batch": spec.batch, "q_heads": spec.num_q_heads,
+                   "kv_heads": spec.num_kv_heads, "head_dim": spec.head_dim, "page_size": spec.page_size,
+                   "vocab": spec.vocab, "total_q_rows": b.total_q, "kv_tokens": sum(b.seq_lens_host),
+                   "kv_bytes": kv_bytes, "logits_bytes": logit_bytes, "tokens_per_step": tokens_per_step,
+                   "l2": "inputs larger than L2 (KV + logits re-read from HBM every step)",
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "clocks": clock_info,
+        "e2e": e2e,
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "verify-attention", "achieved": achieved, "peak": peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": NCU_TRAFFIC_BYTES.get(spec.name), "algorithmic_bytes": kv_bytes,
+                     "avg_launch_ms": attn_avg_ms},
+        "step_hbm": {"bytes": kv_bytes + logit_bytes, "achieved_gbs": step_gbs,
+                     "frac_of_measured": step_gbs / peak, "frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS},
+    }
+    if not args.no_cpu_baseline:
+        try:
+            n_req = oracle_sample_size(spec)
+            dt, otok, threads = time_oracle(b_host if b_host is not None else b.to("cpu"), n_req)
+            result["cpu_baseline"] = {"value": otok / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                      "sample": f"first {n_req} of {spec.batch} requests, one pass ({dt:.1f} s)"}
+        except Exception as exc:
+            result["cpu_baseline"] = {"value": None, "unit": UNIT, "error": repr(exc), "kind": "oracle"}
+    print(json.dumps(result))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,187 @@
+/*
+ * spx.h - C ABI of libspx: the speculative-decoding verify step on one NVIDIA B200 (sm_100a).
+ *
+ * The verify step is the per-iteration GPU work underneath speculative(-parallel) scheduling:
+ * a batch of requests each carries k_r >= 0 draft tokens (k_r = 0 where selective speculation,
+ * Section 5.1 of the paper, switched speculation off for that request); the target model's
+ * k_r+1 new positions attend jointly over the request's paged, shared KV cache (Section 2
+ * "Speculative decoding", Section 4 "Self-speculation and parallel scheduling": drafts are
+ * "verified jointly", the cache is shared between speculative and normal execution), and the
+ * drafts are then accepted or rejected by speculative sampling (the rule of the
+ * speculative-decoding work cited in Section 2).
+ *
+ * Conventions for every entry point
+ *   - Pointers inside the argument structs are DEVICE pointers unless the field name ends in
+ *     _host.  The structs themselves, `ws_bytes` and all scalars live on the host.
+ *   - The caller owns every buffer and the CUDA stream (`cuda_stream` is a cudaStream_t passed
+ *     as void*; NULL = the legacy default stream).  The library allocates no device memory.
+ *   - Calls only enqueue work on the stream and return; nothing synchronises the device.
+ *   - Host-visible argument errors return a non-zero spx_status_t and launch nothing.
+ *   - Errors in device-resident data (a page id out of range, a draft token id >= vocab, a
+ *     context shorter than its query count) cannot be seen by the host without a sync: they OR
+ *     a SPX_DEV_* bit into *dev_status (a caller-owned int32 on the device, which the caller
+ *     zeroes and reads back when it wants), the affected request gets sentinel outputs
+ *     (attention rows zero, lse NaN; accepted_len 0 and out_tokens -1) and the other requests
+ *     are unaffected.  No kernel traps, asserts or waits without bound.
+ *   - `ws` is scratch of at least spx_workspace_size(...) bytes, 256-byte aligned.  Its
+ *     contents are meaningless between calls.  Two calls may overlap on the device only if
+ *     they use different workspaces.
+ *   - bf16 means the upper half of an IEEE binary32 (round-to-nearest-even on output).
+ */
+#ifndef SPX_H_
+#define SPX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPX_MAX_K 15            /* at most 15 draft tokens (16 query positions) per request   */
+#define SPX_MAX_PACKED_ROWS 128 /* (num_q_heads / num_kv_heads) * (k+1) must not exceed this  */
+
+typedef enum {
+  SPX_OK = 0,
+  SPX_ERR_INVALID_ARG = 1, /* NULL where a pointer is required, negative size, misalignment  */
+  SPX_ERR_UNSUPPORTED = 2, /* shape outside what the kernels implement (see each call)        */
+  SPX_ERR_WORKSPACE = 3,   /* ws is NULL, misaligned or smaller than spx_workspace_size       */
+  SPX_ERR_CUDA = 4         /* a CUDA runtime/driver call failed (launch error, no sm_100 GPU) */
+} spx_status_t;
+
+/* Bits OR-ed into *dev_status by the kernels. */
+enum {
+  SPX_DEV_BAD_PAGE = 1,   /* a needed block-table entry was outside [0, num_pages)            */
+  SPX_DEV_BAD_TOKEN = 2,  /* a draft token id was outside [0, vocab)                          */
+  SPX_DEV_BAD_LEN = 4,    /* seq_len < k+1, k+1 outside [1, max_q_len], or too many pages     */
+  SPX_DEV_TIMEOUT = 8,    /* a bounded wait inside a kernel gave up                           */
+  SPX_DEV_DEGENERATE = 16 /* residual mass was zero; the target row was sampled instead       */
+};
+
+typedef enum { SPX_BF16 = 0, SPX_F32 = 1 } spx_dtype_t;
+
+/*
+ * Attention half.  For request r with m_r = q_indptr[r+1]-q_indptr[r] = k_r+1 query rows and
+ * L_r = seq_lens[r] cached tokens (the m_r new positions INCLUDED, their K/V already written),
+ * query j (0 <= j < m_r), q-head h, kv-head g = h / (num_q_heads/num_kv_heads):
+ *     visible tokens t = 0 .. L_r - m_r + j            (causal among the new positions)
+ *     s_t = sm_scale * <Q[q_indptr[r]+j, h, :], K[r, t, g, :]>
+ *     out[q_indptr[r]+j, h, :] = sum_t softmax_t(s)_t * V[r, t, g, :]
+ *     lse[q_indptr[r]+j, h]    = log sum_t exp(s_t)       (natural log)
+ * Token t of request r lives in page block_table[r*max_pages_per_req + t/page_size], slot
+ * t % page_size; element (page, g, slot, d) of a pool is at
+ *     page*kv_stride_page + g*kv_stride_head + slot*kv_stride_token + d        (elements).
+ * Slots past L_r and block-table entries past ceil(L_r/page_size) are never read.
+ *
+ * Supported: head_dim 64 or 128; num_q_heads a multiple of num_kv_heads with
+ * (num_q_heads/num_kv_heads)*max_q_len <= SPX_MAX_PACKED_ROWS; page_size a power of two in
+ * 1..128; kv_dtype BF16 (tensor-core path; pools and strides 16-byte aligned) or F32 (true fp32
+ * arithmetic).  Accumulation is fp32 in both.
+ */
+typedef struct {
+  int32_t batch;             /* B >= 0                                                        */
+  int32_t total_q;           /* TQ = q_indptr[B] = rows of q/out (host copy of that number)   */
+  int32_t max_q_len;         /* upper bound on k_r+1 over the batch, 1..SPX_MAX_K+1; 0 = 16   */
+  int32_t num_q_heads, num_kv_heads, head_dim, page_size;
+  int32_t num_pages;         /* pages in each pool                                            */
+  int32_t max_pages_per_req; /* row length of block_table                                     */
+  spx_dtype_t kv_dtype;      /* dtype of q, k_cache, v_cache and out                          */
+  float sm_scale;            /* 0 => 1/sqrt(head_dim)                                         */
+  const void *q;             /* [TQ, num_q_heads, head_dim] contiguous                        */
+  const void *k_cache;       /* K pool                                                        */
+  const void *v_cache;       /* V pool (same strides)                                         */
+  int64_t kv_stride_page, kv_stride_head, kv_stride_token; /* elements; head_dim contiguous   */
+  const int32_t *block_table; /* [B, max_pages_per_req]                                       */
+  const int32_t *seq_lens;    /* [B]                                                          */
+  const int32_t *q_indptr;    /* [B+1], q_indptr[0] = 0, non-decreasing                       */
+  void *out;                  /* [TQ, num_q_heads, head_dim], written                         */
+  float *lse;                 /* [TQ, num_q_heads], written; may be NULL                      */
+} spx_attn_args_t;
+
+/*
+ * Sampling half.  Request r has target rows T_0..T_k (rows q_indptr[r] .. q_indptr[r]+k of
+ * target_logits), draft rows D_0..D_{k-1} (rows q_indptr[r]-r .. of draft_logits), draft ids
+ * x_i and uniforms a_i at the same indices as the draft rows, and one uniform s = u_sample[r].
+ * With p_i = softmax(T_i), q_i = softmax(D_i) over the whole vocabulary at temperature 1:
+ *   for i = 0..k-1 in order: accept x_i iff a_i < p_i(x_i)/q_i(x_i); stop at the first failure, n = i;
+ *   if n < k : y = invCDF over r(v) = max(0, p_n(v) - q_n(v)), i.e. the first v (ascending id)
+ *              whose inclusive cumulative sum exceeds s * sum_v r(v);
+ *   if n = k : y = the same inverse CDF over p_k (the bonus token);
+ *   accepted_len[r] = n; out_tokens[q_indptr[r] ..] = x_0..x_{n-1}, y, then -1 up to k+1 slots.
+ * Logits rows after n are never needed.  Arithmetic: fp32 exponentials and in-segment sums,
+ * float64 across segments and for the accept ratio.
+ *
+ * Supported: vocab >= 1; logits_row_stride >= vocab and a multiple of 8 (BF16) or 4 (F32)
+ * elements; both logits pointers 16-byte aligned.
+ */
+typedef struct {
+  int32_t batch;               /* B >= 0                                                      */
+  int32_t total_q;             /* TQ = q_indptr[B]; draft rows TD = TQ - B                    */
+  int32_t vocab;
+  int64_t logits_row_stride;   /* elements, same for target and draft                         */
+  spx_dtype_t logits_dtype;
+  const void *target_logits;   /* [TQ, vocab]                                                 */
+  const void *draft_logits;    /* [TD, vocab]; may be NULL when TD = 0                        */
+  const int32_t *draft_token_ids; /* [TD]                                                     */
+  const int32_t *q_indptr;     /* [B+1]                                                       */
+  const float *u_accept;       /* [TD], each in [0,1)                                         */
+  const float *u_sample;       /* [B], each in [0,1)                                          */
+  int32_t *accepted_len;       /* [B], written                                                */
+  int32_t *out_tokens;         /* [TQ], written                                               */
+  float *diag_ratio;           /* optional [TD]: p/q of each consulted draft (NaN otherwise)  */
+} spx_sample_args_t;
+
+/*
+ * Bytes of scratch the calls below need for these arguments (host integers only are read;
+ * either pointer may be NULL to size one half alone).  Returns 0 on invalid arguments.
+ */
+size_t spx_workspace_size(const spx_attn_args_t *attn, const spx_sample_args_t *sample);
+
+/* The attention half alone (see spx_attn_args_t). */
+spx_status_t spx_verify_attention(const spx_attn_args_t *args, void *ws, size_t ws_bytes,
+                                  int32_t *dev_status, void *cuda_stream);
+
+/* The sampling half alone (see spx_sample_args_t). */
+spx_status_t spx_rejection_sample(const spx_sample_args_t *args, void *ws, size_t ws_bytes,
+                                  int32_t *dev_status, void *cuda_stream);
+
+/*
+ * The whole verify step: both halves on the caller's stream.  The halves are independent given
+ * their inputs (logits are inputs here), so the library may interleave them.  `ws` must hold
+ * spx_workspace_size(attn, sample) bytes.
+ */
+spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_t *sample, void *ws,
+                             size_t ws_bytes, int32_t *dev_status, void *cuda_stream);
+
+/*
+ * Convenience for callers whose data lives on the HOST: every pointer in the two structs is a
+ * host pointer (pinned memory recommended); device staging buffers, the workspace and the
+ * status word are carved from `dev_arena` (device memory, `arena_bytes` >=
+ * spx_host_step_arena_size).  Copies inputs host->device, runs spx_verify_step, copies
+ * out/lse/accepted_len/out_tokens and the status word back, all on `cuda_stream`, and returns
+ * after enqueueing; *dev_status_host is valid after the stream is synchronised.  `kv_pool_elems`
+ * is the number of elements of each KV pool to copy.
+ */
+size_t spx_host_step_arena_size(const spx_attn_args_t *attn, const spx_sample_args_t *sample,
+                                int64_t kv_pool_elems);
+spx_status_t spx_verify_step_host(const spx_attn_args_t *attn, const spx_sample_args_t *sample,
+                                  int64_t kv_pool_elems, void *dev_arena, size_t arena_bytes,
+                                  int32_t *dev_status_host, void *cuda_stream);
+
+const char *spx_status_string(spx_status_t status);
+
+/*
+ * Measurement aid.  While a pair of cudaEvent_t (created by the caller with timing enabled) is
+ * set on the calling thread, every spx_verify_attention / spx_verify_step call from that thread
+ * records `start` immediately before and `stop` immediately after its verify-attention kernel
+ * (the kernel that streams the KV cache) on the call's stream.  Pass NULL, NULL to clear.
+ */
+void spx_set_timing_events(void *start_event, void *stop_event);
+
+/* Number of kernels the last call on this thread enqueued (for launch accounting). */
+int32_t spx_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPX_H_ */

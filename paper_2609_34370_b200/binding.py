@@ -1,0 +1,257 @@
+"""ctypes binding of include/spx.h.  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional, Tuple
+
+import torch
+
+from .build import LIB_PATH
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = 0, 1, 2, 3, 4
+DEV_BAD_PAGE, DEV_BAD_TOKEN, DEV_BAD_LEN, DEV_TIMEOUT, DEV_DEGENERATE = 1, 2, 4, 8, 16
+BF16, F32 = 0, 1
+
+EXPORTS = ("spx_workspace_size", "spx_verify_attention", "spx_rejection_sample", "spx_verify_step",
+           "spx_host_step_arena_size", "spx_verify_step_host", "spx_status_string", "spx_last_launch_count",
+           "spx_set_timing_events")
+
+
+class AttnArgs(C.Structure):
+    _fields_ = [
+        ("batch", C.c_int32), ("total_q", C.c_int32), ("max_q_len", C.c_int32),
+        ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+        ("page_size", C.c_int32), ("num_pages", C.c_int32), ("max_pages_per_req", C.c_int32),
+        ("kv_dtype", C.c_int), ("sm_scale", C.c_float),
+        ("q", C.c_void_p), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+        ("kv_stride_page", C.c_int64), ("kv_stride_head", C.c_int64), ("kv_stride_token", C.c_int64),
+        ("block_table", C.c_void_p), ("seq_lens", C.c_void_p), ("q_indptr", C.c_void_p),
+        ("out", C.c_void_p), ("lse", C.c_void_p),
+    ]
+
+
+class SampleArgs(C.Structure):
+    _fields_ = [
+        ("batch", C.c_int32), ("total_q", C.c_int32), ("vocab", C.c_int32),
+        ("logits_row_stride", C.c_int64), ("logits_dtype", C.c_int),
+        ("target_logits", C.c_void_p), ("draft_logits", C.c_void_p), ("draft_token_ids", C.c_void_p),
+        ("q_indptr", C.c_void_p), ("u_accept", C.c_void_p), ("u_sample", C.c_void_p),
+        ("accepted_len", C.c_void_p), ("out_tokens", C.c_void_p), ("diag_ratio", C.c_void_p),
+    ]
+
+
+class SpxError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"libspx: {what} (status {code})")
+        self.code = code
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return LIB_PATH
+
+
+def load_library():
+    """Load libspx.so; raises if it has not been built (there is no other implementation)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise SpxError(-1, f"{LIB_PATH} is missing: run paper_2609_34370_b200.build.build() "
+                               "(or __graft_entry__.build()) first")
+        lib = C.CDLL(LIB_PATH)
+        lib.spx_workspace_size.restype = C.c_size_t
+        lib.spx_workspace_size.argtypes = [C.POINTER(AttnArgs), C.POINTER(SampleArgs)]
+        for name in ("spx_verify_attention", "spx_rejection_sample"):
+            fn = getattr(lib, name)
+            fn.restype = C.c_int
+            fn.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        lib.spx_verify_step.restype = C.c_int
+        lib.spx_verify_step.argtypes = [C.POINTER(AttnArgs), C.POINTER(SampleArgs), C.c_void_p, C.c_size_t,
+                                        C.c_void_p, C.c_void_p]
+        lib.spx_host_step_arena_size.restype = C.c_size_t
+        lib.spx_host_step_arena_size.argtypes = [C.POINTER(AttnArgs), C.POINTER(SampleArgs), C.c_int64]
+        lib.spx_verify_step_host.restype = C.c_int
+        lib.spx_verify_step_host.argtypes = [C.POINTER(AttnArgs), C.POINTER(SampleArgs), C.c_int64, C.c_void_p,
+                                             C.c_size_t, C.c_void_p, C.c_void_p]
+        lib.spx_status_string.restype = C.c_char_p
+        lib.spx_status_string.argtypes = [C.c_int]
+        lib.spx_last_launch_count.restype = C.c_int32
+        lib.spx_set_timing_events.restype = None
+        lib.spx_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
+        _lib = lib
+    return _lib
+
+
+def exported_symbols() -> Tuple[str, ...]:
+    return EXPORTS
+
+
+def _check(code: int):
+    if code != OK:
+        raise SpxError(code, load_library().spx_status_string(code).decode())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError(f"bf16 or fp32 expected, got {t.dtype}")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None or t.numel() == 0 else t.data_ptr()
+
+
+def _stream(device) -> int:
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+def _require_cuda(*tensors):
+    for t in tensors:
+        if t is not None and t.device.type != "cuda":
+            raise SpxError(ERR_INVALID_ARG, "device tensors required (there is no CPU path)")
+
+
+def make_attn_args(q, k_cache, v_cache, kv_strides, block_table, seq_lens, q_indptr, num_kv_heads, page_size,
+                   num_pages, out, lse=None, sm_scale=0.0, max_q_len=0) -> AttnArgs:
+    TQ, Hq, D = q.shape
+    a = AttnArgs()
+    a.batch = seq_lens.numel()
+    a.total_q = TQ
+    a.max_q_len = max_q_len
+    a.num_q_heads, a.num_kv_heads, a.head_dim, a.page_size = Hq, num_kv_heads, D, page_size
+    a.num_pages = num_pages
+    a.max_pages_per_req = block_table.shape[1] if block_table.dim() == 2 else 0
+    a.kv_dtype = _dtype_code(q)
+    a.sm_scale = sm_scale
+    a.q, a.k_cache, a.v_cache = _ptr(q), _ptr(k_cache), _ptr(v_cache)
+    a.kv_stride_page, a.kv_stride_head, a.kv_stride_token = (int(x) for x in kv_strides)
+    a.block_table, a.seq_lens, a.q_indptr = _ptr(block_table), _ptr(seq_lens), q_indptr.data_ptr()
+    a.out, a.lse = _ptr(out), _ptr(lse)
+    return a
+
+
+def make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, accepted_len,
+                     out_tokens, diag_ratio=None, vocab=None) -> SampleArgs:
+    s = SampleArgs()
+    s.batch = q_indptr.numel() - 1
+    s.total_q = target_logits.shape[0]
+    s.vocab = int(vocab if vocab is not None else target_logits.shape[1])
+    s.logits_row_stride = target_logits.stride(0)
+    s.logits_dtype = _dtype_code(target_logits)
+    s.target_logits, s.draft_logits = _ptr(target_logits), _ptr(draft_logits)
+    s.draft_token_ids, s.q_indptr = _ptr(draft_ids), q_indptr.data_ptr()
+    s.u_accept, s.u_sample = _ptr(u_accept), _ptr(u_sample)
+    s.accepted_len, s.out_tokens, s.diag_ratio = _ptr(accepted_len), _ptr(out_tokens), _ptr(diag_ratio)
+    return s
+
+
+def workspace_size(attn: Optional[AttnArgs], sample: Optional[SampleArgs]) -> int:
+    lib = load_library()
+    n = lib.spx_workspace_size(C.byref(attn) if attn is not None else None,
+                               C.byref(sample) if sample is not None else None)
+    if n == 0:
+        raise SpxError(ERR_INVALID_ARG, "invalid arguments for workspace sizing")
+    return int(n)
+
+
+@dataclass
+class Workspace:
+    """Caller-owned scratch and status word (torch is used for the allocation only)."""
+    buf: torch.Tensor
+    status: torch.Tensor
+
+    @staticmethod
+    def allocate(nbytes: int, device) -> "Workspace":
+        return Workspace(torch.empty(nbytes, dtype=torch.uint8, device=device),
+                         torch.zeros(1, dtype=torch.int32, device=device))
+
+    def ensure(self, nbytes: int):
+        if self.buf.numel() < nbytes:
+            self.buf = torch.empty(nbytes, dtype=torch.uint8, device=self.buf.device)
+
+
+def verify_attention(q, k_cache, v_cache, kv_strides, block_table, seq_lens, q_indptr, num_kv_heads, page_size,
+                     num_pages, out=None, lse=None, sm_scale=0.0, max_q_len=0, ws: Optional[Workspace] = None,
+                     want_lse=True):
+    """spx_verify_attention on the current stream.  Returns (out, lse, ws)."""
+    _require_cuda(q, k_cache, v_cache, block_table, seq_lens, q_indptr)
+    lib = load_library()
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None and want_lse:
+        lse = torch.empty(q.shape[:2], dtype=torch.float32, device=q.device)
+    a = make_attn_args(q, k_cache, v_cache, kv_strides, block_table, seq_lens, q_indptr, num_kv_heads, page_size,
+                       num_pages, out, lse, sm_scale, max_q_len)
+    need = workspace_size(a, None)
+    if ws is None:
+        ws = Workspace.allocate(need, q.device)
+    ws.ensure(need)
+    _check(lib.spx_verify_attention(C.byref(a), ws.buf.data_ptr(), ws.buf.numel(), ws.status.data_ptr(),
+                                    _stream(q.device)))
+    return out, lse, ws
+
+
+def rejection_sample(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, vocab=None,
+                     want_ratio=False, ws: Optional[Workspace] = None):
+    """spx_rejection_sample on the current stream.  Returns (accepted_len, out_tokens, ratio, ws)."""
+    _require_cuda(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample)
+    lib = load_library()
+    dev = target_logits.device
+    B = q_indptr.numel() - 1
+    TQ = target_logits.shape[0]
+    accepted = torch.empty(B, dtype=torch.int32, device=dev)
+    tokens = torch.empty(TQ, dtype=torch.int32, device=dev)
+    ratio = torch.empty(TQ - B, dtype=torch.float32, device=dev) if want_ratio else None
+    s = make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, accepted, tokens,
+                         ratio, vocab)
+    need = workspace_size(None, s)
+    if ws is None:
+        ws = Workspace.allocate(need, dev)
+    ws.ensure(need)
+    _check(lib.spx_rejection_sample(C.byref(s), ws.buf.data_ptr(), ws.buf.numel(), ws.status.data_ptr(),
+                                    _stream(dev)))
+    return accepted, tokens, ratio, ws
+
+
+def verify_step(attn: AttnArgs, sample: SampleArgs, ws: Workspace, device):
+    """spx_verify_step with prebuilt argument structs (the benchmark's hot call)."""
+    lib = load_library()
+    _check(lib.spx_verify_step(C.byref(attn), C.byref(sample), ws.buf.data_ptr(), ws.buf.numel(),
+                               ws.status.data_ptr(), _stream(device)))
+
+
+def verify_step_host(attn: AttnArgs, sample: SampleArgs, kv_pool_elems: int, arena: torch.Tensor,
+                     status_host: torch.Tensor, device):
+    """spx_verify_step_host: every pointer in the structs is a host pointer."""
+    lib = load_library()
+    _check(lib.spx_verify_step_host(C.byref(attn), C.byref(sample), int(kv_pool_elems), arena.data_ptr(),
+                                    arena.numel(), status_host.data_ptr(), _stream(device)))
+
+
+def host_step_arena_size(attn: AttnArgs, sample: SampleArgs, kv_pool_elems: int) -> int:
+    n = load_library().spx_host_step_arena_size(C.byref(attn), C.byref(sample), int(kv_pool_elems))
+    if n == 0:
+        raise SpxError(ERR_INVALID_ARG, "invalid arguments for arena sizing")
+    return int(n)
+
+
+def last_launch_count() -> int:
+    return int(load_library().spx_last_launch_count())
+
+
+def set_timing_events(start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]):
+    """Record `start`/`stop` around the verify-attention kernel of later calls (None, None clears).
+
+    The events must have been recorded once already so that their CUDA handles exist.
+    """
+    lib = load_library()
+    if start is None or stop is None:
+        lib.spx_set_timing_events(None, None)
+    else:
+        lib.spx_set_timing_events(start.cuda_event, stop.cuda_event)

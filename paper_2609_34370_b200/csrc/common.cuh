@@ -1,0 +1,90 @@
+// Shared device helpers for the verify-step kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "spx.h"
+
+namespace spx {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kTileTokens = 128;   // KV tokens per attention tile (both attention kernels plan in this unit)
+constexpr int kPlanWaves = 8;      // target number of work chunks per SM
+
+__device__ __forceinline__ float ld_as_float(const float *p, int64_t i) { return p[i]; }
+__device__ __forceinline__ float ld_as_float(const __nv_bfloat16 *p, int64_t i) { return __bfloat162float(p[i]); }
+
+__device__ __forceinline__ void st_from_float(float *p, int64_t i, float v) { p[i] = v; }
+__device__ __forceinline__ void st_from_float(__nv_bfloat16 *p, int64_t i, float v) { p[i] = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ------------------------------------------------------------------------------------------
+// Work plan shared by the attention kernels.  Built on the device by plan_kernel so that no
+// host copy of seq_lens is needed.
+//
+// Each request's KV range is cut into tiles of kTileTokens tokens and the tiles into
+// n_chunks[r] balanced chunks of at most chunk_tiles tiles; one work entry is one
+// (request, chunk) and is executed once per kv-head.  Entries are ordered by decreasing size
+// so that the dynamic scheduler (an atomic counter) approximates longest-processing-time-first.
+// ------------------------------------------------------------------------------------------
+struct PlanHeader {
+  int32_t n_work;        // number of (request, chunk) entries
+  int32_t chunk_tiles;   // largest chunk, in tiles
+  int32_t n_part_slots;  // partial-result slots in use (chunks of split requests)
+  int32_t total_tiles;   // sum over requests of tiles (one kv-head)
+  int32_t work_counter;  // dynamic scheduler cursor, zeroed by the planner
+  int32_t overflow;      // 1 if the plan did not fit the workspace (nothing is executed then)
+  int32_t pad[2];
+};
+
+struct WorkEntry {
+  int32_t req;         // request index
+  int32_t tile_begin;  // first tile of the chunk
+  int32_t tile_end;    // one past the last tile
+  int32_t part_slot;   // partial slot, or -1 when the request is not split (direct output)
+};
+
+struct AttnParams {
+  int32_t batch, total_q, max_q_len, Hq, Hkv, G, D, P, log2P, num_pages, max_pages_per_req;
+  float scale_log2;  // sm_scale * log2(e)
+  const void *q;
+  const void *k_cache;
+  const void *v_cache;
+  int64_t stride_page, stride_head, stride_token;
+  const int32_t *block_table;
+  const int32_t *seq_lens;
+  const int32_t *q_indptr;
+  void *out;
+  float *lse;
+  // plan + partials (workspace)
+  PlanHeader *hdr;
+  int32_t *req_nchunks;    // [B]  0 = invalid request
+  int32_t *req_part_base;  // [B]
+  WorkEntry *work;         // [max_work]
+  WorkEntry *work_tmp;     // [max_work]
+  int32_t max_work;
+  float *part_o;           // [slot][Hkv][rows_cap][D]
+  float2 *part_ml;         // [slot][Hkv][rows_cap]  (m in log2 domain, l)
+  int32_t rows_cap;        // G * max_q_len
+  int32_t *dev_status;
+};
+
+}  // namespace spx

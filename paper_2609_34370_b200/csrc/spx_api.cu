@@ -1,0 +1,385 @@
+// libspx: C ABI, argument validation, workspace layout and kernel launches.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+
+#include "attn_simt.cuh"
+#include "common.cuh"
+#include "plan.cuh"
+#include "sampler.cuh"
+#include "spx.h"
+
+namespace spx {
+
+static thread_local int32_t t_launches = 0;
+static thread_local cudaEvent_t t_ev_start = nullptr, t_ev_stop = nullptr;
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct DeviceInfo {
+  int device = -1;
+  int num_sms = 0;
+  int cc_major = 0;
+  int max_smem_optin = 0;
+};
+
+// Properties of the current device (queried per call: cheap attribute reads, no global state).
+static bool get_device_info(DeviceInfo *info) {
+  if (cudaGetDevice(&info->device) != cudaSuccess) return false;
+  if (cudaDeviceGetAttribute(&info->num_sms, cudaDevAttrMultiProcessorCount, info->device) != cudaSuccess) return false;
+  if (cudaDeviceGetAttribute(&info->cc_major, cudaDevAttrComputeCapabilityMajor, info->device) != cudaSuccess) return false;
+  if (cudaDeviceGetAttribute(&info->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, info->device) != cudaSuccess) return false;
+  return true;
+}
+
+constexpr int kPlanSmCount = 148;  // workspace sizing must not depend on a device query
+
+// ---------------------------------------------------------------------------------------------
+// workspace layout
+// ---------------------------------------------------------------------------------------------
+struct AttnWs {
+  size_t hdr, nchunks, part_base, work, work_tmp, part_ml, part_o, total;
+  int32_t max_work, rows_cap;
+};
+
+static spx_status_t check_attn(const spx_attn_args_t *a, bool need_ptrs) {
+  if (!a) return SPX_ERR_INVALID_ARG;
+  if (a->batch < 0 || a->total_q < a->batch || a->num_q_heads <= 0 || a->num_kv_heads <= 0 || a->head_dim <= 0 ||
+      a->page_size <= 0 || a->num_pages < 0 || a->max_pages_per_req < 0 || a->max_q_len < 0)
+    return SPX_ERR_INVALID_ARG;
+  if (a->kv_dtype != SPX_BF16 && a->kv_dtype != SPX_F32) return SPX_ERR_INVALID_ARG;
+  if (!(a->sm_scale >= 0.f) || std::isinf(a->sm_scale)) return SPX_ERR_INVALID_ARG;
+  if (a->head_dim != 64 && a->head_dim != 128) return SPX_ERR_UNSUPPORTED;
+  if (a->num_q_heads % a->num_kv_heads != 0) return SPX_ERR_UNSUPPORTED;
+  if (a->page_size > 128 || (a->page_size & (a->page_size - 1)) != 0) return SPX_ERR_UNSUPPORTED;
+  const int max_q = a->max_q_len == 0 ? SPX_MAX_K + 1 : a->max_q_len;
+  if (max_q > SPX_MAX_K + 1) return SPX_ERR_UNSUPPORTED;
+  if ((a->num_q_heads / a->num_kv_heads) * max_q > SPX_MAX_PACKED_ROWS) return SPX_ERR_UNSUPPORTED;
+  if (a->kv_stride_page < 0 || a->kv_stride_head < 0 || a->kv_stride_token < a->head_dim) return SPX_ERR_INVALID_ARG;
+  if (need_ptrs && a->batch > 0) {
+    if (!a->q || !a->k_cache || !a->v_cache || !a->block_table || !a->seq_lens || !a->q_indptr || !a->out)
+      return SPX_ERR_INVALID_ARG;
+    const int es = a->kv_dtype == SPX_BF16 ? 2 : 4;
+    if (((uintptr_t)a->q | (uintptr_t)a->k_cache | (uintptr_t)a->v_cache | (uintptr_t)a->out) & 15) return SPX_ERR_INVALID_ARG;
+    if (((a->kv_stride_page * es) | (a->kv_stride_head * es) | (a->kv_stride_token * es)) & 15) return SPX_ERR_INVALID_ARG;
+  }
+  return SPX_OK;
+}
+
+static AttnWs attn_ws_layout(const spx_attn_args_t *a) {
+  AttnWs w{};
+  const int max_q = a->max_q_len == 0 ? SPX_MAX_K + 1 : a->max_q_len;
+  const int G = a->num_q_heads / a->num_kv_heads;
+  w.rows_cap = G * max_q;
+  // sum_r ceil(tiles_r / c) <= sum_r tiles_r / c + B with c >= total*Hkv / (sms*waves)
+  w.max_work = a->batch + kPlanSmCount * kPlanWaves + 1;
+  size_t off = 0;
+  w.hdr = off; off = align_up(off + sizeof(PlanHeader), 256);
+  w.nchunks = off; off = align_up(off + sizeof(int32_t) * (size_t)a->batch, 256);
+  w.part_base = off; off = align_up(off + sizeof(int32_t) * (size_t)a->batch, 256);
+  w.work = off; off = align_up(off + sizeof(WorkEntry) * (size_t)w.max_work, 256);
+  w.work_tmp = off; off = align_up(off + sizeof(WorkEntry) * (size_t)w.max_work, 256);
+  const size_t slots = (size_t)w.max_work;
+  w.part_ml = off; off = align_up(off + sizeof(float2) * slots * a->num_kv_heads * w.rows_cap, 256);
+  w.part_o = off; off = align_up(off + sizeof(float) * slots * a->num_kv_heads * w.rows_cap * a->head_dim, 256);
+  w.total = off;
+  return w;
+}
+
+struct SampleWs {
+  size_t seg_stats, seg_resid, req_norm, total;
+  int32_t nseg;
+};
+
+static spx_status_t check_sample(const spx_sample_args_t *s, bool need_ptrs) {
+  if (!s) return SPX_ERR_INVALID_ARG;
+  if (s->batch < 0 || s->total_q < s->batch || s->vocab <= 0 || s->logits_row_stride < s->vocab) return SPX_ERR_INVALID_ARG;
+  if (s->logits_dtype != SPX_BF16 && s->logits_dtype != SPX_F32) return SPX_ERR_INVALID_ARG;
+  const int vec = s->logits_dtype == SPX_BF16 ? 8 : 4;
+  if (s->logits_row_stride % vec != 0) return SPX_ERR_INVALID_ARG;
+  if ((int64_t)s->total_q - s->batch > (int64_t)s->batch * SPX_MAX_K) return SPX_ERR_INVALID_ARG;
+  if (need_ptrs && s->batch > 0) {
+    const int td = s->total_q - s->batch;
+    if (!s->target_logits || !s->q_indptr || !s->u_sample || !s->accepted_len || !s->out_tokens) return SPX_ERR_INVALID_ARG;
+    if (td > 0 && (!s->draft_logits || !s->draft_token_ids || !s->u_accept)) return SPX_ERR_INVALID_ARG;
+    if (((uintptr_t)s->target_logits | (uintptr_t)s->draft_logits) & 15) return SPX_ERR_INVALID_ARG;
+  }
+  return SPX_OK;
+}
+
+static SampleWs sample_ws_layout(const spx_sample_args_t *s) {
+  SampleWs w{};
+  w.nseg = (s->vocab + kSegElems - 1) / kSegElems;
+  const size_t rows = (size_t)s->total_q + (size_t)(s->total_q - s->batch);
+  size_t off = 0;
+  w.seg_stats = off; off = align_up(off + sizeof(float2) * rows * w.nseg, 256);
+  w.seg_resid = off; off = align_up(off + sizeof(float) * (size_t)s->batch * w.nseg, 256);
+  w.req_norm = off; off = align_up(off + sizeof(float4) * (size_t)s->batch, 256);
+  w.total = off;
+  return w;
+}
+
+// ---------------------------------------------------------------------------------------------
+// launches
+// ---------------------------------------------------------------------------------------------
+static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws, int32_t *dev_status,
+                                     cudaStream_t stream, const DeviceInfo &dev) {
+  if (a->batch == 0) return SPX_OK;
+  const AttnWs w = attn_ws_layout(a);
+  AttnParams p{};
+  p.batch = a->batch; p.total_q = a->total_q;
+  p.max_q_len = a->max_q_len == 0 ? SPX_MAX_K + 1 : a->max_q_len;
+  p.Hq = a->num_q_heads; p.Hkv = a->num_kv_heads; p.G = p.Hq / p.Hkv; p.D = a->head_dim; p.P = a->page_size;
+  p.log2P = 0;
+  while ((1 << p.log2P) < p.P) ++p.log2P;
+  p.num_pages = a->num_pages; p.max_pages_per_req = a->max_pages_per_req;
+  const float scale = a->sm_scale == 0.f ? 1.f / sqrtf((float)a->head_dim) : a->sm_scale;
+  p.scale_log2 = scale * kLog2e;
+  p.q = a->q; p.k_cache = a->k_cache; p.v_cache = a->v_cache;
+  p.stride_page = a->kv_stride_page; p.stride_head = a->kv_stride_head; p.stride_token = a->kv_stride_token;
+  p.block_table = a->block_table; p.seq_lens = a->seq_lens; p.q_indptr = a->q_indptr;
+  p.out = a->out; p.lse = a->lse;
+  p.hdr = reinterpret_cast<PlanHeader *>(ws + w.hdr);
+  p.req_nchunks = reinterpret_cast<int32_t *>(ws + w.nchunks);
+  p.req_part_base = reinterpret_cast<int32_t *>(ws + w.part_base);
+  p.work = reinterpret_cast<WorkEntry *>(ws + w.work);
+  p.work_tmp = reinterpret_cast<WorkEntry *>(ws + w.work_tmp);
+  p.max_work = w.max_work;
+  p.part_ml = reinterpret_cast<float2 *>(ws + w.part_ml);
+  p.part_o = reinterpret_cast<float *>(ws + w.part_o);
+  p.rows_cap = w.rows_cap;
+  p.dev_status = dev_status;
+
+  // the plan never targets more chunks than the workspace was sized for
+  const int sms = dev.num_sms < kPlanSmCount ? dev.num_sms : kPlanSmCount;
+  plan_kernel<<<1, 1024, 0, stream>>>(p, sms * kPlanWaves);
+  ++t_launches;
+
+  const SimtSmem lay(p.rows_cap, p.D);
+  if (lay.total > dev.max_smem_optin) return SPX_ERR_UNSUPPORTED;
+  auto launch_simt = [&](auto kernel) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lay.total);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kSimtThreads, lay.total);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    if (t_ev_start) cudaEventRecord(t_ev_start, stream);
+    kernel<<<dev.num_sms * per_sm, kSimtThreads, lay.total, stream>>>(p);
+    if (t_ev_stop) cudaEventRecord(t_ev_stop, stream);
+    ++t_launches;
+    return cudaGetLastError();
+  };
+  cudaError_t e;
+  if (a->kv_dtype == SPX_F32) {
+    e = p.D == 64 ? launch_simt(attn_simt_kernel<float, 64>) : launch_simt(attn_simt_kernel<float, 128>);
+  } else {
+    e = p.D == 64 ? launch_simt(attn_simt_kernel<__nv_bfloat16, 64>) : launch_simt(attn_simt_kernel<__nv_bfloat16, 128>);
+  }
+  if (e != cudaSuccess) return SPX_ERR_CUDA;
+  if (a->kv_dtype == SPX_F32)
+    combine_kernel<float><<<p.batch * p.Hkv, 256, 0, stream>>>(p);
+  else
+    combine_kernel<__nv_bfloat16><<<p.batch * p.Hkv, 256, 0, stream>>>(p);
+  ++t_launches;
+  return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
+}
+
+template <typename T>
+static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream) {
+  const int rows = p.total_q + p.total_d;
+  row_stats_kernel<T><<<dim3(p.nseg, rows), kSampThreads, 0, stream>>>(p);
+  accept_kernel<T><<<(p.batch + 127) / 128, 128, 0, stream>>>(p);
+  resid_seg_kernel<T><<<dim3(p.nseg, p.batch), kSampThreads, 0, stream>>>(p);
+  select_kernel<T><<<p.batch, kSampThreads, 0, stream>>>(p);
+  t_launches += 4;
+  return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
+}
+
+static spx_status_t launch_sampler(const spx_sample_args_t *s, unsigned char *ws, int32_t *dev_status,
+                                   cudaStream_t stream) {
+  if (s->batch == 0) return SPX_OK;
+  if (s->total_q > 65535 * 2 || s->batch > 65535) return SPX_ERR_UNSUPPORTED;  // grid.y limits
+  const SampleWs w = sample_ws_layout(s);
+  SampleParams p{};
+  p.batch = s->batch; p.total_q = s->total_q; p.total_d = s->total_q - s->batch; p.vocab = s->vocab; p.nseg = w.nseg;
+  if (p.total_q + p.total_d > 65535) return SPX_ERR_UNSUPPORTED;
+  p.row_stride = s->logits_row_stride;
+  p.target = s->target_logits; p.draft = s->draft_logits; p.draft_ids = s->draft_token_ids;
+  p.q_indptr = s->q_indptr; p.u_accept = s->u_accept; p.u_sample = s->u_sample;
+  p.accepted_len = s->accepted_len; p.out_tokens = s->out_tokens; p.diag_ratio = s->diag_ratio;
+  p.seg_stats = reinterpret_cast<float2 *>(ws + w.seg_stats);
+  p.seg_resid = reinterpret_cast<float *>(ws + w.seg_resid);
+  p.req_norm = reinterpret_cast<float4 *>(ws + w.req_norm);
+  p.dev_status = dev_status;
+  return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16>(p, stream) : launch_sampler_t<float>(p, stream);
+}
+
+static spx_status_t check_ws(const void *ws, size_t ws_bytes, size_t need, const int32_t *dev_status) {
+  if (!dev_status) return SPX_ERR_INVALID_ARG;
+  if (need == 0) return SPX_OK;
+  if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need) return SPX_ERR_WORKSPACE;
+  return SPX_OK;
+}
+
+}  // namespace spx
+
+using namespace spx;
+
+extern "C" {
+
+size_t spx_workspace_size(const spx_attn_args_t *attn, const spx_sample_args_t *sample) {
+  size_t total = 0;
+  if (attn) {
+    if (check_attn(attn, false) != SPX_OK) return 0;
+    total += attn_ws_layout(attn).total;
+  }
+  if (sample) {
+    if (check_sample(sample, false) != SPX_OK) return 0;
+    total += sample_ws_layout(sample).total;
+  }
+  return total ? total : 256;
+}
+
+spx_status_t spx_verify_attention(const spx_attn_args_t *args, void *ws, size_t ws_bytes, int32_t *dev_status,
+                                  void *cuda_stream) {
+  t_launches = 0;
+  spx_status_t st = check_attn(args, true);
+  if (st != SPX_OK) return st;
+  st = check_ws(ws, ws_bytes, attn_ws_layout(args).total, dev_status);
+  if (st != SPX_OK) return st;
+  DeviceInfo dev;
+  if (!get_device_info(&dev) || dev.cc_major < 10) return SPX_ERR_CUDA;
+  return launch_attention(args, static_cast<unsigned char *>(ws), dev_status, static_cast<cudaStream_t>(cuda_stream), dev);
+}
+
+spx_status_t spx_rejection_sample(const spx_sample_args_t *args, void *ws, size_t ws_bytes, int32_t *dev_status,
+                                  void *cuda_stream) {
+  t_launches = 0;
+  spx_status_t st = check_sample(args, true);
+  if (st != SPX_OK) return st;
+  st = check_ws(ws, ws_bytes, sample_ws_layout(args).total, dev_status);
+  if (st != SPX_OK) return st;
+  DeviceInfo dev;
+  if (!get_device_info(&dev) || dev.cc_major < 10) return SPX_ERR_CUDA;
+  return launch_sampler(args, static_cast<unsigned char *>(ws), dev_status, static_cast<cudaStream_t>(cuda_stream));
+}
+
+spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_t *sample, void *ws, size_t ws_bytes,
+                             int32_t *dev_status, void *cuda_stream) {
+  t_launches = 0;
+  spx_status_t st = check_attn(attn, true);
+  if (st != SPX_OK) return st;
+  st = check_sample(sample, true);
+  if (st != SPX_OK) return st;
+  if (attn->batch != sample->batch || attn->total_q != sample->total_q) return SPX_ERR_INVALID_ARG;
+  const size_t attn_bytes = attn_ws_layout(attn).total;
+  st = check_ws(ws, ws_bytes, attn_bytes + sample_ws_layout(sample).total, dev_status);
+  if (st != SPX_OK) return st;
+  DeviceInfo dev;
+  if (!get_device_info(&dev) || dev.cc_major < 10) return SPX_ERR_CUDA;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char *base = static_cast<unsigned char *>(ws);
+  // sampler first: its short kernels drain while the attention plan is built
+  st = launch_sampler(sample, base + attn_bytes, dev_status, stream);
+  if (st != SPX_OK) return st;
+  return launch_attention(attn, base, dev_status, stream, dev);
+}
+
+// ---- host-buffer convenience ---------------------------------------------------------------
+namespace {
+struct HostStepLayout {
+  size_t q, k, v, bt, sl, qi, out, lse, tl, dl, ids, ua, us, acc, tok, status, ws, total;
+  size_t q_bytes, kv_bytes, bt_bytes, out_bytes, lse_bytes, tl_bytes, dl_bytes, ws_bytes;
+};
+HostStepLayout host_layout(const spx_attn_args_t *a, const spx_sample_args_t *s, int64_t kv_pool_elems) {
+  HostStepLayout L{};
+  const size_t es = a->kv_dtype == SPX_BF16 ? 2 : 4, ls = s->logits_dtype == SPX_BF16 ? 2 : 4;
+  const size_t B = a->batch, TQ = a->total_q, TD = TQ - B;
+  L.q_bytes = TQ * a->num_q_heads * a->head_dim * es;
+  L.kv_bytes = (size_t)kv_pool_elems * es;
+  L.bt_bytes = B * (size_t)a->max_pages_per_req * 4;
+  L.out_bytes = L.q_bytes;
+  L.lse_bytes = TQ * a->num_q_heads * 4;
+  L.tl_bytes = TQ ? ((TQ - 1) * (size_t)s->logits_row_stride + s->vocab) * ls : 0;
+  L.dl_bytes = TD ? ((TD - 1) * (size_t)s->logits_row_stride + s->vocab) * ls : 0;
+  L.ws_bytes = spx_workspace_size(a, s);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { const size_t o = off; off = align_up(off + bytes, 256); return o; };
+  L.q = take(L.q_bytes); L.k = take(L.kv_bytes); L.v = take(L.kv_bytes); L.bt = take(L.bt_bytes);
+  L.sl = take(B * 4); L.qi = take((B + 1) * 4); L.out = take(L.out_bytes); L.lse = take(L.lse_bytes);
+  L.tl = take(L.tl_bytes); L.dl = take(L.dl_bytes); L.ids = take(TD * 4); L.ua = take(TD * 4); L.us = take(B * 4);
+  L.acc = take(B * 4); L.tok = take(TQ * 4); L.status = take(4); L.ws = take(L.ws_bytes);
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+size_t spx_host_step_arena_size(const spx_attn_args_t *attn, const spx_sample_args_t *sample, int64_t kv_pool_elems) {
+  if (check_attn(attn, false) != SPX_OK || check_sample(sample, false) != SPX_OK || kv_pool_elems < 0) return 0;
+  if (attn->batch != sample->batch || attn->total_q != sample->total_q) return 0;
+  return host_layout(attn, sample, kv_pool_elems).total;
+}
+
+spx_status_t spx_verify_step_host(const spx_attn_args_t *attn, const spx_sample_args_t *sample, int64_t kv_pool_elems,
+                                  void *dev_arena, size_t arena_bytes, int32_t *dev_status_host, void *cuda_stream) {
+  t_launches = 0;
+  if (check_attn(attn, false) != SPX_OK || check_sample(sample, false) != SPX_OK || kv_pool_elems < 0 || !dev_status_host)
+    return SPX_ERR_INVALID_ARG;
+  if (attn->batch != sample->batch || attn->total_q != sample->total_q) return SPX_ERR_INVALID_ARG;
+  const HostStepLayout L = host_layout(attn, sample, kv_pool_elems);
+  if (!dev_arena || ((uintptr_t)dev_arena & 255) || arena_bytes < L.total) return SPX_ERR_WORKSPACE;
+  unsigned char *d = static_cast<unsigned char *>(dev_arena);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const size_t B = attn->batch, TQ = attn->total_q, TD = TQ - B;
+  bool ok = true;
+  auto h2d = [&](size_t off, const void *src, size_t bytes) {
+    if (bytes && src) ok = ok && cudaMemcpyAsync(d + off, src, bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  };
+  auto d2h = [&](void *dst, size_t off, size_t bytes) {
+    if (bytes && dst) ok = ok && cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  };
+  h2d(L.q, attn->q, L.q_bytes); h2d(L.k, attn->k_cache, L.kv_bytes); h2d(L.v, attn->v_cache, L.kv_bytes);
+  h2d(L.bt, attn->block_table, L.bt_bytes); h2d(L.sl, attn->seq_lens, B * 4); h2d(L.qi, attn->q_indptr, (B + 1) * 4);
+  h2d(L.tl, sample->target_logits, L.tl_bytes); h2d(L.dl, sample->draft_logits, L.dl_bytes);
+  h2d(L.ids, sample->draft_token_ids, TD * 4); h2d(L.ua, sample->u_accept, TD * 4); h2d(L.us, sample->u_sample, B * 4);
+  ok = ok && cudaMemsetAsync(d + L.status, 0, 4, stream) == cudaSuccess;
+  if (!ok) return SPX_ERR_CUDA;
+  spx_attn_args_t a = *attn;
+  spx_sample_args_t s = *sample;
+  a.q = d + L.q; a.k_cache = d + L.k; a.v_cache = d + L.v;
+  a.block_table = reinterpret_cast<int32_t *>(d + L.bt); a.seq_lens = reinterpret_cast<int32_t *>(d + L.sl);
+  a.q_indptr = reinterpret_cast<int32_t *>(d + L.qi); a.out = d + L.out;
+  a.lse = attn->lse ? reinterpret_cast<float *>(d + L.lse) : nullptr;
+  s.target_logits = d + L.tl; s.draft_logits = d + L.dl; s.draft_token_ids = reinterpret_cast<int32_t *>(d + L.ids);
+  s.q_indptr = a.q_indptr; s.u_accept = reinterpret_cast<float *>(d + L.ua); s.u_sample = reinterpret_cast<float *>(d + L.us);
+  s.accepted_len = reinterpret_cast<int32_t *>(d + L.acc); s.out_tokens = reinterpret_cast<int32_t *>(d + L.tok);
+  s.diag_ratio = nullptr;
+  const spx_status_t st = spx_verify_step(&a, &s, d + L.ws, L.ws_bytes, reinterpret_cast<int32_t *>(d + L.status), cuda_stream);
+  if (st != SPX_OK) return st;
+  d2h(attn->out, L.out, L.out_bytes); d2h(attn->lse, L.lse, L.lse_bytes);
+  d2h(sample->accepted_len, L.acc, B * 4); d2h(sample->out_tokens, L.tok, TQ * 4); d2h(dev_status_host, L.status, 4);
+  return ok ? SPX_OK : SPX_ERR_CUDA;
+}
+
+const char *spx_status_string(spx_status_t status) {
+  switch (status) {
+    case SPX_OK: return "ok";
+    case SPX_ERR_INVALID_ARG: return "invalid argument";
+    case SPX_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case SPX_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case SPX_ERR_CUDA: return "CUDA error (or no sm_100 device)";
+  }
+  return "unknown status";
+}
+
+void spx_set_timing_events(void *start_event, void *stop_event) {
+  t_ev_start = static_cast<cudaEvent_t>(start_event);
+  t_ev_stop = static_cast<cudaEvent_t>(stop_event);
+}
+
+int32_t spx_last_launch_count(void) { return t_launches; }
+
+}  // extern "C"
