@@ -120,7 +120,7 @@ def sub_batch(b_cpu: W.VerifyBatch, n_req: int) -> W.VerifyBatch:
 
 def oracle_sample_size(spec: W.WorkloadSpec) -> int:
     """Requests in the CPU-baseline sample: about 10-30 s of float64 work on ~8-32 cores."""
-    return {0: 4, 1: 16, 2: 16, 3: 1, 4: 16}.get(spec.index, min(spec.batch, 8))
+    return {0: 4, 1: 64, 2: 128, 3: 4, 4: 64}.get(spec.index, min(spec.batch, 8))
 
 
 def time_oracle(b_cpu: W.VerifyBatch, n_req: int):

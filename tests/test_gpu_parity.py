@@ -103,7 +103,16 @@ def test_edge_cases_k0_minimal_context_and_page_boundaries():
     for L, k in cases:
         spec = dataclasses.replace(base, ctx=("const", L), k=("const", k))
         b_cpu = W.generate(spec, seed=1000 + L * 16 + k)
+        # vocab 777 is not a multiple of the 16-byte vector: rows are padded to a stride of 784
+        padded = {}
+        for name in ("target_logits", "draft_logits"):
+            t = getattr(b_cpu, name)
+            padded[name] = torch.full((t.shape[0], 784), 30.0, dtype=t.dtype)      # poison in the padding
+            padded[name][:, :777] = t
+            setattr(b_cpu, name, padded[name][:, :777])
         b = b_cpu.to(DEV)
+        b.target_logits = padded["target_logits"].to(DEV)[:, :777]
+        b.draft_logits = padded["draft_logits"].to(DEV)[:, :777]
         out, lse, ws = gpu_attention(b)
         assert int(ws.status.item()) == 0
         ref_o, ref_l = oracle_attention(b_cpu)
@@ -120,10 +129,10 @@ def test_empty_batch_is_a_no_op():
     a.batch, a.total_q, a.num_q_heads, a.num_kv_heads, a.head_dim, a.page_size = 0, 0, 8, 2, 64, 16
     a.kv_stride_page, a.kv_stride_head, a.kv_stride_token = 2048, 1024, 64
     st = torch.zeros(1, dtype=torch.int32, device=DEV)
-    ws = torch.empty(1 << 20, dtype=torch.uint8, device=DEV)
-    assert lib.spx_verify_attention(C.byref(a), ws.data_ptr(), ws.numel(), st.data_ptr(), None) == 0
     s = binding.SampleArgs()
     s.batch, s.total_q, s.vocab, s.logits_row_stride, s.logits_dtype = 0, 0, 64, 64, 1
+    ws = torch.empty(spx.workspace_size(a, s), dtype=torch.uint8, device=DEV)
+    assert lib.spx_verify_attention(C.byref(a), ws.data_ptr(), ws.numel(), st.data_ptr(), None) == 0
     assert lib.spx_rejection_sample(C.byref(s), ws.data_ptr(), ws.numel(), st.data_ptr(), None) == 0
     torch.cuda.synchronize()
     assert int(st.item()) == 0
