@@ -78,6 +78,8 @@ struct AttnParams {
   PlanHeader *hdr;
   int32_t *req_nchunks;    // [B]  0 = invalid request
   int32_t *req_part_base;  // [B]
+  int32_t *req_bad;        // [B]  set when a needed page id was out of range
+  int32_t head_inner;      // tensor-map dimension order: 1 = (d, head, token, page), 0 = (d, token, head, page)
   WorkEntry *work;         // [max_work]
   WorkEntry *work_tmp;     // [max_work]
   int32_t max_work;

@@ -56,6 +56,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int target_chu
     const int tiles = ok ? (L + kTileTokens - 1) / kTileTokens : 0;
     if (!ok) s_bad = 1;
     p.req_nchunks[r] = tiles;  // tiles for now, chunk count after pass 2
+    p.req_bad[r] = 0;
     local_tiles += tiles;
   }
   __syncthreads();
@@ -137,7 +138,7 @@ __global__ void __launch_bounds__(256) combine_kernel(AttnParams p) {
   int m = p.q_indptr[r + 1] - q0;
   T *out = reinterpret_cast<T *>(p.out);
   const int D = p.D, G = p.G;
-  if (nch == 0 || p.hdr->overflow) {
+  if (nch == 0 || p.hdr->overflow || p.req_bad[r]) {
     // invalid request (or unusable plan): zero rows, NaN lse; clamp the row range to the tensor
     if (m < 0) m = 0;
     if (m > p.max_q_len) m = p.max_q_len;

@@ -6,6 +6,7 @@
 #include <cstring>
 
 #include "attn_simt.cuh"
+#include "attn_tc.cuh"
 #include "common.cuh"
 #include "plan.cuh"
 #include "sampler.cuh"
@@ -40,7 +41,7 @@ constexpr int kPlanSmCount = 148;  // workspace sizing must not depend on a devi
 // workspace layout
 // ---------------------------------------------------------------------------------------------
 struct AttnWs {
-  size_t hdr, nchunks, part_base, work, work_tmp, part_ml, part_o, total;
+  size_t hdr, nchunks, part_base, req_bad, work, work_tmp, part_ml, part_o, total;
   int32_t max_work, rows_cap;
 };
 
@@ -79,6 +80,7 @@ static AttnWs attn_ws_layout(const spx_attn_args_t *a) {
   w.hdr = off; off = align_up(off + sizeof(PlanHeader), 256);
   w.nchunks = off; off = align_up(off + sizeof(int32_t) * (size_t)a->batch, 256);
   w.part_base = off; off = align_up(off + sizeof(int32_t) * (size_t)a->batch, 256);
+  w.req_bad = off; off = align_up(off + sizeof(int32_t) * (size_t)a->batch, 256);
   w.work = off; off = align_up(off + sizeof(WorkEntry) * (size_t)w.max_work, 256);
   w.work_tmp = off; off = align_up(off + sizeof(WorkEntry) * (size_t)w.max_work, 256);
   const size_t slots = (size_t)w.max_work;
@@ -121,6 +123,69 @@ static SampleWs sample_ws_layout(const spx_sample_args_t *s) {
   return w;
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// TMA tensor maps over the KV pools
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void *ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess) ptr = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(ptr);
+  }();
+  return fn;
+}
+
+// 4-D bf16 view of a pool: dims ordered by increasing stride, (d, head, token, page) when heads are
+// the inner dimension and (d, token, head, page) otherwise; one box = one page x one kv-head x 64
+// columns, 128-byte swizzle.
+static bool make_pool_map(CUtensorMap *map, const void *pool, const spx_attn_args_t *a, bool head_inner) {
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) return false;
+  const cuuint64_t D = a->head_dim, P = a->page_size, H = a->num_kv_heads, N = a->num_pages > 0 ? a->num_pages : 1;
+  const cuuint64_t st = (cuuint64_t)a->kv_stride_token * 2, sh = (cuuint64_t)a->kv_stride_head * 2,
+                   sp = (cuuint64_t)a->kv_stride_page * 2;
+  cuuint64_t dims[4], strides[3];
+  cuuint32_t box[4], estr[4] = {1, 1, 1, 1};
+  if (head_inner) {
+    dims[0] = D; dims[1] = H; dims[2] = P; dims[3] = N;
+    strides[0] = sh; strides[1] = st; strides[2] = sp;
+    box[0] = 64; box[1] = 1; box[2] = (cuuint32_t)P; box[3] = 1;
+  } else {
+    dims[0] = D; dims[1] = P; dims[2] = H; dims[3] = N;
+    strides[0] = st; strides[1] = sh; strides[2] = sp;
+    box[0] = 64; box[1] = (cuuint32_t)P; box[2] = 1; box[3] = 1;
+  }
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The tensor-core kernel handles bf16 pools whose pages hold at least one 8-row swizzle atom.
+static bool use_tensor_core_path(const spx_attn_args_t *a) {
+  return a->kv_dtype == SPX_BF16 && a->page_size >= 8 && a->num_pages > 0 && a->kv_stride_page > 0 &&
+         a->kv_stride_head > 0;
+}
+
+template <int D, int QROWS>
+static cudaError_t launch_tc(const CUtensorMap &kmap, const CUtensorMap &vmap, const AttnParams &p, int num_sms,
+                             cudaStream_t stream) {
+  using Cfg = TcCfg<D, QROWS>;
+  auto kernel = attn_tc_kernel<D, QROWS>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  if (t_ev_start) cudaEventRecord(t_ev_start, stream);
+  kernel<<<num_sms, kTcThreads, Cfg::kSmemBytes, stream>>>(kmap, vmap, p);
+  if (t_ev_stop) cudaEventRecord(t_ev_stop, stream);
+  ++t_launches;
+  return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------------------------------------
 // launches
 // ---------------------------------------------------------------------------------------------
@@ -144,6 +209,7 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
   p.hdr = reinterpret_cast<PlanHeader *>(ws + w.hdr);
   p.req_nchunks = reinterpret_cast<int32_t *>(ws + w.nchunks);
   p.req_part_base = reinterpret_cast<int32_t *>(ws + w.part_base);
+  p.req_bad = reinterpret_cast<int32_t *>(ws + w.req_bad);
   p.work = reinterpret_cast<WorkEntry *>(ws + w.work);
   p.work_tmp = reinterpret_cast<WorkEntry *>(ws + w.work_tmp);
   p.max_work = w.max_work;
@@ -157,26 +223,38 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
   plan_kernel<<<1, 1024, 0, stream>>>(p, sms * kPlanWaves);
   ++t_launches;
 
-  const SimtSmem lay(p.rows_cap, p.D);
-  if (lay.total > dev.max_smem_optin) return SPX_ERR_UNSUPPORTED;
-  auto launch_simt = [&](auto kernel) -> cudaError_t {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lay.total);
-    if (e != cudaSuccess) return e;
-    int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kSimtThreads, lay.total);
-    if (e != cudaSuccess) return e;
-    if (per_sm < 1) per_sm = 1;
-    if (t_ev_start) cudaEventRecord(t_ev_start, stream);
-    kernel<<<dev.num_sms * per_sm, kSimtThreads, lay.total, stream>>>(p);
-    if (t_ev_stop) cudaEventRecord(t_ev_stop, stream);
-    ++t_launches;
-    return cudaGetLastError();
-  };
   cudaError_t e;
-  if (a->kv_dtype == SPX_F32) {
-    e = p.D == 64 ? launch_simt(attn_simt_kernel<float, 64>) : launch_simt(attn_simt_kernel<float, 128>);
+  if (use_tensor_core_path(a)) {
+    p.head_inner = a->kv_stride_head < a->kv_stride_token ? 1 : 0;
+    CUtensorMap kmap, vmap;
+    if (!make_pool_map(&kmap, a->k_cache, a, p.head_inner) || !make_pool_map(&vmap, a->v_cache, a, p.head_inner))
+      return SPX_ERR_CUDA;
+    if (p.D == 128)
+      e = p.rows_cap <= 64 ? launch_tc<128, 64>(kmap, vmap, p, dev.num_sms, stream)
+                           : launch_tc<128, 128>(kmap, vmap, p, dev.num_sms, stream);
+    else
+      e = p.rows_cap <= 64 ? launch_tc<64, 64>(kmap, vmap, p, dev.num_sms, stream)
+                           : launch_tc<64, 128>(kmap, vmap, p, dev.num_sms, stream);
   } else {
-    e = p.D == 64 ? launch_simt(attn_simt_kernel<__nv_bfloat16, 64>) : launch_simt(attn_simt_kernel<__nv_bfloat16, 128>);
+    const SimtSmem lay(p.rows_cap, p.D);
+    if (lay.total > dev.max_smem_optin) return SPX_ERR_UNSUPPORTED;
+    auto launch_simt = [&](auto kernel) -> cudaError_t {
+      cudaError_t er = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lay.total);
+      if (er != cudaSuccess) return er;
+      int per_sm = 0;
+      er = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kSimtThreads, lay.total);
+      if (er != cudaSuccess) return er;
+      if (per_sm < 1) per_sm = 1;
+      if (t_ev_start) cudaEventRecord(t_ev_start, stream);
+      kernel<<<dev.num_sms * per_sm, kSimtThreads, lay.total, stream>>>(p);
+      if (t_ev_stop) cudaEventRecord(t_ev_stop, stream);
+      ++t_launches;
+      return cudaGetLastError();
+    };
+    if (a->kv_dtype == SPX_F32)
+      e = p.D == 64 ? launch_simt(attn_simt_kernel<float, 64>) : launch_simt(attn_simt_kernel<float, 128>);
+    else
+      e = p.D == 64 ? launch_simt(attn_simt_kernel<__nv_bfloat16, 64>) : launch_simt(attn_simt_kernel<__nv_bfloat16, 128>);
   }
   if (e != cudaSuccess) return SPX_ERR_CUDA;
   if (a->kv_dtype == SPX_F32)
