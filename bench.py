@@ -173,6 +173,7 @@ def main():
     ap.add_argument("--impl", default="spx", choices=["spx", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 2000:
@@ -254,6 +255,8 @@ def main():
     b_host = None
     e2e = None
     try:
+        if args.no_e2e:
+            raise RuntimeError("skipped (--no-e2e)")
         b_host = b.to("cpu")
         pin = {n: getattr(b_host, n).pin_memory() for n in W.VerifyBatch._TENSORS}
         out_h = torch.empty(out.shape, dtype=out.dtype).pin_memory()

@@ -22,7 +22,10 @@
 namespace spx {
 
 constexpr int kTcThreads = 192;
-constexpr float kRescaleThreshold = 8.f;  // log2 units
+#ifndef SPX_RESCALE_THRESHOLD
+#define SPX_RESCALE_THRESHOLD 8.f
+#endif
+constexpr float kRescaleThreshold = SPX_RESCALE_THRESHOLD;  // log2 units
 
 template <int D, int QROWS>
 struct TcCfg {
@@ -44,7 +47,7 @@ struct TcCfg {
 struct TcBarriers {
   uint64_t k_full[4], v_full[4], k_empty[4], v_empty[4];
   uint64_t s_full[2], p_full[2], q_full[2], q_empty[2];
-  uint64_t pv_done, o_free;
+  uint64_t pv_done[2], o_free, e_bar;  // pv_done alternates per tile: a waiter may lag the MMA by two tiles
   uint32_t tmem_base;
   volatile int32_t abort;
 };
@@ -166,7 +169,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
   if (tid == 0) {
     for (int s = 0; s < 4; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->v_full[s], 1); mbar_init(&bars->k_empty[s], 1); mbar_init(&bars->v_empty[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&bars->s_full[b], 1); mbar_init(&bars->p_full[b], 4); mbar_init(&bars->q_full[b], 4); mbar_init(&bars->q_empty[b], 1); }
-    mbar_init(&bars->pv_done, 1);
+    mbar_init(&bars->pv_done[0], 1);
+    mbar_init(&bars->pv_done[1], 1);
     mbar_init(&bars->o_free, 4);
     bars->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -299,7 +303,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
           for (int k = 0; k < kTileTokens / 16; ++k)
             mma_ts(tmem + Cfg::kColO, tp + k * 8, smem_desc(va + k * 2048, Cfg::kHalfBytes, 1024), kIdescPV, (i > 0) || (k > 0));
           mma_commit(&bars->v_empty[slot]);
-          mma_commit(&bars->pv_done);
+          mma_commit(&bars->pv_done[tc_ & 1]);
         }
       }
     }
@@ -389,7 +393,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
           }
           if (__any_sync(0xffffffffu, need_scale)) {
             // O holds contributions of earlier tiles: wait for the last PV, then scale the rows
-            ok = warp_wait(&bars->pv_done, (tc_ - 1) & 1);
+            ok = warp_wait(&bars->pv_done[(tc_ - 1) & 1], ((tc_ - 1) >> 1) & 1);
             if (!ok) break;
             fence_after();
 #pragma unroll 1
@@ -450,7 +454,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
       }
       if (!ok) break;
       // epilogue: wait for the last PV of the item, normalise and store
-      ok = warp_wait(&bars->pv_done, (tc_ - 1) & 1);
+      ok = warp_wait(&bars->pv_done[(tc_ - 1) & 1], ((tc_ - 1) >> 1) & 1);
       if (!ok) break;
       fence_after();
       if (active) {

@@ -11,7 +11,10 @@ namespace spx {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTileTokens = 128;   // KV tokens per attention tile (both attention kernels plan in this unit)
-constexpr int kPlanWaves = 8;      // target number of work chunks per SM
+#ifndef SPX_PLAN_WAVES
+#define SPX_PLAN_WAVES 8
+#endif
+constexpr int kPlanWaves = SPX_PLAN_WAVES;  // target number of work chunks per SM
 
 __device__ __forceinline__ float ld_as_float(const float *p, int64_t i) { return p[i]; }
 __device__ __forceinline__ float ld_as_float(const __nv_bfloat16 *p, int64_t i) { return __bfloat162float(p[i]); }
@@ -55,11 +58,15 @@ struct PlanHeader {
   int32_t pad[2];
 };
 
-struct WorkEntry {
+struct __align__(16) WorkEntry {
   int32_t req;         // request index
   int32_t tile_begin;  // first tile of the chunk
   int32_t tile_end;    // one past the last tile
   int32_t part_slot;   // partial slot, or -1 when the request is not split (direct output)
+  int32_t q0;          // q_indptr[req]: first query row of the request
+  int32_t m;           // k+1 query positions
+  int32_t L;           // seq_lens[req]
+  int32_t pad;
 };
 
 struct AttnParams {
@@ -87,6 +94,13 @@ struct AttnParams {
   float2 *part_ml;         // [slot][Hkv][rows_cap]  (m in log2 domain, l)
   int32_t rows_cap;        // G * max_q_len
   int32_t *dev_status;
+  long long *prof;         // optional per-CTA cycle counters (profiling builds only), else NULL
 };
+
+#ifndef SPX_PROFILE
+#define SPX_PROFILE 0
+#endif
+constexpr bool kProfile = SPX_PROFILE != 0;
+constexpr int kProfSlots = 16;
 
 }  // namespace spx

@@ -92,6 +92,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int target_chu
           const int sz = q + (i < rem ? 1 : 0);
           WorkEntry e;
           e.req = r; e.tile_begin = tb; e.tile_end = tb + sz; e.part_slot = npart ? off_p + i : -1;
+          e.q0 = p.q_indptr[r]; e.m = p.q_indptr[r + 1] - e.q0; e.L = p.seq_lens[r]; e.pad = 0;
           p.work_tmp[off_w + i] = e;
           atomicAdd(&s_hist[1023 - min(sz, 1023)], 1);
           tb += sz;

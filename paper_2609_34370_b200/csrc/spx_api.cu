@@ -7,6 +7,7 @@
 
 #include "attn_simt.cuh"
 #include "attn_tc.cuh"
+#include "attn_tc4.cuh"
 #include "common.cuh"
 #include "plan.cuh"
 #include "sampler.cuh"
@@ -16,6 +17,7 @@ namespace spx {
 
 static thread_local int32_t t_launches = 0;
 static thread_local cudaEvent_t t_ev_start = nullptr, t_ev_stop = nullptr;
+static thread_local long long *t_prof = nullptr;  // profiling builds only
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -172,6 +174,20 @@ static bool use_tensor_core_path(const spx_attn_args_t *a) {
          a->kv_stride_head > 0;
 }
 
+template <int D>
+static cudaError_t launch_tc4(const CUtensorMap &kmap, const CUtensorMap &vmap, const AttnParams &p, int num_sms,
+                              cudaStream_t stream) {
+  using Cfg = Tc4Cfg<D>;
+  auto kernel = attn_tc4_kernel<D>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  if (t_ev_start) cudaEventRecord(t_ev_start, stream);
+  kernel<<<num_sms, kTcThreads, Cfg::kSmemBytes, stream>>>(kmap, vmap, p);
+  if (t_ev_stop) cudaEventRecord(t_ev_stop, stream);
+  ++t_launches;
+  return cudaGetLastError();
+}
+
 template <int D, int QROWS>
 static cudaError_t launch_tc(const CUtensorMap &kmap, const CUtensorMap &vmap, const AttnParams &p, int num_sms,
                              cudaStream_t stream) {
@@ -217,6 +233,7 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
   p.part_o = reinterpret_cast<float *>(ws + w.part_o);
   p.rows_cap = w.rows_cap;
   p.dev_status = dev_status;
+  p.prof = t_prof;
 
   // the plan never targets more chunks than the workspace was sized for
   const int sms = dev.num_sms < kPlanSmCount ? dev.num_sms : kPlanSmCount;
@@ -229,7 +246,9 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
     CUtensorMap kmap, vmap;
     if (!make_pool_map(&kmap, a->k_cache, a, p.head_inner) || !make_pool_map(&vmap, a->v_cache, a, p.head_inner))
       return SPX_ERR_CUDA;
-    if (p.D == 128)
+    if (p.rows_cap <= 32)
+      e = p.D == 128 ? launch_tc4<128>(kmap, vmap, p, dev.num_sms, stream) : launch_tc4<64>(kmap, vmap, p, dev.num_sms, stream);
+    else if (p.D == 128)
       e = p.rows_cap <= 64 ? launch_tc<128, 64>(kmap, vmap, p, dev.num_sms, stream)
                            : launch_tc<128, 128>(kmap, vmap, p, dev.num_sms, stream);
     else
@@ -459,5 +478,10 @@ void spx_set_timing_events(void *start_event, void *stop_event) {
 }
 
 int32_t spx_last_launch_count(void) { return t_launches; }
+
+#if SPX_PROFILE
+// Profiling builds only (not declared in spx.h): per-CTA cycle counters of the attention kernel.
+void spx_debug_set_profile_buffer(long long *device_buffer) { t_prof = device_buffer; }
+#endif
 
 }  // extern "C"
