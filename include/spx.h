@@ -14,7 +14,8 @@
  *   - Pointers inside the argument structs are DEVICE pointers unless the field name ends in
  *     _host.  The structs themselves, `ws_bytes` and all scalars live on the host.
  *   - The caller owns every buffer and the CUDA stream (`cuda_stream` is a cudaStream_t passed
- *     as void*; NULL = the legacy default stream).  The library allocates no device memory.
+ *     as void*; NULL = the legacy default stream).  The library allocates no device memory
+ *     (spx_verify_step keeps one internal stream and two events per host thread and device).
  *   - Calls only enqueue work on the stream and return; nothing synchronises the device.
  *   - Host-visible argument errors return a non-zero spx_status_t and launch nothing.
  *   - Errors in device-resident data (a page id out of range, a draft token id >= vocab, a
@@ -146,8 +147,11 @@ spx_status_t spx_rejection_sample(const spx_sample_args_t *args, void *ws, size_
                                   int32_t *dev_status, void *cuda_stream);
 
 /*
- * The whole verify step: both halves on the caller's stream.  The halves are independent given
- * their inputs (logits are inputs here), so the library may interleave them.  `ws` must hold
+ * The whole verify step.  The halves are independent given their inputs (logits are inputs
+ * here), so the sampling half is forked onto a library-internal stream and joined back into
+ * `cuda_stream` before the call returns: work enqueued on `cuda_stream` afterwards sees both
+ * halves' outputs.  The internal stream and its two events are created on the first call of a
+ * host thread on a device and live until the thread exits.  `ws` must hold
  * spx_workspace_size(attn, sample) bytes.
  */
 spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_t *sample, void *ws,

@@ -47,7 +47,7 @@ struct TcCfg {
 struct TcBarriers {
   uint64_t k_full[4], v_full[4], k_empty[4], v_empty[4];
   uint64_t s_full[2], p_full[2], q_full[2], q_empty[2];
-  uint64_t pv_done[2], o_free, e_bar;  // pv_done alternates per tile: a waiter may lag the MMA by two tiles
+  uint64_t pv_done[2], o_free, o_free2[2], e_bar;  // pv_done alternates per tile: a waiter may lag the MMA by two tiles
   uint32_t tmem_base;
   volatile int32_t abort;
 };
@@ -301,7 +301,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
           const uint32_t tp = tmem + ((tc_ & 1) ? Cfg::kColS1 : Cfg::kColS0);
 #pragma unroll
           for (int k = 0; k < kTileTokens / 16; ++k)
-            mma_ts(tmem + Cfg::kColO, tp + k * 8, smem_desc(va + k * 2048, Cfg::kHalfBytes, 1024), kIdescPV, (i > 0) || (k > 0));
+            mma_ts(tmem + Cfg::kColO, tp + k * 8, smem_desc(va + k * 2 * 1024, Cfg::kHalfBytes, 1024), kIdescPV, (i > 0) || (k > 0));
           mma_commit(&bars->v_empty[slot]);
           mma_commit(&bars->pv_done[tc_ & 1]);
         }
@@ -444,7 +444,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
           for (int i = sm_tid; i < n_chunks; i += 128) {
             const int h = i / ((kTileTokens - ntok) * 8), rem = i % ((kTileTokens - ntok) * 8);
             const int tok = ntok + rem / 8, c = rem % 8;
-            *reinterpret_cast<uint4 *>(vt + h * Cfg::kHalfBytes + tok * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4 *>(vt + (tok >> 3) * 1024 + h * Cfg::kHalfBytes + (tok & 7) * 128 + c * 16) = make_uint4(0, 0, 0, 0);
           }
           fence_async_smem();
         }

@@ -26,12 +26,13 @@ struct Tc4Cfg {
   static constexpr int kQHalfBytes = 32 * 128;
   static constexpr int kQBytes = kHalves * kQHalfBytes;
   static constexpr int kPBytes = 2 * 32 * 128;   // one P tile: 32 rows x 128 tokens bf16, two 64-token halves
-  static constexpr int kBarBytes = 2048;         // barriers, per-quadrant row maxima and row sums
-  static constexpr int kBudget = 232448 - 1024 - kBarBytes - 2 * kQBytes - 2 * kPBytes;
+  static constexpr int kBarBytes = 2304;         // barriers (256) + row maxima (1024) + row sums (1024)
+  static constexpr int kSlack = 512;             // room to round the dynamic shared base up to 1024 bytes
+  static constexpr int kBudget = 232448 - kSlack - kBarBytes - 2 * kQBytes - 2 * kPBytes;
   static constexpr int kStagesRaw = kBudget / (2 * kTileBytes);
   static constexpr int kStages = kStagesRaw > 4 ? 4 : kStagesRaw;
-  static constexpr int kSmemBytes = 1024 + 2 * kQBytes + kStages * 2 * kTileBytes + 2 * kPBytes + kBarBytes;
-  static constexpr int kTmemCols = 128;
+  static constexpr int kSmemBytes = kSlack + 2 * kQBytes + kStages * 2 * kTileBytes + 2 * kPBytes + kBarBytes;
+  static constexpr int kTmemCols = 128;          // two score buffers (64) + two O buffers (2 * D/4)
   static constexpr int kColS0 = 0, kColS1 = 32, kColO = 64;
   static constexpr int kColBlock = D / 4;        // output columns held by one quadrant
   static_assert(kStages >= 2, "need at least two stages");
@@ -68,15 +69,19 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, AttnParams p) {
   using Cfg = Tc4Cfg<D>;
   using namespace tc;
-  extern __shared__ unsigned char smem_dyn[];
+  extern __shared__ __align__(1024) unsigned char smem_dyn[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  if (smem - smem_dyn > Cfg::kSlack) {  // cannot happen with the declared alignment; never run past the allocation
+    if (threadIdx.x == 0) atomicOr(p.dev_status, SPX_DEV_TIMEOUT);
+    return;
+  }
   unsigned char *sQ = smem;
   unsigned char *sK = smem + 2 * Cfg::kQBytes;
   unsigned char *sV = sK + Cfg::kStages * Cfg::kTileBytes;
   unsigned char *sP = sV + Cfg::kStages * Cfg::kTileBytes;  // two P tiles
   TcBarriers *bars = reinterpret_cast<TcBarriers *>(sP + 2 * Cfg::kPBytes);
   float *sMx = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(bars) + 256);  // [2 tiles][4 quadrants][32 rows]
-  float *sL = sMx + 2 * 4 * 32;                                                          // [4 quadrants][32 rows]
+  float *sL = sMx + 2 * 4 * 32;                                                          // [2 items][4 quadrants][32 rows]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   long long prof_g0 = 0;
@@ -86,7 +91,8 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
     for (int b = 0; b < 2; ++b) { mbar_init(&bars->s_full[b], 1); mbar_init(&bars->p_full[b], 4); mbar_init(&bars->q_full[b], 4); mbar_init(&bars->q_empty[b], 1); }
     mbar_init(&bars->pv_done[0], 1);
     mbar_init(&bars->pv_done[1], 1);
-    mbar_init(&bars->o_free, 4);
+    mbar_init(&bars->o_free2[0], 4);
+    mbar_init(&bars->o_free2[1], 4);
     mbar_init(&bars->e_bar, 4);
     bars->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -269,7 +275,8 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
         if (!ok) break;
         const uint32_t t = pv.t;
         ok = lane_wait(&bars->p_full[t & 1], (t >> 1) & 1, 1);
-        if (ok && pv.i == 0 && pv.qc > 0) ok = lane_wait(&bars->o_free, (pv.qc - 1) & 1, 3);
+        // the O buffer of this item's parity was last used two items ago
+        if (ok && pv.i == 0 && pv.qc >= 2) ok = lane_wait(&bars->o_free2[pv.qc & 1], ((pv.qc >> 1) - 1) & 1, 3);
         const int slot = t % Cfg::kStages;
         if (ok) ok = lane_wait(&bars->v_full[slot], (t / Cfg::kStages) & 1, 2);
         if (!ok) break;
@@ -278,8 +285,8 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
         const uint32_t pa = smem_u32(sP + (t & 1) * Cfg::kPBytes);
 #pragma unroll
         for (int k = 0; k < kTileTokens / 16; ++k)
-          mma_ws_ss(tmem + Cfg::kColO, smem_desc(pa + (k / 4) * 4096 + (k % 4) * 32, 16, 1024),
-                    smem_desc(va + k * 2048, Cfg::kHalfBytes, 1024), kIdescPV, (pv.i > 0) || (k > 0));
+          mma_ws_ss(tmem + Cfg::kColO + (pv.qc & 1) * Cfg::kColBlock, smem_desc(pa + (k / 4) * 4096 + (k % 4) * 32, 16, 1024),
+                    smem_desc(va + k * 2 * 1024, Cfg::kHalfBytes, 1024), kIdescPV, (pv.i > 0) || (k > 0));
         mma_commit(&bars->v_empty[slot]);
         mma_commit(&bars->pv_done[t & 1]);
         advance(pv);
@@ -336,6 +343,52 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
       const bool r = warp_wait(&bars->e_bar, ec & 1, 2);
       ++ec;
       return r;
+    };
+    // Row sums of the four quadrants are merged through sL (written at the end of the item's last
+    // tile, visible after the next bounded barrier); each thread then finishes its D/4 columns.
+    struct Pending { bool valid; ItemInfo I; float m_ref; uint32_t last_tc, qc; } pend;
+    pend.valid = false;
+    auto run_epilogue = [&]() -> bool {
+      const long long pe0 = kProfile ? clock64() : 0;
+      const ItemInfo &J = pend.I;
+      const float *sl = sL + (pend.qc & 1) * 128;
+      const float l_row = sl[row] + sl[32 + row] + sl[64 + row] + sl[96 + row];
+      if (!warp_wait(&bars->pv_done[pend.last_tc & 1], (pend.last_tc >> 1) & 1, 1)) return false;
+      fence_after();
+      uint32_t o[CB];
+      tmem_ld<CB>(tmem + Cfg::kColO + (pend.qc & 1) * CB + lane_addr, o);
+      wait_ld();
+      // O has been read: the item after next may overwrite this buffer
+      fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->o_free2[pend.qc & 1]);
+      const int j = row / p.G, hg = row % p.G;
+      if (row < J.R) {
+        if (J.part_slot < 0) {
+          const float inv = 1.f / l_row;
+          __nv_bfloat16 *dst = out + ((int64_t)(J.q0 + j) * p.Hq + J.g * p.G + hg) * D + quad * CB;
+#pragma unroll
+          for (int v = 0; v < CB / 8; ++v) {
+            uint4 u;
+            u.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+            u.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+            u.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+            u.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+            *reinterpret_cast<uint4 *>(dst + v * 8) = u;
+          }
+          if (quad == 0 && p.lse) p.lse[(int64_t)(J.q0 + j) * p.Hq + J.g * p.G + hg] = (pend.m_ref + log2f(l_row)) * kLn2;
+        } else {
+          const int64_t slot = ((int64_t)J.part_slot * p.Hkv + J.g) * p.rows_cap + row;
+          float *dst = p.part_o + slot * D + quad * CB;
+#pragma unroll
+          for (int v = 0; v < CB / 4; ++v)
+            *reinterpret_cast<uint4 *>(dst + v * 4) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+          if (quad == 0) p.part_ml[slot] = make_float2(pend.m_ref, l_row);
+        }
+      }
+      pend.valid = false;
+      if (kProfile) prof_acc[3] += clock64() - pe0;
+      return true;
     };
     ItemInfo I, Inext;
     int idx = item_index(0);
@@ -416,11 +469,11 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
           if (!ok) break;
           fence_after();
           uint32_t o[CB];
-          tmem_ld<CB>(tmem + Cfg::kColO + lane_addr, o);
+          tmem_ld<CB>(tmem + Cfg::kColO + (qc & 1) * CB + lane_addr, o);
           wait_ld();
 #pragma unroll
           for (int i = 0; i < CB; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-          tmem_st<CB>(tmem + Cfg::kColO + lane_addr, o);
+          tmem_st<CB>(tmem + Cfg::kColO + (qc & 1) * CB + lane_addr, o);
           wait_st();
         }
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
@@ -453,71 +506,32 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
           const int per_half = (kTileTokens - ntok) * 8;
           for (int i = sm_tid; i < per_half * Cfg::kHalves; i += 128) {
             const int h = i / per_half, rem = i % per_half;
-            *reinterpret_cast<uint4 *>(vt + h * Cfg::kHalfBytes + (ntok + rem / 8) * 128 + (rem % 8) * 16) = make_uint4(0, 0, 0, 0);
+            const int tok = ntok + rem / 8;
+            *reinterpret_cast<uint4 *>(vt + (tok >> 3) * 1024 + h * Cfg::kHalfBytes + (tok & 7) * 128 + (rem % 8) * 16) = make_uint4(0, 0, 0, 0);
           }
         }
         fence_async_smem();
         fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->p_full[b]);
-        ok = q_step();
+        if (pend.valid) ok = run_epilogue();  // previous item (its sL became visible at this tile's barrier)
+        if (ok) ok = q_step();
       }
       while (ok && q_stage < 2) ok = q_step();
       if (!ok) break;
 
-      // ---- epilogue: row sums of the four quadrants, then each thread finishes its D/4 columns
-      const long long prof_e0 = kProfile ? clock64() : 0;
-      sL[quad * 32 + row] = l_sum;
-      ok = softmax_sync();
-      if (!ok) break;
-      const long long prof_e1 = kProfile ? clock64() : 0;
-      const float l_row = sL[row] + sL[32 + row] + sL[64 + row] + sL[96 + row];
-      ok = warp_wait(&bars->pv_done[(tc_ - 1) & 1], ((tc_ - 1) >> 1) & 1, 1);
-      if (!ok) break;
-      fence_after();
-      const long long prof_e2 = kProfile ? clock64() : 0;
-      {
-        uint32_t o[CB];
-        tmem_ld<CB>(tmem + Cfg::kColO + lane_addr, o);
-        wait_ld();
-        // O has been read: the next item may overwrite it
-        fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->o_free);
-        const int j = row / p.G, hg = row % p.G;
-        if (valid_row) {
-          if (I.part_slot < 0) {
-            const float inv = 1.f / l_row;
-            __nv_bfloat16 *dst = out + ((int64_t)(I.q0 + j) * p.Hq + I.g * p.G + hg) * D + quad * CB;
-#pragma unroll
-            for (int v = 0; v < CB / 8; ++v) {
-              uint4 u;
-              u.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-              u.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-              u.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-              u.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-              *reinterpret_cast<uint4 *>(dst + v * 8) = u;
-            }
-            if (quad == 0 && p.lse) p.lse[(int64_t)(I.q0 + j) * p.Hq + I.g * p.G + hg] = (m_ref + log2f(l_row)) * kLn2;
-          } else {
-            const int64_t slot = ((int64_t)I.part_slot * p.Hkv + I.g) * p.rows_cap + row;
-            float *dst = p.part_o + slot * D + quad * CB;
-#pragma unroll
-            for (int v = 0; v < CB / 4; ++v)
-              *reinterpret_cast<uint4 *>(dst + v * 4) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
-            if (quad == 0) p.part_ml[slot] = make_float2(m_ref, l_row);
-          }
-        }
-      }
-      if (kProfile) {
-        const long long now = clock64();
-        prof_acc[3] += now - prof_e0;  // whole epilogue
-        prof_x[0] += prof_e1 - prof_e0;  // wait for the last PV
-        prof_x[1] += prof_e2 - prof_e1;  // first sync
-        prof_x[2] += now - prof_e2;      // merge loop + stores
-      }
+      // ---- the item's epilogue is deferred: it runs after the first tile of the next item, when
+      // the last PV has long completed, so the softmax never idles at an item boundary
+      sL[((qc & 1) * 4 + quad) * 32 + row] = l_sum;
+      pend.valid = true; pend.I = I; pend.m_ref = m_ref; pend.last_tc = tc_ - 1; pend.qc = qc;
+      const long long prof_e0 = 0, prof_e1 = 0, prof_e2 = 0;
+      (void)prof_e0; (void)prof_e1; (void)prof_e2;
       idx = idx_next;
       I = Inext;
+    }
+    if (ok && pend.valid && !bars->abort) {
+      ok = softmax_sync();  // make the last item's row sums visible
+      if (ok) ok = run_epilogue();
     }
   }
   if (kProfile && p.prof && lane == 0 && (warp == 0 || warp == 1 || warp == 4)) {

@@ -2,11 +2,12 @@
 // test, residual / bonus inverse-CDF draw.
 //
 // Every logits row is cut into segments of kSegElems tokens.  Pass 1 (row_stats_kernel, the
-// bandwidth-bound kernel) reduces each segment to (max, sum exp(x - max)).  accept_kernel merges
-// the segment pairs per row in float64, evaluates p(x)/q(x) for the drafts in order and fixes
-// n.  resid_seg_kernel re-reads rows n of the rejecting requests and reduces max(0, p - q) per
-// segment.  select_kernel picks the segment by a float64 scan of the segment masses and the
-// token by an fp32 scan inside that one segment.
+// bandwidth-bound kernel: persistent blocks that prefetch their next segment while reducing the
+// current one) reduces each segment to (max, sum exp(x - max)).  accept_kernel (one warp per
+// request, one lane per row) merges the segment pairs per row, evaluates p(x)/q(x) for the
+// drafts in float64 and fixes n.  resid_select_kernel re-reads rows n of the rejecting requests,
+// reduces max(0, p - q) per segment, and the block that finishes a request last picks the
+// segment by a float64 scan of the segment masses and the token by an fp32 scan inside it.
 #pragma once
 #include "common.cuh"
 
@@ -32,6 +33,7 @@ struct SampleParams {
   float2 *seg_stats;   // [(TQ+TD)][nseg]  (max in log2 domain, sum)
   float *seg_resid;    // [B][nseg]        residual mass of each segment of row n (units of 1)
   float4 *req_norm;    // [B]  (Mt, 1/St, Md, 1/Sd) of row n, log2 domain maxima; Md = NaN => bonus
+  int32_t *req_done;   // [B]  segments of row n finished (zeroed by accept_kernel)
   int32_t *dev_status;
 };
 
@@ -85,69 +87,106 @@ __device__ __forceinline__ void merge_ms(float &m, float &s, float m2, float s2)
   m = mn;
 }
 
-// Pass 1.  grid = (nseg, TQ + TD).  Rows [0,TQ) are target rows, [TQ, TQ+TD) draft rows.
-// Threads interleave 16-byte vectors so that a warp reads 512 contiguous bytes per load.
+// Raw 16-byte loads of one segment slice owned by a thread (vectors interleaved across the block
+// so that a warp reads 512 contiguous bytes per load).  Vectors that straddle the end of the
+// vocabulary are not loaded here; convert() reads their in-range elements one by one.
 template <typename T>
-__global__ void __launch_bounds__(kSampThreads) row_stats_kernel(SampleParams p) {
-  constexpr int N = Vec<T>::N;
-  constexpr int NV = kElemsPerThread / N;  // vectors per thread
-  const int seg = blockIdx.x, row = blockIdx.y;
-  const T *base = (row < p.total_q)
-                      ? reinterpret_cast<const T *>(p.target) + (int64_t)row * p.row_stride
-                      : reinterpret_cast<const T *>(p.draft) + (int64_t)(row - p.total_q) * p.row_stride;
-  const int seg0 = seg * kSegElems;
-  float x[NV][N];
+struct SegSlice {
+  static constexpr int N = Vec<T>::N;
+  static constexpr int NV = kElemsPerThread / N;
+  uint4 raw[NV];
+  const T *base;
+  int seg0;
+  __device__ __forceinline__ void issue(const T *row_base, int seg, int vocab) {
+    base = row_base;
+    seg0 = seg * kSegElems;
 #pragma unroll
-  for (int c = 0; c < NV; ++c) {
-    const int v = seg0 + (c * kSampThreads + threadIdx.x) * N;
-    if (v + N <= p.vocab) {
-      Vec<T>::load(base + v, x[c]);
-    } else {
-#pragma unroll
-      for (int i = 0; i < N; ++i) x[c][i] = (v + i < p.vocab) ? ld_as_float(base, v + i) * kLog2e : -INFINITY;
+    for (int c = 0; c < NV; ++c) {
+      const int v = seg0 + (c * kSampThreads + threadIdx.x) * N;
+      if (v + N <= vocab) raw[c] = __ldg(reinterpret_cast<const uint4 *>(row_base + v));
     }
   }
-  float m = -INFINITY;
+  // element c*N+i of the slice in the log2 domain (-inf beyond the vocabulary)
+  __device__ __forceinline__ void convert(int c, int vocab, float (&f)[N]) const {
+    const int v = seg0 + (c * kSampThreads + threadIdx.x) * N;
+    if (v + N <= vocab) {
+      if constexpr (N == 8) {
+        const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
 #pragma unroll
-  for (int c = 0; c < NV; ++c)
+        for (int i = 0; i < 4; ++i) {
+          f[2 * i] = __uint_as_float(w[i] << 16) * kLog2e;
+          f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u) * kLog2e;
+        }
+      } else {
+        f[0] = __uint_as_float(raw[c].x) * kLog2e; f[1] = __uint_as_float(raw[c].y) * kLog2e;
+        f[2] = __uint_as_float(raw[c].z) * kLog2e; f[3] = __uint_as_float(raw[c].w) * kLog2e;
+      }
+    } else {
 #pragma unroll
-    for (int i = 0; i < N; ++i) m = fmaxf(m, x[c][i]);
-  float s = 0.f;
-  if (m > -INFINITY) {
-#pragma unroll
-    for (int c = 0; c < NV; ++c)
-#pragma unroll
-      for (int i = 0; i < N; ++i) s += fast_exp2(x[c][i] - m);
+      for (int i = 0; i < N; ++i) f[i] = (v + i < vocab) ? ld_as_float(base, v + i) * kLog2e : -INFINITY;
+    }
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
-    const float s2 = __shfl_xor_sync(0xffffffffu, s, o);
-    merge_ms(m, s, m2, s2);
-  }
-  __shared__ float2 s_w[kSampThreads / 32];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (lane == 0) s_w[warp] = make_float2(m, s);
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    for (int w = 1; w < kSampThreads / 32; ++w) merge_ms(m, s, s_w[w].x, s_w[w].y);
-    p.seg_stats[(int64_t)row * p.nseg + seg] = make_float2(m, s);
-  }
-}
+};
 
-// Row normalisers from segment pairs, in float64: returns max M (log2 domain) and S = sum 2^(x-M).
-__device__ __forceinline__ void row_norm(const float2 *st, int nseg, float &M, double &S) {
-  M = -INFINITY;
-  for (int i = 0; i < nseg; ++i) M = fmaxf(M, st[i].x);
-  S = 0.0;
-  for (int i = 0; i < nseg; ++i) S += (double)st[i].y * exp2((double)st[i].x - (double)M);
-}
-
-// One thread per request (the work is k+1 tiny serial steps).  Fixes n, writes accepted_len, the
-// accepted ids and the -1 padding; leaves slot n for select_kernel.
+// Pass 1.  Persistent blocks; unit u = row * nseg + seg, rows [0,TQ) target, [TQ,TQ+TD) draft.
+// Each block reduces its units in turn and has the loads of the following unit in flight
+// meanwhile.
 template <typename T>
-__global__ void accept_kernel(SampleParams p) {
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+__global__ void __launch_bounds__(kSampThreads) row_stats_kernel(SampleParams p, int n_units) {
+  constexpr int N = Vec<T>::N;
+  constexpr int NV = kElemsPerThread / N;
+  __shared__ float2 s_w[2][kSampThreads / 32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  auto row_base = [&](int u) -> const T * {
+    const int row = u / p.nseg;
+    return (row < p.total_q) ? reinterpret_cast<const T *>(p.target) + (int64_t)row * p.row_stride
+                             : reinterpret_cast<const T *>(p.draft) + (int64_t)(row - p.total_q) * p.row_stride;
+  };
+  SegSlice<T> cur, nxt;
+  int u = blockIdx.x;
+  if (u < n_units) cur.issue(row_base(u), u % p.nseg, p.vocab);
+  for (int it = 0; u < n_units; u += gridDim.x, ++it) {
+    const int un = u + gridDim.x;
+    if (un < n_units) nxt.issue(row_base(un), un % p.nseg, p.vocab);
+    float m = -INFINITY;
+    float x[NV][N];
+#pragma unroll
+    for (int c = 0; c < NV; ++c) {
+      cur.convert(c, p.vocab, x[c]);
+#pragma unroll
+      for (int i = 0; i < N; ++i) m = fmaxf(m, x[c][i]);
+    }
+    float s = 0.f;
+    if (m > -INFINITY) {
+#pragma unroll
+      for (int c = 0; c < NV; ++c)
+#pragma unroll
+        for (int i = 0; i < N; ++i) s += fast_exp2(x[c][i] - m);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+      const float s2 = __shfl_xor_sync(0xffffffffu, s, o);
+      merge_ms(m, s, m2, s2);
+    }
+    if (lane == 0) s_w[it & 1][warp] = make_float2(m, s);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int w = 1; w < kSampThreads / 32; ++w) merge_ms(m, s, s_w[it & 1][w].x, s_w[it & 1][w].y);
+      p.seg_stats[u] = make_float2(m, s);
+    }
+    cur = nxt;
+  }
+}
+
+// One warp per request, lane = row (lanes 0..k: target rows, lanes k+1..2k: draft rows).  Each lane
+// merges its row's segment pairs (fp32 exponentials, float64 sum); the accept ratios of all
+// drafts are evaluated in parallel in float64 and the first failure fixes n.  Writes
+// accepted_len, the accepted ids and the -1 padding; slot n is left for resid_select_kernel.
+template <typename T>
+__global__ void __launch_bounds__(128) accept_kernel(SampleParams p) {
+  const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
   if (r >= p.batch) return;
   const int t0 = p.q_indptr[r];
   const int k = p.q_indptr[r + 1] - t0 - 1;
@@ -155,90 +194,111 @@ __global__ void accept_kernel(SampleParams p) {
   const T *target = reinterpret_cast<const T *>(p.target);
   const T *draft = reinterpret_cast<const T *>(p.draft);
   const float nanf_ = __int_as_float(0x7fc00000);
+  if (lane == 0) p.req_done[r] = 0;
   if (k < 0 || k > SPX_MAX_K || t0 < 0 || t0 + k + 1 > p.total_q) {
-    atomicOr(p.dev_status, SPX_DEV_BAD_LEN);
-    p.accepted_len[r] = 0;
-    p.req_norm[r] = make_float4(nanf_, nanf_, nanf_, -1.f);  // w < 0: skip this request
+    if (lane == 0) {
+      atomicOr(p.dev_status, SPX_DEV_BAD_LEN);
+      p.accepted_len[r] = 0;
+      p.req_norm[r] = make_float4(nanf_, nanf_, nanf_, -1.f);  // w < 0: skip this request
+    }
     return;
   }
+  int x = 0;
   bool bad = false;
-  for (int i = 0; i < k; ++i) {
-    const int x = p.draft_ids[d0 + i];
-    if (x < 0 || x >= p.vocab) bad = true;
-    if (p.diag_ratio) p.diag_ratio[d0 + i] = nanf_;
+  if (lane < k) {
+    x = p.draft_ids[d0 + lane];
+    bad = x < 0 || x >= p.vocab;
+    if (p.diag_ratio) p.diag_ratio[d0 + lane] = nanf_;
   }
-  if (bad) {
-    atomicOr(p.dev_status, SPX_DEV_BAD_TOKEN);
-    p.accepted_len[r] = 0;
-    for (int i = 0; i <= k; ++i) p.out_tokens[t0 + i] = -1;
-    p.req_norm[r] = make_float4(nanf_, nanf_, nanf_, -1.f);
+  if (__any_sync(0xffffffffu, bad)) {
+    if (lane == 0) {
+      atomicOr(p.dev_status, SPX_DEV_BAD_TOKEN);
+      p.accepted_len[r] = 0;
+      p.req_norm[r] = make_float4(nanf_, nanf_, nanf_, -1.f);
+    }
+    if (lane <= k) p.out_tokens[t0 + lane] = -1;
     return;
   }
-  int n = k;
-  float Mt = 0.f, Md = 0.f;
-  double St = 1.0, Sd = 1.0;
-  for (int i = 0; i < k; ++i) {
-    row_norm(p.seg_stats + (int64_t)(t0 + i) * p.nseg, p.nseg, Mt, St);
-    row_norm(p.seg_stats + (int64_t)(p.total_q + d0 + i) * p.nseg, p.nseg, Md, Sd);
-    const int x = p.draft_ids[d0 + i];
-    const double tx = (double)(ld_as_float(target, (int64_t)(t0 + i) * p.row_stride + x) * kLog2e);
-    const double dx = (double)(ld_as_float(draft, (int64_t)(d0 + i) * p.row_stride + x) * kLog2e);
-    // rho = p(x)/q(x) = 2^(tx-Mt)/St * Sd/2^(dx-Md)
-    const double rho = exp2((tx - (double)Mt) - (dx - (double)Md)) * (Sd / St);
-    if (p.diag_ratio) p.diag_ratio[d0 + i] = (float)rho;
-    if (!((double)p.u_accept[d0 + i] < rho)) { n = i; break; }
+  // row normalisers: M (log2 domain) and S = sum 2^(x - M)
+  float M = -INFINITY;
+  double S = 0.0;
+  if (lane < 2 * k + 1) {
+    const int row = lane <= k ? t0 + lane : p.total_q + d0 + (lane - k - 1);
+    const float2 *st = p.seg_stats + (int64_t)row * p.nseg;
+    for (int i = 0; i < p.nseg; ++i) M = fmaxf(M, st[i].x);
+    for (int i = 0; i < p.nseg; ++i) S += (double)(st[i].y * fast_exp2(st[i].x - M));
   }
-  p.accepted_len[r] = n;
-  for (int i = 0; i < n; ++i) p.out_tokens[t0 + i] = p.draft_ids[d0 + i];
-  for (int i = n + 1; i <= k; ++i) p.out_tokens[t0 + i] = -1;
-  if (n < k) {
-    p.req_norm[r] = make_float4(Mt, (float)(1.0 / St), Md, (float)(1.0 / Sd));
-  } else {
-    row_norm(p.seg_stats + (int64_t)(t0 + k) * p.nseg, p.nseg, Mt, St);
-    p.req_norm[r] = make_float4(Mt, (float)(1.0 / St), nanf_, 0.f);
+  // lane i < k pairs target row i (its own) with draft row i (lane k+1+i)
+  const float Md = __shfl_sync(0xffffffffu, M, (k + 1 + lane) & 31);
+  const double Sd = __shfl_sync(0xffffffffu, S, (k + 1 + lane) & 31);
+  bool reject = false;
+  if (lane < k) {
+    const double tx = (double)(ld_as_float(target, (int64_t)(t0 + lane) * p.row_stride + x) * kLog2e);
+    const double dx = (double)(ld_as_float(draft, (int64_t)(d0 + lane) * p.row_stride + x) * kLog2e);
+    // rho = p(x)/q(x) = 2^(tx-Mt)/St * Sd/2^(dx-Md)
+    const double rho = exp2((tx - (double)M) - (dx - (double)Md)) * (Sd / S);
+    reject = !((double)p.u_accept[d0 + lane] < rho);
+    if (p.diag_ratio) p.diag_ratio[d0 + lane] = (float)rho;
+  }
+  const uint32_t rej_mask = __ballot_sync(0xffffffffu, reject);
+  const int n = rej_mask ? __ffs(rej_mask) - 1 : k;
+  if (p.diag_ratio && lane < k && lane > n) p.diag_ratio[d0 + lane] = nanf_;  // rows after n are not consulted
+  if (lane == 0) p.accepted_len[r] = n;
+  if (lane < n) p.out_tokens[t0 + lane] = x;
+  if (lane > n && lane <= k) p.out_tokens[t0 + lane] = -1;
+  // normalisers of row n for the residual pass (target: lane n; draft: lane k+1+n)
+  const float Mt_n = __shfl_sync(0xffffffffu, M, n);
+  const double St_n = __shfl_sync(0xffffffffu, S, n);
+  const float Md_n = __shfl_sync(0xffffffffu, M, (k + 1 + n) & 31);
+  const double Sd_n = __shfl_sync(0xffffffffu, S, (k + 1 + n) & 31);
+  if (lane == 0) {
+    if (n < k) p.req_norm[r] = make_float4(Mt_n, (float)(1.0 / St_n), Md_n, (float)(1.0 / Sd_n));
+    else p.req_norm[r] = make_float4(Mt_n, (float)(1.0 / St_n), nanf_, 0.f);
   }
 }
 
-// Residual mass per segment of row n for rejecting requests.  grid = (nseg, B).
+// Residual mass per segment of row n, then the final draw by the block that finishes the request
+// last (bonus requests need no residual pass: their block 0 draws at once).  grid = (nseg, B).
+// Segment choice in float64 over the segment masses, token choice by an fp32 scan of the chosen
+// segment (thread t owns tokens [32t, 32t+32) of it).
 template <typename T>
-__global__ void __launch_bounds__(kSampThreads) resid_seg_kernel(SampleParams p) {
-  const int seg = blockIdx.x, r = blockIdx.y;
+__global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams p) {
+  const int seg_mine = blockIdx.x, r = blockIdx.y;
   const float4 nm = p.req_norm[r];
-  if (nm.w < 0.f || nm.z != nm.z) return;  // invalid request, or bonus case (segment stats suffice)
+  if (nm.w < 0.f) return;  // invalid request
+  const bool bonus = (nm.z != nm.z);
+  if (bonus && seg_mine != 0) return;
   const int t0 = p.q_indptr[r];
   const int n = p.accepted_len[r];
   const T *trow = reinterpret_cast<const T *>(p.target) + (int64_t)(t0 + n) * p.row_stride;
   const T *drow = reinterpret_cast<const T *>(p.draft) + (int64_t)(t0 - r + n) * p.row_stride;
-  const int v0 = seg * kSegElems + threadIdx.x * kElemsPerThread;
-  float xt[kElemsPerThread], xd[kElemsPerThread];
-  load_thread_span(trow, v0, p.vocab, xt);
-  load_thread_span(drow, v0, p.vocab, xd);
-  float acc = 0.f;
-#pragma unroll
-  for (int i = 0; i < kElemsPerThread; ++i)
-    acc += fmaxf(0.f, fast_exp2(xt[i] - nm.x) * nm.y - fast_exp2(xd[i] - nm.z) * nm.w);
-  acc = warp_sum(acc);
-  __shared__ float s_w[kSampThreads / 32];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (lane == 0) s_w[warp] = acc;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    float tot = 0.f;
-    for (int w = 0; w < kSampThreads / 32; ++w) tot += s_w[w];
-    p.seg_resid[(int64_t)r * p.nseg + seg] = tot;
+  __shared__ float s_w[kSampThreads / 32];
+  __shared__ int s_last;
+  if (!bonus) {
+    const int v0 = seg_mine * kSegElems + threadIdx.x * kElemsPerThread;
+    float xt[kElemsPerThread], xd[kElemsPerThread];
+    load_thread_span(trow, v0, p.vocab, xt);
+    load_thread_span(drow, v0, p.vocab, xd);
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < kElemsPerThread; ++i)
+      acc += fmaxf(0.f, fast_exp2(xt[i] - nm.x) * nm.y - fast_exp2(xd[i] - nm.z) * nm.w);
+    acc = warp_sum(acc);
+    if (lane == 0) s_w[warp] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float tot = 0.f;
+      for (int w = 0; w < kSampThreads / 32; ++w) tot += s_w[w];
+      p.seg_resid[(int64_t)r * p.nseg + seg_mine] = tot;
+      __threadfence();
+      s_last = (atomicAdd(&p.req_done[r], 1) == p.nseg - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();  // the other blocks' segment masses are visible from here on
   }
-}
 
-// Final draw.  grid = B, block = 256.  Segment choice in float64, token choice by an fp32 scan of
-// the chosen segment (thread t owns tokens [32t, 32t+32) of the segment).
-template <typename T>
-__global__ void __launch_bounds__(kSampThreads) select_kernel(SampleParams p) {
-  const int r = blockIdx.x;
-  float4 nm = p.req_norm[r];
-  if (nm.w < 0.f) return;
-  const bool bonus = (nm.z != nm.z);
-  const int t0 = p.q_indptr[r];
-  const int n = p.accepted_len[r];
   const float2 *tstats = p.seg_stats + (int64_t)(t0 + n) * p.nseg;
   __shared__ int s_seg;
   __shared__ float s_target;
@@ -247,25 +307,24 @@ __global__ void __launch_bounds__(kSampThreads) select_kernel(SampleParams p) {
   __shared__ int s_tok;
   if (threadIdx.x == 0) {
     // segment masses (float64), total R, target s*R, first segment whose inclusive sum exceeds it
+    const volatile float *resid = p.seg_resid + (int64_t)r * p.nseg;
     double R = 0.0;
     int degenerate = 0;
     if (!bonus) {
-      for (int i = 0; i < p.nseg; ++i) R += (double)p.seg_resid[(int64_t)r * p.nseg + i];
+      for (int i = 0; i < p.nseg; ++i) R += (double)resid[i];
       if (!(R > 0.0)) degenerate = 1;
     }
     const bool use_target = bonus || degenerate;
     if (use_target) {
       R = 0.0;
-      for (int i = 0; i < p.nseg; ++i) R += (double)tstats[i].y * exp2((double)tstats[i].x - (double)nm.x) * (double)nm.y;
+      for (int i = 0; i < p.nseg; ++i) R += (double)(tstats[i].y * fast_exp2(tstats[i].x - nm.x)) * (double)nm.y;
     }
     const double target = (double)p.u_sample[r] * R;
     double cum = 0.0;
     int seg = -1, last_pos = -1;
     double before = 0.0, last_before = 0.0;
     for (int i = 0; i < p.nseg; ++i) {
-      const double mass = use_target
-                              ? (double)tstats[i].y * exp2((double)tstats[i].x - (double)nm.x) * (double)nm.y
-                              : (double)p.seg_resid[(int64_t)r * p.nseg + i];
+      const double mass = use_target ? (double)(tstats[i].y * fast_exp2(tstats[i].x - nm.x)) * (double)nm.y : (double)resid[i];
       if (mass > 0.0) { last_pos = i; last_before = cum; }
       if (cum + mass > target) { seg = i; before = cum; break; }
       cum += mass;
@@ -274,6 +333,7 @@ __global__ void __launch_bounds__(kSampThreads) select_kernel(SampleParams p) {
     s_seg = seg;
     s_target = (float)(target - before);
     s_degenerate = degenerate;
+    s_tok = 0x7fffffff;
     if (degenerate) atomicOr(p.dev_status, SPX_DEV_DEGENERATE);
   }
   __syncthreads();
@@ -284,8 +344,6 @@ __global__ void __launch_bounds__(kSampThreads) select_kernel(SampleParams p) {
   }
   const bool use_target = bonus || s_degenerate;
   const float target = s_target;
-  const T *trow = reinterpret_cast<const T *>(p.target) + (int64_t)(t0 + n) * p.row_stride;
-  const T *drow = reinterpret_cast<const T *>(p.draft) + (int64_t)(t0 - r + n) * p.row_stride;
   const int v0 = seg * kSegElems + threadIdx.x * kElemsPerThread;
   float w[kElemsPerThread];
   {
@@ -306,7 +364,6 @@ __global__ void __launch_bounds__(kSampThreads) select_kernel(SampleParams p) {
 #pragma unroll
   for (int i = 0; i < kElemsPerThread; ++i) tsum += w[i];
   // block exclusive scan of thread sums
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   float incl = tsum;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -314,21 +371,22 @@ __global__ void __launch_bounds__(kSampThreads) select_kernel(SampleParams p) {
     if (lane >= o) incl += nb;
   }
   if (lane == 31) s_scan[warp] = incl;
-  if (threadIdx.x == 0) s_tok = 0x7fffffff;
   __syncthreads();
   float woff = 0.f;
   for (int i = 0; i < warp; ++i) woff += s_scan[i];
   const float excl = woff + incl - tsum;
-  // the thread whose span contains the crossing walks it; ties across threads resolve to the
-  // smallest token through atomicMin
+  // the thread whose span contains the crossing walks it; if rounding leaves its running sum
+  // short of the target it takes its last token with positive weight
   if (excl <= target && excl + tsum > target) {
     float cum = excl;
-    int tok = -1;
+    int tok = -1, last = -1;
 #pragma unroll
     for (int i = 0; i < kElemsPerThread; ++i) {
       cum += w[i];
+      if (w[i] > 0.f) last = v0 + i;
       if (tok < 0 && cum > target) tok = v0 + i;
     }
+    if (tok < 0) tok = last;
     if (tok >= 0) atomicMin(&s_tok, tok);
   }
   __syncthreads();
