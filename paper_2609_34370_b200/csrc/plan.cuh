@@ -130,60 +130,66 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int target_chu
 
 // Merge the chunk partials of split requests: m* = max_c m_c, l* = sum_c 2^(m_c-m*) l_c,
 // O = sum_c 2^(m_c-m*) O_c / l*, LSE = (m* + log2 l*) ln 2.  Also writes the sentinel rows of
-// invalid requests.  grid = (B * Hkv), block = 256.
+// invalid requests.  grid = (B * Hkv, ceil(rows_cap * D/4 / 256)), block = 256: one thread per
+// (row, 4 columns), chunks walked four at a time so that their loads are in flight together.
 template <typename T>
 __global__ void __launch_bounds__(256) combine_kernel(AttnParams p) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the attention kernel's partials (no-op without PDL)
   const int r = blockIdx.x / p.Hkv, g = blockIdx.x % p.Hkv;
   const int nch = p.req_nchunks[r];
   const int q0 = p.q_indptr[r];
   int m = p.q_indptr[r + 1] - q0;
   T *out = reinterpret_cast<T *>(p.out);
   const int D = p.D, G = p.G;
+  const int vecs = D / 4;
+  const int item = blockIdx.y * blockDim.x + threadIdx.x;  // (row, dv)
   if (nch == 0 || p.hdr->overflow || p.req_bad[r]) {
     // invalid request (or unusable plan): zero rows, NaN lse; clamp the row range to the tensor
     if (m < 0) m = 0;
     if (m > p.max_q_len) m = p.max_q_len;
     if (q0 < 0 || q0 + m > p.total_q) return;
-    for (int i = threadIdx.x; i < m * G * D; i += blockDim.x) {
-      const int row = i / D, d = i % D, j = row / G, hg = row % G;
-      st_from_float(out, ((int64_t)(q0 + j) * p.Hq + g * G + hg) * D + d, 0.f);
+    if (item < m * G * vecs) {
+      const int row = item / vecs, dv = item % vecs, j = row / G, hg = row % G;
+      const int64_t o_idx = ((int64_t)(q0 + j) * p.Hq + g * G + hg) * D + dv * 4;
+      for (int i = 0; i < 4; ++i) st_from_float(out, o_idx + i, 0.f);
+      if (dv == 0 && p.lse) p.lse[(int64_t)(q0 + j) * p.Hq + g * G + hg] = __int_as_float(0x7fc00000);
     }
-    if (p.lse)
-      for (int row = threadIdx.x; row < m * G; row += blockDim.x)
-        p.lse[(int64_t)(q0 + row / G) * p.Hq + g * G + row % G] = __int_as_float(0x7fc00000);
     return;
   }
   if (nch == 1) return;  // written directly by the attention kernel
-  const int rows = m * G;
-  const int base = p.req_part_base[r];
-  const int vecs = D / 4;
-  for (int i = threadIdx.x; i < rows * vecs; i += blockDim.x) {
-    const int row = i / vecs, dv = i % vecs;
-    float mstar = -INFINITY;
-    for (int c = 0; c < nch; ++c) {
-      const float2 ml = p.part_ml[((int64_t)(base + c) * p.Hkv + g) * p.rows_cap + row];
-      mstar = fmaxf(mstar, ml.x);
+  if (item >= m * G * vecs) return;
+  const int row = item / vecs, dv = item % vecs;
+  const int64_t slot0 = ((int64_t)p.req_part_base[r] * p.Hkv + g) * p.rows_cap + row;
+  const int64_t slot_step = (int64_t)p.Hkv * p.rows_cap;
+  float mstar = -INFINITY;
+  for (int c = 0; c < nch; ++c) mstar = fmaxf(mstar, p.part_ml[slot0 + c * slot_step].x);
+  float lstar = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int c0 = 0; c0 < nch; c0 += 4) {
+    float2 ml[4];
+    float4 o[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int c = min(c0 + u, nch - 1);
+      ml[u] = p.part_ml[slot0 + c * slot_step];
+      o[u] = *reinterpret_cast<const float4 *>(p.part_o + (slot0 + c * slot_step) * D + dv * 4);
     }
-    float lstar = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c = 0; c < nch; ++c) {
-      const int64_t slot = ((int64_t)(base + c) * p.Hkv + g) * p.rows_cap + row;
-      const float2 ml = p.part_ml[slot];
-      if (ml.x == -INFINITY) continue;
-      const float w = fast_exp2(ml.x - mstar);
-      lstar += w * ml.y;
-      const float4 o = *reinterpret_cast<const float4 *>(p.part_o + slot * D + dv * 4);
-      acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (c0 + u >= nch || ml[u].x == -INFINITY) continue;
+      const float w = fast_exp2(ml[u].x - mstar);
+      lstar += w * ml[u].y;
+      acc.x += w * o[u].x; acc.y += w * o[u].y; acc.z += w * o[u].z; acc.w += w * o[u].w;
     }
-    const float inv = 1.f / lstar;
-    const int j = row / G, hg = row % G;
-    const int64_t o_idx = ((int64_t)(q0 + j) * p.Hq + g * G + hg) * D + dv * 4;
-    st_from_float(out, o_idx + 0, acc.x * inv);
-    st_from_float(out, o_idx + 1, acc.y * inv);
-    st_from_float(out, o_idx + 2, acc.z * inv);
-    st_from_float(out, o_idx + 3, acc.w * inv);
-    if (dv == 0 && p.lse) p.lse[(int64_t)(q0 + j) * p.Hq + g * G + hg] = (mstar + log2f(lstar)) * kLn2;
   }
+  const float inv = 1.f / lstar;
+  const int j = row / G, hg = row % G;
+  const int64_t o_idx = ((int64_t)(q0 + j) * p.Hq + g * G + hg) * D + dv * 4;
+  st_from_float(out, o_idx + 0, acc.x * inv);
+  st_from_float(out, o_idx + 1, acc.y * inv);
+  st_from_float(out, o_idx + 2, acc.z * inv);
+  st_from_float(out, o_idx + 3, acc.w * inv);
+  if (dv == 0 && p.lse) p.lse[(int64_t)(q0 + j) * p.Hq + g * G + hg] = (mstar + log2f(lstar)) * kLn2;
 }
 
 }  // namespace spx

@@ -1,9 +1,10 @@
 // Speculative rejection sampling: vocabulary-parallel softmax statistics, sequential accept
 // test, residual / bonus inverse-CDF draw.
 //
-// Every logits row is cut into segments of kSegElems tokens.  Pass 1 (row_stats_kernel, the
-// bandwidth-bound kernel: persistent blocks that prefetch their next segment while reducing the
-// current one) reduces each segment to (max, sum exp(x - max)).  accept_kernel (one warp per
+// Every logits row is cut into sub-segments of kSubElems tokens, four of which make a segment of
+// kSegElems.  Pass 1 (row_stats_kernel, the bandwidth-bound kernel: persistent warps, each with
+// the loads of its next sub-segment in flight while it reduces the current one, no block-level
+// synchronisation) reduces each sub-segment to (max, sum exp(x - max)).  accept_kernel (one warp per
 // request, one lane per row) merges the segment pairs per row, evaluates p(x)/q(x) for the
 // drafts in float64 and fixes n.  resid_select_kernel re-reads rows n of the rejecting requests,
 // reduces max(0, p - q) per segment, and the block that finishes a request last picks the
@@ -13,12 +14,14 @@
 
 namespace spx {
 
-constexpr int kSegElems = 8192;       // tokens per segment
+constexpr int kSegElems = 8192;       // tokens per segment (residual pass, final draw)
+constexpr int kSubElems = 2048;       // tokens per sub-segment (statistics pass)
+constexpr int kSubPerSeg = kSegElems / kSubElems;
 constexpr int kSampThreads = 256;
 constexpr int kElemsPerThread = kSegElems / kSampThreads;  // 32
 
 struct SampleParams {
-  int32_t batch, total_q, total_d, vocab, nseg;
+  int32_t batch, total_q, total_d, vocab, nseg, nsub;
   int64_t row_stride;
   const void *target;
   const void *draft;
@@ -30,7 +33,7 @@ struct SampleParams {
   int32_t *out_tokens;
   float *diag_ratio;
   // workspace
-  float2 *seg_stats;   // [(TQ+TD)][nseg]  (max in log2 domain, sum)
+  float2 *seg_stats;   // [(TQ+TD)][nsub]  per sub-segment (max in log2 domain, sum)
   float *seg_resid;    // [B][nseg]        residual mass of each segment of row n (units of 1)
   float4 *req_norm;    // [B]  (Mt, 1/St, Md, 1/Sd) of row n, log2 domain maxima; Md = NaN => bonus
   int32_t *req_done;   // [B]  segments of row n finished (zeroed by accept_kernel)
@@ -87,94 +90,103 @@ __device__ __forceinline__ void merge_ms(float &m, float &s, float m2, float s2)
   m = mn;
 }
 
-// Raw 16-byte loads of one segment slice owned by a thread (vectors interleaved across the block
-// so that a warp reads 512 contiguous bytes per load).  Vectors that straddle the end of the
-// vocabulary are not loaded here; convert() reads their in-range elements one by one.
+// The kSubElems / 32 tokens of a sub-segment that a lane owns, as raw 16-byte vectors interleaved
+// across the warp (a warp reads 512 contiguous bytes per load).  Vectors that straddle the end of
+// the vocabulary are assembled element by element with -inf padding.
 template <typename T>
-struct SegSlice {
-  static constexpr int N = Vec<T>::N;
-  static constexpr int NV = kElemsPerThread / N;
+struct SubSlice {
+  static constexpr int N = Vec<T>::N;                 // elements per 16-byte vector
+  static constexpr int NV = kSubElems / 32 / N;       // vectors per lane
   uint4 raw[NV];
-  const T *base;
-  int seg0;
-  __device__ __forceinline__ void issue(const T *row_base, int seg, int vocab) {
-    base = row_base;
-    seg0 = seg * kSegElems;
+  __device__ __forceinline__ void issue(const T *row_base, int sub, int vocab, int lane) {
 #pragma unroll
     for (int c = 0; c < NV; ++c) {
-      const int v = seg0 + (c * kSampThreads + threadIdx.x) * N;
-      if (v + N <= vocab) raw[c] = __ldg(reinterpret_cast<const uint4 *>(row_base + v));
-    }
-  }
-  // element c*N+i of the slice in the log2 domain (-inf beyond the vocabulary)
-  __device__ __forceinline__ void convert(int c, int vocab, float (&f)[N]) const {
-    const int v = seg0 + (c * kSampThreads + threadIdx.x) * N;
-    if (v + N <= vocab) {
-      if constexpr (N == 8) {
-        const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          f[2 * i] = __uint_as_float(w[i] << 16) * kLog2e;
-          f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u) * kLog2e;
-        }
+      const int v = sub * kSubElems + (c * 32 + lane) * N;
+      if (v + N <= vocab) {
+        raw[c] = __ldg(reinterpret_cast<const uint4 *>(row_base + v));
       } else {
-        f[0] = __uint_as_float(raw[c].x) * kLog2e; f[1] = __uint_as_float(raw[c].y) * kLog2e;
-        f[2] = __uint_as_float(raw[c].z) * kLog2e; f[3] = __uint_as_float(raw[c].w) * kLog2e;
-      }
-    } else {
+        union { uint4 u; T e[N]; } tmp;
 #pragma unroll
-      for (int i = 0; i < N; ++i) f[i] = (v + i < vocab) ? ld_as_float(base, v + i) * kLog2e : -INFINITY;
+        for (int i = 0; i < N; ++i) {
+          if (v + i < vocab) tmp.e[i] = row_base[v + i];
+          else st_from_float(tmp.e, i, -INFINITY);
+        }
+        raw[c] = tmp.u;
+      }
     }
   }
 };
 
-// Pass 1.  Persistent blocks; unit u = row * nseg + seg, rows [0,TQ) target, [TQ,TQ+TD) draft.
-// Each block reduces its units in turn and has the loads of the following unit in flight
-// meanwhile.
+// thread-local (max, sum 2^(x*log2e - max)) of a slice; the maximum is returned in the log2 domain
+__device__ __forceinline__ void slice_stats(const SubSlice<__nv_bfloat16> &sl, float &m, float &s) {
+  constexpr int NV = SubSlice<__nv_bfloat16>::NV;
+  // packed bf16 maximum: one instruction per two tokens
+  __nv_bfloat162 mx = *reinterpret_cast<const __nv_bfloat162 *>(&sl.raw[0].x);
+#pragma unroll
+  for (int c = 0; c < NV; ++c) {
+    const uint32_t w[4] = {sl.raw[c].x, sl.raw[c].y, sl.raw[c].z, sl.raw[c].w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) mx = __hmax2(mx, *reinterpret_cast<const __nv_bfloat162 *>(&w[i]));
+  }
+  m = fmaxf(__low2float(mx), __high2float(mx)) * kLog2e;
+  s = 0.f;
+  if (m == -INFINITY) return;
+#pragma unroll
+  for (int c = 0; c < NV; ++c) {
+    const uint32_t w[4] = {sl.raw[c].x, sl.raw[c].y, sl.raw[c].z, sl.raw[c].w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      s += fast_exp2(fmaf(__uint_as_float(w[i] << 16), kLog2e, -m));
+      s += fast_exp2(fmaf(__uint_as_float(w[i] & 0xffff0000u), kLog2e, -m));
+    }
+  }
+}
+__device__ __forceinline__ void slice_stats(const SubSlice<float> &sl, float &m, float &s) {
+  constexpr int NV = SubSlice<float>::NV;
+  float mx = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < NV; ++c)
+    mx = fmaxf(fmaxf(mx, fmaxf(__uint_as_float(sl.raw[c].x), __uint_as_float(sl.raw[c].y))),
+               fmaxf(__uint_as_float(sl.raw[c].z), __uint_as_float(sl.raw[c].w)));
+  m = mx * kLog2e;
+  s = 0.f;
+  if (m == -INFINITY) return;
+#pragma unroll
+  for (int c = 0; c < NV; ++c) {
+    s += fast_exp2(fmaf(__uint_as_float(sl.raw[c].x), kLog2e, -m));
+    s += fast_exp2(fmaf(__uint_as_float(sl.raw[c].y), kLog2e, -m));
+    s += fast_exp2(fmaf(__uint_as_float(sl.raw[c].z), kLog2e, -m));
+    s += fast_exp2(fmaf(__uint_as_float(sl.raw[c].w), kLog2e, -m));
+  }
+}
+
+// Pass 1.  Persistent warps; unit u = row * nsub + sub, rows [0,TQ) target, [TQ,TQ+TD) draft.
+// (Skipping the rows after a request's first rejection inside this pass was tried - rows walked
+// position-major, completion counters, a steering accept test - and measured slower: the
+// bookkeeping cost more than the 22 % of bytes it saved.)
 template <typename T>
 __global__ void __launch_bounds__(kSampThreads) row_stats_kernel(SampleParams p, int n_units) {
-  constexpr int N = Vec<T>::N;
-  constexpr int NV = kElemsPerThread / N;
-  __shared__ float2 s_w[2][kSampThreads / 32];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int warp_global = (blockIdx.x * kSampThreads + threadIdx.x) >> 5;
+  const int n_warps = (gridDim.x * kSampThreads) >> 5;
   auto row_base = [&](int u) -> const T * {
-    const int row = u / p.nseg;
+    const int row = u / p.nsub;
     return (row < p.total_q) ? reinterpret_cast<const T *>(p.target) + (int64_t)row * p.row_stride
                              : reinterpret_cast<const T *>(p.draft) + (int64_t)(row - p.total_q) * p.row_stride;
   };
-  SegSlice<T> cur, nxt;
-  int u = blockIdx.x;
-  if (u < n_units) cur.issue(row_base(u), u % p.nseg, p.vocab);
-  for (int it = 0; u < n_units; u += gridDim.x, ++it) {
-    const int un = u + gridDim.x;
-    if (un < n_units) nxt.issue(row_base(un), un % p.nseg, p.vocab);
-    float m = -INFINITY;
-    float x[NV][N];
-#pragma unroll
-    for (int c = 0; c < NV; ++c) {
-      cur.convert(c, p.vocab, x[c]);
-#pragma unroll
-      for (int i = 0; i < N; ++i) m = fmaxf(m, x[c][i]);
-    }
-    float s = 0.f;
-    if (m > -INFINITY) {
-#pragma unroll
-      for (int c = 0; c < NV; ++c)
-#pragma unroll
-        for (int i = 0; i < N; ++i) s += fast_exp2(x[c][i] - m);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
-      const float s2 = __shfl_xor_sync(0xffffffffu, s, o);
-      merge_ms(m, s, m2, s2);
-    }
-    if (lane == 0) s_w[it & 1][warp] = make_float2(m, s);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      for (int w = 1; w < kSampThreads / 32; ++w) merge_ms(m, s, s_w[it & 1][w].x, s_w[it & 1][w].y);
-      p.seg_stats[u] = make_float2(m, s);
-    }
+  SubSlice<T> cur, nxt;
+  int u = warp_global;
+  if (u < n_units) cur.issue(row_base(u), u % p.nsub, p.vocab, lane);
+  for (; u < n_units; u += n_warps) {
+    const int un = u + n_warps;
+    if (un < n_units) nxt.issue(row_base(un), un % p.nsub, p.vocab, lane);
+    float m, s;
+    slice_stats(cur, m, s);
+    // warp merge: one exponential per lane (rescale to the warp maximum), then a plain sum
+    const float M = warp_max(m);
+    if (M > -INFINITY) s *= fast_exp2(m - M);
+    const float S = warp_sum(s);
+    if (lane == 0) p.seg_stats[u] = make_float2(M, S);
     cur = nxt;
   }
 }
@@ -224,9 +236,9 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p) {
   double S = 0.0;
   if (lane < 2 * k + 1) {
     const int row = lane <= k ? t0 + lane : p.total_q + d0 + (lane - k - 1);
-    const float2 *st = p.seg_stats + (int64_t)row * p.nseg;
-    for (int i = 0; i < p.nseg; ++i) M = fmaxf(M, st[i].x);
-    for (int i = 0; i < p.nseg; ++i) S += (double)(st[i].y * fast_exp2(st[i].x - M));
+    const float2 *st = p.seg_stats + (int64_t)row * p.nsub;
+    for (int i = 0; i < p.nsub; ++i) M = fmaxf(M, st[i].x);
+    for (int i = 0; i < p.nsub; ++i) S += (double)(st[i].y * fast_exp2(st[i].x - M));
   }
   // lane i < k pairs target row i (its own) with draft row i (lane k+1+i)
   const float Md = __shfl_sync(0xffffffffu, M, (k + 1 + lane) & 31);
@@ -299,7 +311,14 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
     __threadfence();  // the other blocks' segment masses are visible from here on
   }
 
-  const float2 *tstats = p.seg_stats + (int64_t)(t0 + n) * p.nseg;
+  const float2 *tstats = p.seg_stats + (int64_t)(t0 + n) * p.nsub;
+  // probability mass of segment i of the target row, from its sub-segment statistics
+  auto target_mass = [&](int i) -> double {
+    double acc = 0.0;
+    for (int j = i * kSubPerSeg; j < min((i + 1) * kSubPerSeg, p.nsub); ++j)
+      acc += (double)(tstats[j].y * fast_exp2(tstats[j].x - nm.x));
+    return acc * (double)nm.y;
+  };
   __shared__ int s_seg;
   __shared__ float s_target;
   __shared__ int s_degenerate;
@@ -317,14 +336,14 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
     const bool use_target = bonus || degenerate;
     if (use_target) {
       R = 0.0;
-      for (int i = 0; i < p.nseg; ++i) R += (double)(tstats[i].y * fast_exp2(tstats[i].x - nm.x)) * (double)nm.y;
+      for (int i = 0; i < p.nseg; ++i) R += target_mass(i);
     }
     const double target = (double)p.u_sample[r] * R;
     double cum = 0.0;
     int seg = -1, last_pos = -1;
     double before = 0.0, last_before = 0.0;
     for (int i = 0; i < p.nseg; ++i) {
-      const double mass = use_target ? (double)(tstats[i].y * fast_exp2(tstats[i].x - nm.x)) * (double)nm.y : (double)resid[i];
+      const double mass = use_target ? target_mass(i) : (double)resid[i];
       if (mass > 0.0) { last_pos = i; last_before = cum; }
       if (cum + mass > target) { seg = i; before = cum; break; }
       cum += mass;

@@ -19,13 +19,14 @@ static thread_local int32_t t_launches = 0;
 static thread_local cudaEvent_t t_ev_start = nullptr, t_ev_stop = nullptr;
 static thread_local long long *t_prof = nullptr;  // profiling builds only
 
-// spx_verify_step runs its two halves concurrently: the sampler is forked onto an internal stream
-// and joined back before the call returns control of the caller's stream.  One stream and two
-// events per (host thread, device), created on first use and kept until the thread exits.
+// spx_verify_step overlaps the short, latency-bound kernels of one half with the bandwidth-bound
+// kernels of the other through an internal stream that is forked from and joined back into the
+// caller's stream.  One stream and four events per (host thread, device), created on first use
+// and kept until the thread exits.
 struct SideStream {
   int device = -1;
   cudaStream_t stream = nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr, plan_done = nullptr, stats_done = nullptr;
 };
 static thread_local SideStream t_side[16];
 
@@ -36,6 +37,8 @@ static SideStream *get_side_stream(int device) {
     if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s.plan_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s.stats_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     s.device = device;
   }
   return &s;
@@ -116,7 +119,7 @@ static AttnWs attn_ws_layout(const spx_attn_args_t *a) {
 
 struct SampleWs {
   size_t seg_stats, seg_resid, req_norm, req_done, total;
-  int32_t nseg;
+  int32_t nseg, nsub;
 };
 
 static spx_status_t check_sample(const spx_sample_args_t *s, bool need_ptrs) {
@@ -138,9 +141,10 @@ static spx_status_t check_sample(const spx_sample_args_t *s, bool need_ptrs) {
 static SampleWs sample_ws_layout(const spx_sample_args_t *s) {
   SampleWs w{};
   w.nseg = (s->vocab + kSegElems - 1) / kSegElems;
+  w.nsub = (s->vocab + kSubElems - 1) / kSubElems;
   const size_t rows = (size_t)s->total_q + (size_t)(s->total_q - s->batch);
   size_t off = 0;
-  w.seg_stats = off; off = align_up(off + sizeof(float2) * rows * w.nseg, 256);
+  w.seg_stats = off; off = align_up(off + sizeof(float2) * rows * w.nsub, 256);
   w.seg_resid = off; off = align_up(off + sizeof(float) * (size_t)s->batch * w.nseg, 256);
   w.req_norm = off; off = align_up(off + sizeof(float4) * (size_t)s->batch, 256);
   w.req_done = off; off = align_up(off + sizeof(int32_t) * (size_t)s->batch, 256);
@@ -229,8 +233,24 @@ static cudaError_t launch_tc(const CUtensorMap &kmap, const CUtensorMap &vmap, c
 // ---------------------------------------------------------------------------------------------
 // launches
 // ---------------------------------------------------------------------------------------------
+// Launch with programmatic stream serialization: the grid may be scheduled while the previous
+// kernel of the stream drains; the kernel waits (griddepcontrol.wait) before it touches anything
+// the previous kernel wrote.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+enum { kPhasePlan = 1, kPhaseMain = 2, kPhaseStats = 1, kPhaseTail = 2, kPhaseAll = 3 };
+
 static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws, int32_t *dev_status,
-                                     cudaStream_t stream, const DeviceInfo &dev) {
+                                     cudaStream_t stream, const DeviceInfo &dev, int phases = kPhaseAll) {
   if (a->batch == 0) return SPX_OK;
   const AttnWs w = attn_ws_layout(a);
   AttnParams p{};
@@ -261,8 +281,12 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
 
   // the plan never targets more chunks than the workspace was sized for
   const int sms = dev.num_sms < kPlanSmCount ? dev.num_sms : kPlanSmCount;
-  plan_kernel<<<1, 1024, 0, stream>>>(p, sms * kPlanWaves);
-  ++t_launches;
+  if (phases & kPhasePlan) {
+    plan_kernel<<<1, 1024, 0, stream>>>(p, sms * kPlanWaves);
+    ++t_launches;
+    if (cudaGetLastError() != cudaSuccess) return SPX_ERR_CUDA;
+  }
+  if (!(phases & kPhaseMain)) return SPX_OK;
 
   cudaError_t e;
   if (use_tensor_core_path(a)) {
@@ -300,38 +324,43 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
       e = p.D == 64 ? launch_simt(attn_simt_kernel<__nv_bfloat16, 64>) : launch_simt(attn_simt_kernel<__nv_bfloat16, 128>);
   }
   if (e != cudaSuccess) return SPX_ERR_CUDA;
-  if (a->kv_dtype == SPX_F32)
-    combine_kernel<float><<<p.batch * p.Hkv, 256, 0, stream>>>(p);
-  else
-    combine_kernel<__nv_bfloat16><<<p.batch * p.Hkv, 256, 0, stream>>>(p);
+  const dim3 cgrid(p.batch * p.Hkv, (p.rows_cap * (p.D / 4) + 255) / 256);
+  e = a->kv_dtype == SPX_F32 ? launch_pdl(combine_kernel<float>, cgrid, dim3(256), 0, stream, p)
+                             : launch_pdl(combine_kernel<__nv_bfloat16>, cgrid, dim3(256), 0, stream, p);
   ++t_launches;
-  return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
+  return e == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
 }
 
 template <typename T>
-static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream, int num_sms) {
+static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream, int num_sms, int phases) {
   const int rows = p.total_q + p.total_d;
-  const int n_units = rows * p.nseg;
+  const int n_units = rows * p.nsub;
   int per_sm = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_stats_kernel<T>, kSampThreads, 0) != cudaSuccess) return SPX_ERR_CUDA;
   if (per_sm < 1) per_sm = 1;
   int grid = num_sms * per_sm;
-  if (grid > n_units) grid = n_units;
-  row_stats_kernel<T><<<grid, kSampThreads, 0, stream>>>(p, n_units);
-  accept_kernel<T><<<(p.batch * 32 + 127) / 128, 128, 0, stream>>>(p);
-  resid_select_kernel<T><<<dim3(p.nseg, p.batch), kSampThreads, 0, stream>>>(p);
-  t_launches += 3;
+  const int max_grid = (n_units + kSampThreads / 32 - 1) / (kSampThreads / 32);
+  if (grid > max_grid) grid = max_grid;
+  if (phases & kPhaseStats) {
+    row_stats_kernel<T><<<grid, kSampThreads, 0, stream>>>(p, n_units);
+    ++t_launches;
+  }
+  if (phases & kPhaseTail) {
+    accept_kernel<T><<<(p.batch * 32 + 127) / 128, 128, 0, stream>>>(p);
+    resid_select_kernel<T><<<dim3(p.nseg, p.batch), kSampThreads, 0, stream>>>(p);
+    t_launches += 2;
+  }
   return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
 }
 
 static spx_status_t launch_sampler(const spx_sample_args_t *s, unsigned char *ws, int32_t *dev_status,
-                                   cudaStream_t stream, int num_sms) {
+                                   cudaStream_t stream, int num_sms, int phases = kPhaseAll) {
   if (s->batch == 0) return SPX_OK;
   if (s->batch > 65535) return SPX_ERR_UNSUPPORTED;  // grid.y limit of the residual pass
   const SampleWs w = sample_ws_layout(s);
   SampleParams p{};
-  p.batch = s->batch; p.total_q = s->total_q; p.total_d = s->total_q - s->batch; p.vocab = s->vocab; p.nseg = w.nseg;
-  if ((int64_t)(p.total_q + p.total_d) * p.nseg > 0x7fffffff) return SPX_ERR_UNSUPPORTED;
+  p.batch = s->batch; p.total_q = s->total_q; p.total_d = s->total_q - s->batch; p.vocab = s->vocab; p.nseg = w.nseg; p.nsub = w.nsub;
+  if ((int64_t)(p.total_q + p.total_d) * p.nsub > 0x7fffffff) return SPX_ERR_UNSUPPORTED;
   p.row_stride = s->logits_row_stride;
   p.target = s->target_logits; p.draft = s->draft_logits; p.draft_ids = s->draft_token_ids;
   p.q_indptr = s->q_indptr; p.u_accept = s->u_accept; p.u_sample = s->u_sample;
@@ -341,7 +370,7 @@ static spx_status_t launch_sampler(const spx_sample_args_t *s, unsigned char *ws
   p.req_norm = reinterpret_cast<float4 *>(ws + w.req_norm);
   p.req_done = reinterpret_cast<int32_t *>(ws + w.req_done);
   p.dev_status = dev_status;
-  return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16>(p, stream, num_sms) : launch_sampler_t<float>(p, stream, num_sms);
+  return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16>(p, stream, num_sms, phases) : launch_sampler_t<float>(p, stream, num_sms, phases);
 }
 
 static spx_status_t check_ws(const void *ws, size_t ws_bytes, size_t need, const int32_t *dev_status) {
@@ -409,17 +438,28 @@ spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_
   if (!get_device_info(&dev) || dev.cc_major < 10) return SPX_ERR_CUDA;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   unsigned char *base = static_cast<unsigned char *>(ws);
-  // The halves are independent given their inputs: fork the sampler onto the internal stream so
-  // that its bandwidth-bound pass and its short latency-bound kernels overlap the attention kernels.
+  // The halves are independent given their inputs.  The two bandwidth-bound kernels (logits
+  // statistics, then attention) run back to back on the caller's stream, each with the memory
+  // system to itself; the short kernels run beside them on the internal stream: the attention
+  // plan beside the statistics pass, the accept/resample kernels beside the attention kernel.
   SideStream *side = get_side_stream(dev.device);
   if (!side) return SPX_ERR_CUDA;
-  if (cudaEventRecord(side->fork, stream) != cudaSuccess) return SPX_ERR_CUDA;
-  if (cudaStreamWaitEvent(side->stream, side->fork, 0) != cudaSuccess) return SPX_ERR_CUDA;
-  st = launch_sampler(sample, base + attn_bytes, dev_status, side->stream, dev.num_sms);
-  const bool joined = cudaEventRecord(side->join, side->stream) == cudaSuccess;
-  spx_status_t st2 = launch_attention(attn, base, dev_status, stream, dev);
-  if (!joined || cudaStreamWaitEvent(stream, side->join, 0) != cudaSuccess) return SPX_ERR_CUDA;
-  return st != SPX_OK ? st : st2;
+  unsigned char *sws = base + attn_bytes;
+  bool ok = cudaEventRecord(side->fork, stream) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(side->stream, side->fork, 0) == cudaSuccess;
+  if (!ok) return SPX_ERR_CUDA;
+  const spx_status_t s1 = launch_attention(attn, base, dev_status, side->stream, dev, kPhasePlan);
+  ok = ok && cudaEventRecord(side->plan_done, side->stream) == cudaSuccess;
+  const spx_status_t s2 = launch_sampler(sample, sws, dev_status, stream, dev.num_sms, kPhaseStats);
+  ok = ok && cudaEventRecord(side->stats_done, stream) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(side->stream, side->stats_done, 0) == cudaSuccess;
+  const spx_status_t s3 = launch_sampler(sample, sws, dev_status, side->stream, dev.num_sms, kPhaseTail);
+  ok = ok && cudaEventRecord(side->join, side->stream) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(stream, side->plan_done, 0) == cudaSuccess;
+  const spx_status_t s4 = launch_attention(attn, base, dev_status, stream, dev, kPhaseMain);
+  ok = ok && cudaStreamWaitEvent(stream, side->join, 0) == cudaSuccess;
+  if (!ok) return SPX_ERR_CUDA;
+  return s1 != SPX_OK ? s1 : s2 != SPX_OK ? s2 : s3 != SPX_OK ? s3 : s4;
 }
 
 // ---- host-buffer convenience ---------------------------------------------------------------
