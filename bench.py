@@ -106,6 +106,20 @@ class ClockSampler:
         }
 
 
+def reduce_over_ranks(ms: float, tokens: float, device) -> tuple:
+    """Whole-job figures from per-rank ones: the slowest rank's time, the sum of the tokens.
+
+    Each rank runs an independent replica, so this is the only communication of the benchmark.
+    """
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    n = torch.tensor([tokens], dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(n.item())
+
+
 def sub_batch(b_cpu: W.VerifyBatch, n_req: int) -> W.VerifyBatch:
     """The first n_req requests of a host batch (KV pools shared, not copied)."""
     import dataclasses
@@ -259,13 +273,8 @@ def main():
     torch.cuda.synchronize()
     spx.set_timing_events(None, None)
     attn_ms = [e0.elapsed_time(e1) for e0, e1 in k_events]
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    toks = torch.tensor([tokens_per_step], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
-    ms_total = float(t.item())
-    value = float(toks.item()) * args.steps / (ms_total * 1e-3)
+    ms_total, job_tokens = reduce_over_ranks(ms_total, tokens_per_step, dev)
+    value = job_tokens * args.steps / (ms_total * 1e-3)
     ms_per_step = ms_total / args.steps
 
     # ---- end to end through the host-buffer entry point (every rank, max time) ----
@@ -297,13 +306,11 @@ def main():
             spx.verify_step_host(ah, sh, pool_elems, arena, st_h, dev)
         e1.record()
         torch.cuda.synchronize()
-        te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        te_ms, _ = reduce_over_ranks(e0.elapsed_time(e1), 0.0, dev)
         assert int(st_h.item()) == 0 and torch.equal(acc_h, acc.cpu()) and torch.equal(tok_h, tok.cpu())
         h2d = sum(pin[n].numel() * pin[n].element_size() for n in W.VerifyBatch._TENSORS)
         d2h = out_h.numel() * out_h.element_size() + acc_h.numel() * 4 + tok_h.numel() * 4 + 4
-        e2e = {"value": float(toks.item()) * args.e2e_steps / (float(te.item()) * 1e-3), "unit": UNIT,
+        e2e = {"value": job_tokens * args.e2e_steps / (te_ms * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
         del arena, pin
     except Exception as exc:  # reported, never hidden
