@@ -172,6 +172,33 @@ spx_status_t spx_verify_step_host(const spx_attn_args_t *attn, const spx_sample_
                                   int64_t kv_pool_elems, void *dev_arena, size_t arena_bytes,
                                   int32_t *dev_status_host, void *cuda_stream);
 
+/*
+ * spx_rejection_sample for callers that cannot provide scratch memory.  (The paper has no
+ * counterpart: this entry point exists for integration reasons only.)
+ *
+ * Some callers can neither call cudaMalloc nor hand the library a workspace: code running inside a
+ * CUDA-graph capture or a stream-ordered region where an allocation would synchronise or be
+ * refused, runtimes whose allocator owns all device memory and offers no hook, and plugins that
+ * receive only their input and output tensors.  For them the sampling half is offered with its
+ * scratch in a fixed array that is part of the library image: SPX_STATIC_SCRATCH_BYTES of device
+ * memory, held by every GPU that loads the library until the process exits.
+ *
+ * Same arguments, outputs and arithmetic as spx_rejection_sample (bit-identical results); the
+ * caller still passes every input and output buffer and the status word.  Differences:
+ *   - If spx_workspace_size(NULL, args) exceeds SPX_STATIC_SCRATCH_BYTES the call returns
+ *     SPX_ERR_WORKSPACE and launches nothing (e.g. 704 logits rows of 128256 tokens need 0.4 MB;
+ *     the limit is reached near 8000 such rows).
+ *   - The first call on each device looks up the array's device address (no allocation).  Make
+ *     that first call outside any stream capture.
+ *   - Every call on a device shares the one array, which keeps the previous call's contents.
+ *     Nothing in it has to start at zero from the caller's point of view: the only counters are
+ *     cleared by the call itself before they are read.  Two calls that overlap on the same device
+ *     (different streams, or different host threads) race on it: serialise them.
+ *   - It calls no cudaMalloc, cudaFree or any other allocating routine.
+ */
+#define SPX_STATIC_SCRATCH_BYTES (4u << 20)
+spx_status_t spx_rejection_sample_static(const spx_sample_args_t *args, int32_t *dev_status, void *cuda_stream);
+
 const char *spx_status_string(spx_status_t status);
 
 /*

@@ -16,7 +16,7 @@ BF16, F32 = 0, 1
 
 EXPORTS = ("spx_workspace_size", "spx_verify_attention", "spx_rejection_sample", "spx_verify_step",
            "spx_host_step_arena_size", "spx_verify_step_host", "spx_status_string", "spx_last_launch_count",
-           "spx_set_timing_events")
+           "spx_set_timing_events", "spx_rejection_sample_static")
 
 
 class AttnArgs(C.Structure):
@@ -80,6 +80,8 @@ def load_library():
         lib.spx_status_string.restype = C.c_char_p
         lib.spx_status_string.argtypes = [C.c_int]
         lib.spx_last_launch_count.restype = C.c_int32
+        lib.spx_rejection_sample_static.restype = C.c_int
+        lib.spx_rejection_sample_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         lib.spx_set_timing_events.restype = None
         lib.spx_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
         _lib = lib
@@ -255,3 +257,30 @@ def set_timing_events(start: Optional[torch.cuda.Event], stop: Optional[torch.cu
         lib.spx_set_timing_events(None, None)
     else:
         lib.spx_set_timing_events(start.cuda_event, stop.cuda_event)
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def rejection_sample_static(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, vocab=None,
+                            status: Optional[torch.Tensor] = None):
+    """spx_rejection_sample_static on the current stream: the sampling half for callers that can
+    neither allocate nor pass a workspace (the scratch is a fixed array inside the library).
+
+    Only the outputs and, if none is given, the status word are allocated here, by torch, on the
+    caller's side of the boundary; the library call itself allocates nothing.  Returns
+    (accepted_len, out_tokens, status).  Raises SpxError(ERR_WORKSPACE) when the batch needs more
+    than STATIC_SCRATCH_BYTES of scratch.
+    """
+    _require_cuda(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample)
+    lib = load_library()
+    dev = target_logits.device
+    B = q_indptr.numel() - 1
+    accepted = torch.empty(B, dtype=torch.int32, device=dev)
+    tokens = torch.empty(target_logits.shape[0], dtype=torch.int32, device=dev)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    s = make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, accepted, tokens,
+                         None, vocab)
+    _check(lib.spx_rejection_sample_static(C.byref(s), status.data_ptr(), _stream(dev)))
+    return accepted, tokens, status

@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <mutex>
 
 #include "attn_simt.cuh"
 #include "attn_tc.cuh"
@@ -536,6 +537,41 @@ spx_status_t spx_verify_step_host(const spx_attn_args_t *attn, const spx_sample_
   d2h(attn->out, L.out, L.out_bytes); d2h(attn->lse, L.lse, L.lse_bytes);
   d2h(sample->accepted_len, L.acc, B * 4); d2h(sample->out_tokens, L.tok, TQ * 4); d2h(dev_status_host, L.status, 4);
   return ok ? SPX_OK : SPX_ERR_CUDA;
+}
+
+// ---- sampling without caller-provided scratch ------------------------------------------------
+// The scratch of the sampling kernels in a fixed device array that is part of the library image.
+// In host code `g_static_scratch` is only a handle for the symbol, never an address a kernel could
+// use: the device address is looked up once per device with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_static_scratch[SPX_STATIC_SCRATCH_BYTES];
+
+namespace {
+std::mutex g_static_scratch_mutex;
+void *g_static_scratch_addr[64] = {};  // device address of g_static_scratch, per device ordinal
+}  // namespace
+
+spx_status_t spx_rejection_sample_static(const spx_sample_args_t *args, int32_t *dev_status, void *cuda_stream) {
+  t_launches = 0;
+  spx_status_t st = check_sample(args, true);
+  if (st != SPX_OK) return st;
+  if (!dev_status) return SPX_ERR_INVALID_ARG;
+  if (sample_ws_layout(args).total > SPX_STATIC_SCRATCH_BYTES) return SPX_ERR_WORKSPACE;  // beyond the fixed array
+  DeviceInfo dev;
+  if (!get_device_info(&dev) || dev.cc_major < 10) return SPX_ERR_CUDA;
+  if (dev.device < 0 || dev.device >= 64) return SPX_ERR_UNSUPPORTED;
+  void *scratch = nullptr;
+  {
+    // set-up, once per device, with that device current (it is: dev.device is the current device)
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (!g_static_scratch_addr[dev.device]) {
+      void *addr = nullptr;
+      if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) return SPX_ERR_CUDA;
+      g_static_scratch_addr[dev.device] = addr;
+    }
+    scratch = g_static_scratch_addr[dev.device];
+  }
+  return launch_sampler(args, static_cast<unsigned char *>(scratch), dev_status, static_cast<cudaStream_t>(cuda_stream),
+                        dev.num_sms);
 }
 
 const char *spx_status_string(spx_status_t status) {
