@@ -7,7 +7,8 @@
 //     [32q, 32q+32) of every query row into lane quadrant q;
 //   * the softmax warp of quadrant q owns those 32 tokens.  The four warps agree on the row
 //     maximum of the tile through shared memory (one bounded barrier per tile), so that all of
-//     them use the same reference maximum, and write P as bf16 into a swizzled shared-memory tile;
+//     them use the same reference maximum, and write P as bf16 into a swizzled shared-memory tile
+//     (one tile: it is rewritten as soon as the previous value MMA has consumed it);
 //   * O += P V is again a weight-stationary M = 32 MMA (P from shared memory, V MN-major), so O
 //     comes out column-split the same way: quadrant q holds columns [q*D/4, (q+1)*D/4) of every
 //     row, complete, and the epilogue is one tensor-memory load and one store per thread.
@@ -28,10 +29,12 @@ struct Tc4Cfg {
   static constexpr int kPBytes = 2 * 32 * 128;   // one P tile: 32 rows x 128 tokens bf16, two 64-token halves
   static constexpr int kBarBytes = 2304;         // barriers (256) + row maxima (1024) + row sums (1024)
   static constexpr int kSlack = 512;             // room to round the dynamic shared base up to 1024 bytes
-  static constexpr int kBudget = 232448 - kSlack - kBarBytes - 2 * kQBytes - 2 * kPBytes;
+  // 8 KB are left unused on purpose: with them (and the 1 KB the hardware reserves per block) the
+  // short sampling kernels, which need about 2 KB of shared memory, can share an SM with this CTA
+  static constexpr int kBudget = 232448 - 8192 - kSlack - kBarBytes - 2 * kQBytes - kPBytes;
   static constexpr int kStagesRaw = kBudget / (2 * kTileBytes);
   static constexpr int kStages = kStagesRaw > 4 ? 4 : kStagesRaw;
-  static constexpr int kSmemBytes = kSlack + 2 * kQBytes + kStages * 2 * kTileBytes + 2 * kPBytes + kBarBytes;
+  static constexpr int kSmemBytes = kSlack + 2 * kQBytes + kStages * 2 * kTileBytes + kPBytes + kBarBytes;
   static constexpr int kTmemCols = 128;          // two score buffers (64) + two O buffers (2 * D/4)
   static constexpr int kColS0 = 0, kColS1 = 32, kColO = 64;
   static constexpr int kColBlock = D / 4;        // output columns held by one quadrant
@@ -78,8 +81,8 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   unsigned char *sQ = smem;
   unsigned char *sK = smem + 2 * Cfg::kQBytes;
   unsigned char *sV = sK + Cfg::kStages * Cfg::kTileBytes;
-  unsigned char *sP = sV + Cfg::kStages * Cfg::kTileBytes;  // two P tiles
-  TcBarriers *bars = reinterpret_cast<TcBarriers *>(sP + 2 * Cfg::kPBytes);
+  unsigned char *sP = sV + Cfg::kStages * Cfg::kTileBytes;  // one P tile
+  TcBarriers *bars = reinterpret_cast<TcBarriers *>(sP + Cfg::kPBytes);
   float *sMx = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(bars) + 256);  // [2 tiles][4 quadrants][32 rows]
   float *sL = sMx + 2 * 4 * 32;                                                          // [2 items][4 quadrants][32 rows]
 
@@ -282,7 +285,7 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
         if (!ok) break;
         fence_after();
         const uint32_t va = smem_u32(sV + slot * Cfg::kTileBytes);
-        const uint32_t pa = smem_u32(sP + (t & 1) * Cfg::kPBytes);
+        const uint32_t pa = smem_u32(sP);
 #pragma unroll
         for (int k = 0; k < kTileTokens / 16; ++k)
           mma_ws_ss(tmem + Cfg::kColO + (pv.qc & 1) * Cfg::kColBlock, smem_desc(pa + (k / 4) * 4096 + (k % 4) * 32, 16, 1024),
@@ -487,9 +490,14 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
           pk[i] = pack_bf16(p0, p1);
         }
         l_sum += sum;
+        // the single P tile is free once the previous tile's value MMA has read it
+        if (tc_ > 0) {
+          ok = warp_wait(&bars->pv_done[(tc_ - 1) & 1], ((tc_ - 1) >> 1) & 1, 3);
+          if (!ok) break;
+        }
         {
           // P tile in shared memory: K-major, 128-byte swizzle, tokens [64h, 64h+64) in half h
-          unsigned char *pr = sP + b * Cfg::kPBytes + (quad >> 1) * 4096 + (row >> 3) * 1024 + (row & 7) * 128;
+          unsigned char *pr = sP + (quad >> 1) * 4096 + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
           for (int jj = 0; jj < 4; ++jj) {
             const int c = (quad & 1) * 4 + jj;

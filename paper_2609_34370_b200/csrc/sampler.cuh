@@ -15,7 +15,10 @@
 namespace spx {
 
 constexpr int kSegElems = 8192;       // tokens per segment (residual pass, final draw)
-constexpr int kSubElems = 2048;       // tokens per sub-segment (statistics pass)
+#ifndef SPX_SUB_ELEMS
+#define SPX_SUB_ELEMS 2048
+#endif
+constexpr int kSubElems = SPX_SUB_ELEMS;  // tokens per sub-segment (statistics pass)
 constexpr int kSubPerSeg = kSegElems / kSubElems;
 constexpr int kSampThreads = 256;
 constexpr int kElemsPerThread = kSegElems / kSampThreads;  // 32

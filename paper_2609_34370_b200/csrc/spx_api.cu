@@ -19,6 +19,9 @@ namespace spx {
 static thread_local int32_t t_launches = 0;
 static thread_local cudaEvent_t t_ev_start = nullptr, t_ev_stop = nullptr;
 static thread_local long long *t_prof = nullptr;  // profiling builds only
+#if SPX_PROFILE
+static thread_local cudaEvent_t *g_step_marks = nullptr;
+#endif
 
 // spx_verify_step overlaps the short, latency-bound kernels of one half with the bandwidth-bound
 // kernels of the other through an internal stream that is forked from and joined back into the
@@ -446,19 +449,32 @@ spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_
   SideStream *side = get_side_stream(dev.device);
   if (!side) return SPX_ERR_CUDA;
   unsigned char *sws = base + attn_bytes;
+#if SPX_PROFILE
+  static thread_local cudaEvent_t tl[6] = {};
+  if (!tl[0]) for (auto &e : tl) cudaEventCreate(&e);
+  auto mark = [&](int i) { cudaEventRecord(tl[i], stream); };
+  g_step_marks = tl;
+#else
+  auto mark = [&](int) {};
+#endif
+  mark(0);
   bool ok = cudaEventRecord(side->fork, stream) == cudaSuccess;
   ok = ok && cudaStreamWaitEvent(side->stream, side->fork, 0) == cudaSuccess;
   if (!ok) return SPX_ERR_CUDA;
   const spx_status_t s1 = launch_attention(attn, base, dev_status, side->stream, dev, kPhasePlan);
   ok = ok && cudaEventRecord(side->plan_done, side->stream) == cudaSuccess;
   const spx_status_t s2 = launch_sampler(sample, sws, dev_status, stream, dev.num_sms, kPhaseStats);
+  mark(1);
   ok = ok && cudaEventRecord(side->stats_done, stream) == cudaSuccess;
   ok = ok && cudaStreamWaitEvent(side->stream, side->stats_done, 0) == cudaSuccess;
   const spx_status_t s3 = launch_sampler(sample, sws, dev_status, side->stream, dev.num_sms, kPhaseTail);
   ok = ok && cudaEventRecord(side->join, side->stream) == cudaSuccess;
   ok = ok && cudaStreamWaitEvent(stream, side->plan_done, 0) == cudaSuccess;
+  mark(2);
   const spx_status_t s4 = launch_attention(attn, base, dev_status, stream, dev, kPhaseMain);
+  mark(3);
   ok = ok && cudaStreamWaitEvent(stream, side->join, 0) == cudaSuccess;
+  mark(4);
   if (!ok) return SPX_ERR_CUDA;
   return s1 != SPX_OK ? s1 : s2 != SPX_OK ? s2 : s3 != SPX_OK ? s3 : s4;
 }
@@ -595,6 +611,10 @@ int32_t spx_last_launch_count(void) { return t_launches; }
 #if SPX_PROFILE
 // Profiling builds only (not declared in spx.h): per-CTA cycle counters of the attention kernel.
 void spx_debug_set_profile_buffer(long long *device_buffer) { t_prof = device_buffer; }
+// milliseconds between the step's marks 0..4 of the last spx_verify_step on this thread
+void spx_debug_step_marks(float *out4) {
+  for (int i = 0; i < 4; ++i) { out4[i] = 0.f; if (g_step_marks) cudaEventElapsedTime(&out4[i], g_step_marks[i], g_step_marks[i + 1]); }
+}
 #endif
 
 }  // extern "C"
