@@ -1,17 +1,18 @@
-// Verify attention for at most 32 packed query rows per kv-head: column-split softmax.
+// Verify attention for at most 64 packed query rows per kv-head: column-split softmax.
 //
-// With G*(k+1) <= 32 a 128-lane tensor-memory tile would leave three of the four lane quadrants
-// (and with them three of the SM's four sub-partitions, each with its own issue slot and
-// exponential unit) idle.  This kernel splits every 128-token tile by columns instead:
-//   * S = Q K^T is a weight-stationary MMA with M = 32, whose accumulator layout puts tokens
-//     [32q, 32q+32) of every query row into lane quadrant q;
-//   * the softmax warp of quadrant q owns those 32 tokens.  The four warps agree on the row
-//     maximum of the tile through shared memory (one bounded barrier per tile), so that all of
+// With G*(k+1) <= 64 a 128-lane tensor-memory tile would leave half or three quarters of the lane
+// quadrants (and with them the SM's sub-partitions, each with its own issue slot and exponential
+// unit) idle.  This kernel splits every 128-token tile by columns instead (MROWS = 32: four
+// blocks of 32 tokens; MROWS = 64: two blocks of 64 tokens for each of two row groups):
+//   * S = Q K^T is a weight-stationary MMA with M = MROWS, whose accumulator layout spreads the
+//     tokens of every query row over the lane quadrants;
+//   * each softmax warp owns one (row group, token block).  The warps that share a row agree on the
+//     row maximum of the tile through shared memory (one bounded barrier per tile), so that all of
 //     them use the same reference maximum, and write P as bf16 into a swizzled shared-memory tile
 //     (one tile: it is rewritten as soon as the previous value MMA has consumed it);
-//   * O += P V is again a weight-stationary M = 32 MMA (P from shared memory, V MN-major), so O
-//     comes out column-split the same way: quadrant q holds columns [q*D/4, (q+1)*D/4) of every
-//     row, complete, and the epilogue is one tensor-memory load and one store per thread.
+//   * O += P V is again a weight-stationary M = MROWS MMA (P from shared memory, V MN-major), so O
+//     comes out column-split the same way: each thread holds D/4 (or D/2) columns of one row,
+//     complete, and the epilogue is one tensor-memory load and one store per thread.
 // Producer, stage ring, work plan, bounded waits and partial/direct output are those of
 // attn_tc_kernel.
 #pragma once
@@ -19,25 +20,32 @@
 
 namespace spx {
 
-template <int D>
+template <int D, int MROWS>
 struct Tc4Cfg {
+  static_assert(MROWS == 32 || MROWS == 64, "MROWS is 32 or 64");
+  static constexpr int kSplit = 128 / MROWS;               // token blocks per tile: 4 or 2
+  static constexpr int kTokPerThread = kTileTokens / kSplit;  // 32 or 64 score columns per thread
   static constexpr int kHalves = D / 64;
   static constexpr int kHalfBytes = kTileTokens * 128;
   static constexpr int kTileBytes = kHalves * kHalfBytes;
-  static constexpr int kQHalfBytes = 32 * 128;
+  static constexpr int kQHalfBytes = MROWS * 128;
   static constexpr int kQBytes = kHalves * kQHalfBytes;
-  static constexpr int kPBytes = 2 * 32 * 128;   // one P tile: 32 rows x 128 tokens bf16, two 64-token halves
+  static constexpr int kQBufs = MROWS == 32 ? 2 : 1;       // the 64-row tile leaves room for one Q buffer only
+  static constexpr int kPHalfBytes = MROWS * 128;          // P tile: MROWS rows x 128 tokens bf16, two 64-token halves
+  static constexpr int kPBytes = 2 * kPHalfBytes;
   static constexpr int kBarBytes = 2304;         // barriers (256) + row maxima (1024) + row sums (1024)
   static constexpr int kSlack = 512;             // room to round the dynamic shared base up to 1024 bytes
-  // 8 KB are left unused on purpose: with them (and the 1 KB the hardware reserves per block) the
-  // short sampling kernels, which need about 2 KB of shared memory, can share an SM with this CTA
-  static constexpr int kBudget = 232448 - 8192 - kSlack - kBarBytes - 2 * kQBytes - kPBytes;
+  // With 32 rows 8 KB are left unused on purpose: with them (and the 1 KB the hardware reserves
+  // per block) the short sampling kernels, which need about 2 KB of shared memory, can share an SM
+  // with this CTA.
+  static constexpr int kFree = MROWS == 32 ? 8192 : 0;
+  static constexpr int kBudget = 232448 - kFree - kSlack - kBarBytes - kQBufs * kQBytes - kPBytes;
   static constexpr int kStagesRaw = kBudget / (2 * kTileBytes);
   static constexpr int kStages = kStagesRaw > 4 ? 4 : kStagesRaw;
-  static constexpr int kSmemBytes = kSlack + 2 * kQBytes + kStages * 2 * kTileBytes + kPBytes + kBarBytes;
-  static constexpr int kTmemCols = 128;          // two score buffers (64) + two O buffers (2 * D/4)
-  static constexpr int kColS0 = 0, kColS1 = 32, kColO = 64;
-  static constexpr int kColBlock = D / 4;        // output columns held by one quadrant
+  static constexpr int kSmemBytes = kSlack + kQBufs * kQBytes + kStages * 2 * kTileBytes + kPBytes + kBarBytes;
+  static constexpr int kColBlock = D / kSplit;   // output columns held by one thread
+  static constexpr int kColS0 = 0, kColS1 = kTokPerThread, kColO = 2 * kTokPerThread;  // + two O buffers of kColBlock
+  static constexpr int kTmemCols = (2 * kTokPerThread + 2 * kColBlock) <= 128 ? 128 : 256;
   static_assert(kStages >= 2, "need at least two stages");
 };
 
@@ -55,23 +63,38 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 template <int N>
 __device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t (&r)[N]) {
-  if constexpr (N == 32) tmem_ld32(taddr, r); else tmem_ld16(taddr, r);
+  if constexpr (N == 64) {
+    tmem_ld32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+    tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+  } else if constexpr (N == 32) {
+    tmem_ld32(taddr, r);
+  } else {
+    tmem_ld16(taddr, r);
+  }
 }
 template <int N>
 __device__ __forceinline__ void tmem_st(uint32_t taddr, const uint32_t (&r)[N]) {
-  if constexpr (N == 32) tmem_st32(taddr, r); else tmem_st16(taddr, r);
+  if constexpr (N == 64) {
+    tmem_st32(taddr, *reinterpret_cast<const uint32_t(*)[32]>(&r[0]));
+    tmem_st32(taddr + 32, *reinterpret_cast<const uint32_t(*)[32]>(&r[32]));
+  } else if constexpr (N == 32) {
+    tmem_st32(taddr, r);
+  } else {
+    tmem_st16(taddr, r);
+  }
 }
-// weight-stationary instruction descriptor: D fp32, A/B bf16 K-major, M = 32
-__host__ __device__ constexpr uint32_t idesc_ws32(uint32_t n, bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((n >> 3) << 17) | ((32u >> 4) << 24);
+// weight-stationary instruction descriptor: D fp32, A/B bf16, A K-major, M = 32 or 64
+__host__ __device__ constexpr uint32_t idesc_ws(uint32_t m, uint32_t n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((n >> 3) << 17) | ((m >> 4) << 24);
 }
 }  // namespace tc
 
-template <int D>
+template <int D, int MROWS>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, AttnParams p) {
-  using Cfg = Tc4Cfg<D>;
+  using Cfg = Tc4Cfg<D, MROWS>;
   using namespace tc;
+  constexpr int kSplit = Cfg::kSplit, TPT = Cfg::kTokPerThread;
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   if (smem - smem_dyn > Cfg::kSlack) {  // cannot happen with the declared alignment; never run past the allocation
@@ -79,12 +102,12 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
     return;
   }
   unsigned char *sQ = smem;
-  unsigned char *sK = smem + 2 * Cfg::kQBytes;
+  unsigned char *sK = smem + Cfg::kQBufs * Cfg::kQBytes;
   unsigned char *sV = sK + Cfg::kStages * Cfg::kTileBytes;
   unsigned char *sP = sV + Cfg::kStages * Cfg::kTileBytes;  // one P tile
   TcBarriers *bars = reinterpret_cast<TcBarriers *>(sP + Cfg::kPBytes);
-  float *sMx = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(bars) + 256);  // [2 tiles][4 quadrants][32 rows]
-  float *sL = sMx + 2 * 4 * 32;                                                          // [2 items][4 quadrants][32 rows]
+  float *sMx = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(bars) + 256);  // [2 tiles][kSplit][MROWS]
+  float *sL = sMx + 2 * 128;                                                             // [2 items][kSplit][MROWS]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   long long prof_g0 = 0;
@@ -226,8 +249,8 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t kIdescQK = idesc_ws32(kTileTokens, false);
-      constexpr uint32_t kIdescPV = idesc_ws32(D, true);
+      constexpr uint32_t kIdescQK = idesc_ws(MROWS, kTileTokens, false);
+      constexpr uint32_t kIdescPV = idesc_ws(MROWS, D, true);
       // Two cursors over the CTA's flat tile sequence: the score MMA runs one tile ahead of the
       // value MMA, across work-item boundaries too.
       struct Cursor { int it, n_tiles, n_tiles_next, i; uint32_t qc, t; bool valid; };
@@ -253,8 +276,8 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
       open_item(pv);
       bool ok = true;
       auto issue_qk = [&]() -> bool {
-        const uint32_t t = qk.t, qb = qk.qc & 1;
-        if (qk.i == 0 && !lane_wait(&bars->q_full[qb], (qk.qc >> 1) & 1, 3)) return false;
+        const uint32_t t = qk.t, qb = Cfg::kQBufs == 2 ? (qk.qc & 1) : 0;
+        if (qk.i == 0 && !lane_wait(&bars->q_full[qb], (Cfg::kQBufs == 2 ? (qk.qc >> 1) : qk.qc) & 1, 3)) return false;
         const int slot = t % Cfg::kStages;
         if (!lane_wait(&bars->k_full[slot], (t / Cfg::kStages) & 1, 0)) return false;
         fence_after();
@@ -288,7 +311,7 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
         const uint32_t pa = smem_u32(sP);
 #pragma unroll
         for (int k = 0; k < kTileTokens / 16; ++k)
-          mma_ws_ss(tmem + Cfg::kColO + (pv.qc & 1) * Cfg::kColBlock, smem_desc(pa + (k / 4) * 4096 + (k % 4) * 32, 16, 1024),
+          mma_ws_ss(tmem + Cfg::kColO + (pv.qc & 1) * Cfg::kColBlock, smem_desc(pa + (k / 4) * Cfg::kPHalfBytes + (k % 4) * 32, 16, 1024),
                     smem_desc(va + k * 2 * 1024, Cfg::kHalfBytes, 1024), kIdescPV, (pv.i > 0) || (k > 0));
         mma_commit(&bars->v_empty[slot]);
         mma_commit(&bars->pv_done[t & 1]);
@@ -298,7 +321,11 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   } else {
     // ------------------------------------------------------------------ softmax / epilogue
     const int quad = warp & 3;
-    const int row = lane;                                   // packed query row
+    // the accumulator layouts of the M = 32 / M = 64 weight-stationary MMAs: quadrant -> (row group,
+    // token block); the same split applies to the columns of O
+    const int rgrp = kSplit == 4 ? 0 : (quad & 1);
+    const int tblk = kSplit == 4 ? quad : (quad >> 1);
+    const int row = rgrp * 32 + lane;                       // packed query row
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const int sm_tid = tid - 64;
     const __nv_bfloat16 *Qg = reinterpret_cast<const __nv_bfloat16 *>(p.q);
@@ -309,7 +336,7 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
     // Q rows of an item -> shared memory (K-major, 128-byte swizzle), in two halves so that the
     // global loads can be issued early and stored later: each thread owns up to kQPerThread
     // 16-byte chunks of the 32 x D tile.
-    constexpr int kQPerThread = (32 * kChunksPerRow + 127) / 128;
+    constexpr int kQPerThread = (MROWS * kChunksPerRow + 127) / 128;
     uint4 qreg[kQPerThread];
     auto q_load = [&](const ItemInfo &J) {
 #pragma unroll
@@ -355,7 +382,9 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
       const long long pe0 = kProfile ? clock64() : 0;
       const ItemInfo &J = pend.I;
       const float *sl = sL + (pend.qc & 1) * 128;
-      const float l_row = sl[row] + sl[32 + row] + sl[64 + row] + sl[96 + row];
+      float l_row = 0.f;
+#pragma unroll
+      for (int tb = 0; tb < kSplit; ++tb) l_row += sl[tb * MROWS + row];
       if (!warp_wait(&bars->pv_done[pend.last_tc & 1], (pend.last_tc >> 1) & 1, 1)) return false;
       fence_after();
       uint32_t o[CB];
@@ -369,7 +398,7 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
       if (row < J.R) {
         if (J.part_slot < 0) {
           const float inv = 1.f / l_row;
-          __nv_bfloat16 *dst = out + ((int64_t)(J.q0 + j) * p.Hq + J.g * p.G + hg) * D + quad * CB;
+          __nv_bfloat16 *dst = out + ((int64_t)(J.q0 + j) * p.Hq + J.g * p.G + hg) * D + tblk * CB;
 #pragma unroll
           for (int v = 0; v < CB / 8; ++v) {
             uint4 u;
@@ -379,14 +408,14 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
             u.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
             *reinterpret_cast<uint4 *>(dst + v * 8) = u;
           }
-          if (quad == 0 && p.lse) p.lse[(int64_t)(J.q0 + j) * p.Hq + J.g * p.G + hg] = (pend.m_ref + log2f(l_row)) * kLn2;
+          if (tblk == 0 && p.lse) p.lse[(int64_t)(J.q0 + j) * p.Hq + J.g * p.G + hg] = (pend.m_ref + log2f(l_row)) * kLn2;
         } else {
           const int64_t slot = ((int64_t)J.part_slot * p.Hkv + J.g) * p.rows_cap + row;
-          float *dst = p.part_o + slot * D + quad * CB;
+          float *dst = p.part_o + slot * D + tblk * CB;
 #pragma unroll
           for (int v = 0; v < CB / 4; ++v)
             *reinterpret_cast<uint4 *>(dst + v * 4) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
-          if (quad == 0) p.part_ml[slot] = make_float2(pend.m_ref, l_row);
+          if (tblk == 0) p.part_ml[slot] = make_float2(pend.m_ref, l_row);
         }
       }
       pend.valid = false;
@@ -408,16 +437,24 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
       WorkEntry e_next;
       if (idx_next >= 0) e_next = entry_of(idx_next);
       int q_stage = idx_next >= 0 ? 0 : 2;  // 0: nothing yet, 1: loads issued, 2: stored / nothing to do
-      auto q_step = [&]() -> bool {
+      // With one Q buffer the store has to wait for this item's last score MMA, which is only
+      // issued once the softmax has reached the last tile: it then happens after the tile loop.
+      auto q_step = [&](bool item_done) -> bool {
         if (q_stage == 0) {
           Inext = make_item(e_next, idx_next);
           q_load(Inext);
           q_stage = 1;
         } else if (q_stage == 1) {
-          const uint32_t nb = (qc + 1) & 1;
-          if (qc >= 1 && !warp_wait(&bars->q_empty[nb], ((qc - 1) >> 1) & 1, 3)) return false;
-          q_store(Inext, nb);
-          q_stage = 2;
+          if (Cfg::kQBufs == 2) {
+            const uint32_t nb = (qc + 1) & 1;
+            if (qc >= 1 && !warp_wait(&bars->q_empty[nb], ((qc - 1) >> 1) & 1, 3)) return false;
+            q_store(Inext, nb);
+            q_stage = 2;
+          } else if (item_done) {
+            if (!warp_wait(&bars->q_empty[0], qc & 1, 3)) return false;
+            q_store(Inext, 0);
+            q_stage = 2;
+          }
         }
         return true;
       };
@@ -427,31 +464,32 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
       for (int tile = I.tile_begin; tile < I.tile_end && ok; ++tile, ++tc_) {
         const uint32_t b = tc_ & 1;
         const uint32_t ts = tmem + (b ? Cfg::kColS1 : Cfg::kColS0) + lane_addr;
-        const int t0 = tile * kTileTokens + quad * 32;  // first token of this quadrant's block
+        const int t0 = tile * kTileTokens + tblk * TPT;  // first token of this thread's block
         const bool mask_tile = tile * kTileTokens + kTileTokens - 1 > I.L - I.m;
         ok = warp_wait(&bars->s_full[b], (tc_ >> 1) & 1, 0);
         if (!ok) break;
         fence_after();
-        uint32_t r[32];
-        tmem_ld32(ts, r);
+        uint32_t r[TPT];
+        tmem_ld<TPT>(ts, r);
         wait_ld();
         float mx = -INFINITY;
         if (mask_tile) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
+          for (int i = 0; i < TPT; ++i) {
             r[i] = (t0 + i <= limit) ? r[i] : 0xff800000u;  // -inf
             mx = fmaxf(mx, __uint_as_float(r[i]));
           }
         } else {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+          for (int i = 0; i < TPT; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
         }
         // agree on the row maximum of the whole tile
-        sMx[(b * 4 + quad) * 32 + row] = mx * p.scale_log2;
+        sMx[(b * kSplit + tblk) * MROWS + row] = mx * p.scale_log2;
         ok = softmax_sync();
         if (!ok) break;
-        const float mrow = fmaxf(fmaxf(sMx[(b * 4 + 0) * 32 + row], sMx[(b * 4 + 1) * 32 + row]),
-                                 fmaxf(sMx[(b * 4 + 2) * 32 + row], sMx[(b * 4 + 3) * 32 + row]));
+        float mrow = -INFINITY;
+#pragma unroll
+        for (int tb = 0; tb < kSplit; ++tb) mrow = fmaxf(mrow, sMx[(b * kSplit + tb) * MROWS + row]);
         // lazy rescale: the reference moves only when the maximum grows by more than 2^8; a row
         // that has seen no visible token yet adopts the tile maximum for free (its O is zero)
         float alpha = 1.f;
@@ -481,9 +519,9 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
         }
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
         float sum = 0.f;
-        uint32_t pk[16];
+        uint32_t pk[TPT / 2];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
+        for (int i = 0; i < TPT / 2; ++i) {
           const float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * i]), p.scale_log2, -m_use));
           const float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * i + 1]), p.scale_log2, -m_use));
           sum += p0 + p1;
@@ -497,10 +535,12 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
         }
         {
           // P tile in shared memory: K-major, 128-byte swizzle, tokens [64h, 64h+64) in half h
-          unsigned char *pr = sP + (quad >> 1) * 4096 + (row >> 3) * 1024 + (row & 7) * 128;
+          constexpr int kChunks = TPT / 8;                       // 16-byte chunks this thread writes
+          const int tok0 = tblk * TPT;
+          unsigned char *pr = sP + (tok0 >> 6) * Cfg::kPHalfBytes + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
-          for (int jj = 0; jj < 4; ++jj) {
-            const int c = (quad & 1) * 4 + jj;
+          for (int jj = 0; jj < kChunks; ++jj) {
+            const int c = ((tok0 & 63) >> 3) + jj;
             *reinterpret_cast<uint4 *>(pr + ((c ^ (row & 7)) << 4)) = make_uint4(pk[4 * jj], pk[4 * jj + 1], pk[4 * jj + 2], pk[4 * jj + 3]);
           }
         }
@@ -523,14 +563,14 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->p_full[b]);
         if (pend.valid) ok = run_epilogue();  // previous item (its sL became visible at this tile's barrier)
-        if (ok) ok = q_step();
+        if (ok) ok = q_step(false);
       }
-      while (ok && q_stage < 2) ok = q_step();
+      while (ok && q_stage < 2) ok = q_step(true);
       if (!ok) break;
 
       // ---- the item's epilogue is deferred: it runs after the first tile of the next item, when
       // the last PV has long completed, so the softmax never idles at an item boundary
-      sL[((qc & 1) * 4 + quad) * 32 + row] = l_sum;
+      sL[((qc & 1) * kSplit + tblk) * MROWS + row] = l_sum;
       pend.valid = true; pend.I = I; pend.m_ref = m_ref; pend.last_tc = tc_ - 1; pend.qc = qc;
       const long long prof_e0 = 0, prof_e1 = 0, prof_e2 = 0;
       (void)prof_e0; (void)prof_e1; (void)prof_e2;

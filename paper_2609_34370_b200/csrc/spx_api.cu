@@ -206,11 +206,11 @@ static bool use_tensor_core_path(const spx_attn_args_t *a) {
          a->kv_stride_head > 0;
 }
 
-template <int D>
+template <int D, int MROWS>
 static cudaError_t launch_tc4(const CUtensorMap &kmap, const CUtensorMap &vmap, const AttnParams &p, int num_sms,
                               cudaStream_t stream) {
-  using Cfg = Tc4Cfg<D>;
-  auto kernel = attn_tc4_kernel<D>;
+  using Cfg = Tc4Cfg<D, MROWS>;
+  auto kernel = attn_tc4_kernel<D, MROWS>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
   if (e != cudaSuccess) return e;
   if (t_ev_start) cudaEventRecord(t_ev_start, stream);
@@ -299,7 +299,9 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
     if (!make_pool_map(&kmap, a->k_cache, a, p.head_inner) || !make_pool_map(&vmap, a->v_cache, a, p.head_inner))
       return SPX_ERR_CUDA;
     if (p.rows_cap <= 32)
-      e = p.D == 128 ? launch_tc4<128>(kmap, vmap, p, dev.num_sms, stream) : launch_tc4<64>(kmap, vmap, p, dev.num_sms, stream);
+      e = p.D == 128 ? launch_tc4<128, 32>(kmap, vmap, p, dev.num_sms, stream) : launch_tc4<64, 32>(kmap, vmap, p, dev.num_sms, stream);
+    else if (p.rows_cap <= 64)
+      e = p.D == 128 ? launch_tc4<128, 64>(kmap, vmap, p, dev.num_sms, stream) : launch_tc4<64, 64>(kmap, vmap, p, dev.num_sms, stream);
     else if (p.D == 128)
       e = p.rows_cap <= 64 ? launch_tc<128, 64>(kmap, vmap, p, dev.num_sms, stream)
                            : launch_tc<128, 128>(kmap, vmap, p, dev.num_sms, stream);
