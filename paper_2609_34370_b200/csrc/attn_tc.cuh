@@ -183,6 +183,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
   __syncthreads();
   fence_after();
   const uint32_t tmem = bars->tmem_base;
+  // the plan is read from here on: under programmatic dependent launch, wait for the planner
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   const int n_items = p.hdr->overflow ? 0 : p.hdr->n_work * p.Hkv;
   const int n_cta = gridDim.x;

@@ -131,6 +131,9 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   __syncthreads();
   fence_after();
   const uint32_t tmem = bars->tmem_base;
+  // Everything above touched only this CTA's own resources; the plan is read from here on.  Under
+  // programmatic dependent launch this is where the kernel waits for the planner to finish.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   const int n_items = p.hdr->overflow ? 0 : p.hdr->n_work * p.Hkv;
   const int n_cta = gridDim.x;
