@@ -161,25 +161,46 @@ __global__ void __launch_bounds__(256) combine_kernel(AttnParams p) {
   const int row = item / vecs, dv = item % vecs;
   const int64_t slot0 = ((int64_t)p.req_part_base[r] * p.Hkv + g) * p.rows_cap + row;
   const int64_t slot_step = (int64_t)p.Hkv * p.rows_cap;
-  float mstar = -INFINITY;
-  for (int c = 0; c < nch; ++c) mstar = fmaxf(mstar, p.part_ml[slot0 + c * slot_step].x);
-  float lstar = 0.f;
+  float lstar = 0.f, mstar = -INFINITY;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int c0 = 0; c0 < nch; c0 += 4) {
+  if (nch <= 4) {
+    // the common case: every load of the item is issued at once (one memory round trip)
     float2 ml[4];
     float4 o[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const int c = min(c0 + u, nch - 1);
+      const int c = min(u, nch - 1);
       ml[u] = p.part_ml[slot0 + c * slot_step];
       o[u] = *reinterpret_cast<const float4 *>(p.part_o + (slot0 + c * slot_step) * D + dv * 4);
     }
 #pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (u < nch) mstar = fmaxf(mstar, ml[u].x);
+#pragma unroll
     for (int u = 0; u < 4; ++u) {
-      if (c0 + u >= nch || ml[u].x == -INFINITY) continue;
+      if (u >= nch || ml[u].x == -INFINITY) continue;
       const float w = fast_exp2(ml[u].x - mstar);
       lstar += w * ml[u].y;
       acc.x += w * o[u].x; acc.y += w * o[u].y; acc.z += w * o[u].z; acc.w += w * o[u].w;
+    }
+  } else {
+    for (int c = 0; c < nch; ++c) mstar = fmaxf(mstar, p.part_ml[slot0 + c * slot_step].x);
+    for (int c0 = 0; c0 < nch; c0 += 4) {
+      float2 ml[4];
+      float4 o[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int c = min(c0 + u, nch - 1);
+        ml[u] = p.part_ml[slot0 + c * slot_step];
+        o[u] = *reinterpret_cast<const float4 *>(p.part_o + (slot0 + c * slot_step) * D + dv * 4);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (c0 + u >= nch || ml[u].x == -INFINITY) continue;
+        const float w = fast_exp2(ml[u].x - mstar);
+        lstar += w * ml[u].y;
+        acc.x += w * o[u].x; acc.y += w * o[u].y; acc.z += w * o[u].z; acc.w += w * o[u].w;
+      }
     }
   }
   const float inv = 1.f / lstar;

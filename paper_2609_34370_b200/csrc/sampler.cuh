@@ -120,29 +120,36 @@ struct SubSlice {
   }
 };
 
-// thread-local (max, sum 2^(x*log2e - max)) of a slice; the maximum is returned in the log2 domain
+// thread-local (max, sum 2^(x*log2e - max)) of a slice; the maximum is returned in the log2 domain.
+// Four independent maxima and four independent partial sums keep the dependency chains short
+// (the reduction order is fixed, so results do not depend on scheduling).
 __device__ __forceinline__ void slice_stats(const SubSlice<__nv_bfloat16> &sl, float &m, float &s) {
   constexpr int NV = SubSlice<__nv_bfloat16>::NV;
   // packed bf16 maximum: one instruction per two tokens
-  __nv_bfloat162 mx = *reinterpret_cast<const __nv_bfloat162 *>(&sl.raw[0].x);
+  __nv_bfloat162 mx[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) mx[i] = *reinterpret_cast<const __nv_bfloat162 *>(&sl.raw[0].x);
 #pragma unroll
   for (int c = 0; c < NV; ++c) {
     const uint32_t w[4] = {sl.raw[c].x, sl.raw[c].y, sl.raw[c].z, sl.raw[c].w};
 #pragma unroll
-    for (int i = 0; i < 4; ++i) mx = __hmax2(mx, *reinterpret_cast<const __nv_bfloat162 *>(&w[i]));
+    for (int i = 0; i < 4; ++i) mx[i] = __hmax2(mx[i], *reinterpret_cast<const __nv_bfloat162 *>(&w[i]));
   }
-  m = fmaxf(__low2float(mx), __high2float(mx)) * kLog2e;
+  const __nv_bfloat162 mm = __hmax2(__hmax2(mx[0], mx[1]), __hmax2(mx[2], mx[3]));
+  m = fmaxf(__low2float(mm), __high2float(mm)) * kLog2e;
   s = 0.f;
   if (m == -INFINITY) return;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
   for (int c = 0; c < NV; ++c) {
     const uint32_t w[4] = {sl.raw[c].x, sl.raw[c].y, sl.raw[c].z, sl.raw[c].w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      s += fast_exp2(fmaf(__uint_as_float(w[i] << 16), kLog2e, -m));
-      s += fast_exp2(fmaf(__uint_as_float(w[i] & 0xffff0000u), kLog2e, -m));
+      acc[i] += fast_exp2(fmaf(__uint_as_float(w[i] << 16), kLog2e, -m));
+      acc[i] += fast_exp2(fmaf(__uint_as_float(w[i] & 0xffff0000u), kLog2e, -m));
     }
   }
+  s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
 }
 __device__ __forceinline__ void slice_stats(const SubSlice<float> &sl, float &m, float &s) {
   constexpr int NV = SubSlice<float>::NV;
@@ -191,6 +198,132 @@ __global__ void __launch_bounds__(kSampThreads) row_stats_kernel(SampleParams p,
     const float S = warp_sum(s);
     if (lane == 0) p.seg_stats[u] = make_float2(M, S);
     cur = nxt;
+  }
+}
+
+// Pass 1 for bf16 logits, fed by bulk asynchronous copies.  One CTA per SM: a producer thread
+// streams 32 KB chunks of logits rows (16384 tokens = 8 sub-segments) into a ring of shared-memory
+// stages with cp.async.bulk; eight consumer warps each reduce one sub-segment of every stage.
+// 192 KB are in flight per SM whatever the consumers are doing, which the register-prefetching
+// kernel above cannot offer (its loads in flight are bounded by its registers).  Same outputs
+// (seg_stats layout and values) as row_stats_kernel.
+constexpr int kRingStageElems = 16384;
+constexpr int kRingStages = 6;
+constexpr int kRingConsumerWarps = kRingStageElems / kSubElems;  // 8 warps reduce one stage
+#ifndef SPX_RING_GROUPS
+#define SPX_RING_GROUPS 3
+#endif
+constexpr int kRingGroups = SPX_RING_GROUPS;                     // groups of 8 warps, each takes every kRingGroups-th stage
+constexpr int kRingThreads = (kRingGroups * kRingConsumerWarps + 1) * 32;
+constexpr int kRingSmemBytes = kRingStages * kRingStageElems * 2 + 1024 + 256;
+
+__device__ __forceinline__ bool ring_wait(uint64_t *bar, uint32_t parity, volatile int *abort, int32_t *dev_status) {
+  const uint32_t addr = (uint32_t)__cvta_generic_to_shared(bar);
+  const long long t0 = clock64();
+  for (;;) {
+    for (int i = 0; i < 64; ++i) {
+      uint32_t ok;
+      asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                   : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+      if (ok) return true;
+    }
+    if (*abort) return false;
+    if (clock64() - t0 > (1ll << 31)) {  // about a second: give up, report, let the others leave too
+      *abort = 1;
+      atomicOr(dev_status, SPX_DEV_TIMEOUT);
+      return false;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleParams p, int chunks_per_row, int n_chunks) {
+  extern __shared__ __align__(1024) unsigned char ring_smem[];
+  unsigned char *stages = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(ring_smem) + 1023) & ~uintptr_t(1023));
+  uint64_t *full = reinterpret_cast<uint64_t *>(stages + kRingStages * kRingStageElems * 2);
+  uint64_t *empty = full + kRingStages;
+  volatile int *abort = reinterpret_cast<volatile int *>(empty + kRingStages);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kRingStages; ++s) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(&full[s])), "r"(1));
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(&empty[s])), "r"(kRingConsumerWarps));
+    }
+    *abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const __nv_bfloat16 *target = reinterpret_cast<const __nv_bfloat16 *>(p.target);
+  const __nv_bfloat16 *draft = reinterpret_cast<const __nv_bfloat16 *>(p.draft);
+  auto chunk_src = [&](int g, int &row, int &e0) -> const __nv_bfloat16 * {
+    row = g / chunks_per_row;
+    e0 = (g % chunks_per_row) * kRingStageElems;
+    const __nv_bfloat16 *base = row < p.total_q ? target + (int64_t)row * p.row_stride
+                                                : draft + (int64_t)(row - p.total_q) * p.row_stride;
+    return base + e0;
+  };
+  if (warp == kRingGroups * kRingConsumerWarps) {
+    // ---- producer (one thread)
+    if (lane == 0) {
+      int i = 0;
+      for (int g = blockIdx.x; g < n_chunks; g += gridDim.x, ++i) {
+        const int s = i % kRingStages;
+        if (i >= kRingStages && !ring_wait(&empty[s], ((i / kRingStages) - 1) & 1, abort, p.dev_status)) break;
+        int row, e0;
+        const __nv_bfloat16 *src = chunk_src(g, row, e0);
+        const int elems = min(kRingStageElems, p.vocab - e0);
+        const uint32_t bytes = (uint32_t)((elems * 2 + 15) & ~15);  // stays inside the row: its stride is a multiple of 16 bytes
+        const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&full[s]);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"((uint32_t)__cvta_generic_to_shared(stages + (size_t)s * kRingStageElems * 2)), "l"(src), "r"(bytes), "r"(bar)
+                     : "memory");
+      }
+    }
+  } else {
+    // ---- consumers: group `grp` takes chunks grp, grp + kRingGroups, ...; its warp w reduces
+    // sub-segment w of each of them
+    const int grp = warp / kRingConsumerWarps;
+    const int wsub = warp % kRingConsumerWarps;
+    int i = grp;
+    for (int g = blockIdx.x + grp * gridDim.x; g < n_chunks; g += kRingGroups * gridDim.x, i += kRingGroups) {
+      const int s = i % kRingStages;
+      const bool ok = __all_sync(0xffffffffu, ring_wait(&full[s], (i / kRingStages) & 1, abort, p.dev_status));
+      if (!ok) break;
+      int row, e0;
+      chunk_src(g, row, e0);
+      const int v_sub = e0 + wsub * kSubElems;  // first token of this warp's sub-segment
+      if (v_sub < p.vocab) {
+        SubSlice<__nv_bfloat16> sl;
+        const uint4 *src = reinterpret_cast<const uint4 *>(stages + (size_t)s * kRingStageElems * 2 + (size_t)wsub * kSubElems * 2);
+#pragma unroll
+        for (int c = 0; c < SubSlice<__nv_bfloat16>::NV; ++c) {
+          uint4 v = src[c * 32 + lane];
+          const int tok = v_sub + (c * 32 + lane) * 8;
+          if (tok + 8 > p.vocab) {
+            // tokens past the vocabulary (never copied, or the row's padding): -inf
+            uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (tok + 2 * j >= p.vocab) w[j] = (w[j] & 0xffff0000u) | 0xff80u;
+              if (tok + 2 * j + 1 >= p.vocab) w[j] = (w[j] & 0x0000ffffu) | 0xff800000u;
+            }
+            v = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+          sl.raw[c] = v;
+        }
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"((uint32_t)__cvta_generic_to_shared(&empty[s])) : "memory");
+        float m, sum;
+        slice_stats(sl, m, sum);
+        const float M = warp_max(m);
+        if (M > -INFINITY) sum *= fast_exp2(m - M);
+        const float S = warp_sum(sum);
+        if (lane == 0) p.seg_stats[(int64_t)row * p.nsub + (v_sub / kSubElems)] = make_float2(M, S);
+      } else {
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"((uint32_t)__cvta_generic_to_shared(&empty[s])) : "memory");
+      }
+    }
   }
 }
 

@@ -5,6 +5,7 @@
 #include <cstdint>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 
 #include "attn_simt.cuh"
 #include "attn_tc.cuh"
@@ -346,7 +347,17 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
   const int max_grid = (n_units + kSampThreads / 32 - 1) / (kSampThreads / 32);
   if (grid > max_grid) grid = max_grid;
   if (phases & kPhaseStats) {
-    row_stats_kernel<T><<<grid, kSampThreads, 0, stream>>>(p, n_units);
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+      // bf16 logits: the bulk-copy ring kernel, one CTA per SM
+      static_assert(kSubElems == 2048, "the ring kernel reduces 2048-token sub-segments");
+      if (cudaFuncSetAttribute(row_stats_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmemBytes) != cudaSuccess)
+        return SPX_ERR_CUDA;
+      const int chunks_per_row = (p.vocab + kRingStageElems - 1) / kRingStageElems;
+      const int n_chunks = rows * chunks_per_row;
+      row_stats_ring_kernel<<<num_sms < n_chunks ? num_sms : n_chunks, kRingThreads, kRingSmemBytes, stream>>>(p, chunks_per_row, n_chunks);
+    } else {
+      row_stats_kernel<T><<<grid, kSampThreads, 0, stream>>>(p, n_units);
+    }
     ++t_launches;
   }
   if (phases & kPhaseTail) {
@@ -453,12 +464,15 @@ spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_
   bool ok = cudaEventRecord(side->fork, stream) == cudaSuccess;
   ok = ok && cudaStreamWaitEvent(side->stream, side->fork, 0) == cudaSuccess;
   if (!ok) return SPX_ERR_CUDA;
+  // launch order matters: the one-block planner goes first so that it is not queued behind the
+  // persistent blocks of the logits pass, which occupy every SM for their whole run
+  const spx_status_t s0 = launch_attention(attn, base, dev_status, stream, dev, kPhasePlan);
   const spx_status_t s1 = launch_sampler(sample, base + attn_bytes, dev_status, side->stream, dev.num_sms);
   ok = ok && cudaEventRecord(side->join, side->stream) == cudaSuccess;
-  const spx_status_t s2 = launch_attention(attn, base, dev_status, stream, dev);
+  const spx_status_t s2 = launch_attention(attn, base, dev_status, stream, dev, kPhaseMain);
   ok = ok && cudaStreamWaitEvent(stream, side->join, 0) == cudaSuccess;
   if (!ok) return SPX_ERR_CUDA;
-  return s1 != SPX_OK ? s1 : s2;
+  return s0 != SPX_OK ? s0 : s1 != SPX_OK ? s1 : s2;
 }
 
 // ---- host-buffer convenience ---------------------------------------------------------------
