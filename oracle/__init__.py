@@ -66,6 +66,12 @@ def _load():
         lib.oracle_emit_cdf.argtypes = [c.c_int32, c.c_int32, c.c_int64, c.c_int64, c.c_int32,
                                         c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
         lib.oracle_verify_step.restype = c.c_int
+        lib.oracle_kv_append.restype = c.c_int
+        lib.oracle_kv_append.argtypes = [c.c_int32, c.c_int32, c.c_int32, c.c_int32, c.c_int64, c.c_int32, c.c_int32,
+                                         c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int64, c.c_int64, c.c_int64,
+                                         c.c_void_p, c.c_void_p, c.c_void_p]
+        lib.oracle_kv_rollback.restype = c.c_int
+        lib.oracle_kv_rollback.argtypes = [c.c_int32, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
         _lib = lib
     return _lib
 
@@ -227,3 +233,35 @@ def emit_cdf(r: int, n: int, target_logits: torch.Tensor, draft_logits: torch.Te
     R = lib.oracle_emit_cdf(int(r), int(n), V, tl.stride(0), _dtype_code(tl), _ptr(tl), _ptr(dl),
                             _ptr(qi), _ptr(cdf))
     return cdf, float(R)
+
+
+def kv_append(new_k: torch.Tensor, new_v: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
+              kv_strides: Sequence[int], block_table: torch.Tensor, seq_lens: torch.Tensor, q_indptr: torch.Tensor,
+              page_size: int, num_pages: int) -> None:
+    """Write the new positions' K/V ([TQ, Hkv, D]) into their pages, in place (bit copies)."""
+    lib = _load()
+    nk, nv = _cpu(new_k).contiguous(), _cpu(new_v).contiguous()
+    assert nk.dtype == k_cache.dtype == v_cache.dtype == nv.dtype
+    _dtype_code(nk)
+    TQ, Hkv, D = nk.shape
+    bt = _cpu(block_table, torch.int32).contiguous()
+    sl = _cpu(seq_lens, torch.int32).contiguous()
+    qi = _cpu(q_indptr, torch.int32).contiguous()
+    st = lib.oracle_kv_append(sl.numel(), Hkv, D, page_size, num_pages, bt.shape[1], nk.element_size(), _ptr(nk),
+                              _ptr(nv), _ptr(_cpu(k_cache)), _ptr(_cpu(v_cache)), int(kv_strides[0]),
+                              int(kv_strides[1]), int(kv_strides[2]), _ptr(bt), _ptr(sl), _ptr(qi))
+    if st != OK:
+        raise OracleError(st)
+
+
+def kv_rollback(seq_lens: torch.Tensor, q_indptr: torch.Tensor, accepted_len: torch.Tensor) -> torch.Tensor:
+    """Lengths after dropping the rejected drafts: L - (k - n)."""
+    lib = _load()
+    sl = _cpu(seq_lens, torch.int32).contiguous()
+    qi = _cpu(q_indptr, torch.int32).contiguous()
+    al = _cpu(accepted_len, torch.int32).contiguous()
+    out = torch.empty_like(sl)
+    st = lib.oracle_kv_rollback(sl.numel(), _ptr(sl), _ptr(qi), _ptr(al), _ptr(out))
+    if st != OK:
+        raise OracleError(st)
+    return out

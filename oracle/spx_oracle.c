@@ -30,7 +30,10 @@
  * mean of V and LSE = log n; one token gives V[0]), a needle key, GQA head duplication; for
  * sampling a chi-square test of the output law against the target distribution on a
  * 16-token vocabulary, the identity min(p,q) + (1-beta) r/R = p, closed-form acceptance
- * rates, special cases, and interval-arithmetic brute force on tiny vocabularies.
+ * rates, special cases, and interval-arithmetic brute force on tiny vocabularies; for the
+ * cache maintenance (tests/test_oracle_kv.py) torch's indexed scatter on the un-paged view,
+ * bit-identity of every untouched slot, append-then-attend against attending a cache that was
+ * filled directly, and the closed form of the rolled-back lengths.
  */
 #include <math.h>
 #include <stdint.h>
@@ -412,6 +415,70 @@ double oracle_emit_cdf(int32_t r, int32_t n, int64_t V, int64_t row_stride, int3
   }
   free(p); free(q);
   return R;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* (D) cache maintenance around the step                                                 */
+/* ------------------------------------------------------------------------------------ */
+
+/*
+ * Append: the K/V of request r's m_r = k_r+1 new positions (rows q_indptr[r].. of new_k/new_v,
+ * laid out [TQ, Hkv, D]) are written at logical tokens L_r-m_r .. L_r-1 of the request, i.e.
+ * page block_table[r][t/P], slot t%P.  L_r already counts the new positions.  This is the shared
+ * cache of Section 4 ("speculative execution ... shares the cache with normal execution"): the
+ * drafts' entries go into the same pages as everything else, nothing is duplicated.
+ * elem_size is 2 (bf16) or 4 (fp32); the values are copied bit for bit.
+ */
+int oracle_kv_append(int32_t batch, int32_t Hkv, int32_t D, int32_t P, int64_t num_pages,
+                     int32_t max_pages_per_req, int32_t elem_size, const void *new_k,
+                     const void *new_v, void *k_cache, void *v_cache, int64_t stride_page,
+                     int64_t stride_head, int64_t stride_token, const int32_t *block_table,
+                     const int32_t *seq_lens, const int32_t *q_indptr) {
+  if (batch < 0 || Hkv <= 0 || D <= 0 || P <= 0 || (elem_size != 2 && elem_size != 4)) return ORACLE_ERR_ARG;
+  for (int r = 0; r < batch; ++r) {
+    const int m = q_indptr[r + 1] - q_indptr[r];
+    const int L = seq_lens[r];
+    if (m < 1 || L < m) return ORACLE_ERR_LEN;
+    if ((L + P - 1) / P > max_pages_per_req) return ORACLE_ERR_PAGE;
+    for (int j = 0; j < m; ++j) {
+      const int t = L - m + j;
+      const int32_t phys = block_table[(int64_t)r * max_pages_per_req + t / P];
+      if (phys < 0 || phys >= num_pages) return ORACLE_ERR_PAGE;
+    }
+  }
+  for (int r = 0; r < batch; ++r) {
+    const int m = q_indptr[r + 1] - q_indptr[r];
+    const int L = seq_lens[r];
+    for (int j = 0; j < m; ++j) {
+      const int t = L - m + j;
+      const int64_t page = block_table[(int64_t)r * max_pages_per_req + t / P];
+      for (int g = 0; g < Hkv; ++g) {
+        const int64_t dst = page * stride_page + (int64_t)g * stride_head + (int64_t)(t % P) * stride_token;
+        const int64_t src = (((int64_t)q_indptr[r] + j) * Hkv + g) * D;
+        memcpy((char *)k_cache + dst * elem_size, (const char *)new_k + src * elem_size, (size_t)D * elem_size);
+        memcpy((char *)v_cache + dst * elem_size, (const char *)new_v + src * elem_size, (size_t)D * elem_size);
+      }
+    }
+  }
+  return ORACLE_OK;
+}
+
+/*
+ * Rollback: of the k_r+1 new positions, position 0 (the last committed token) and the n_r accepted
+ * drafts stay in the cache; the k_r - n_r rejected drafts' entries are dropped by shrinking the
+ * length (Figure 3 of the paper: accepted speculation continues, rejected speculation is
+ * re-executed).  new_seq_lens[r] = L_r - (k_r - n_r).  The emitted token is the next step's
+ * position 0 and is not in the cache yet.
+ */
+int oracle_kv_rollback(int32_t batch, const int32_t *seq_lens, const int32_t *q_indptr,
+                       const int32_t *accepted_len, int32_t *new_seq_lens) {
+  for (int r = 0; r < batch; ++r) {
+    const int k = q_indptr[r + 1] - q_indptr[r] - 1;
+    const int n = accepted_len[r];
+    if (k < 0 || n < 0 || n > k || seq_lens[r] < k + 1) return ORACLE_ERR_LEN;
+    new_seq_lens[r] = seq_lens[r] - (k - n);
+  }
+  return ORACLE_OK;
 }
 
 /* ------------------------------------------------------------------------------------ */
