@@ -158,6 +158,41 @@ spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_
                              size_t ws_bytes, int32_t *dev_status, void *cuda_stream);
 
 /*
+ * Cache maintenance around the step (the paper's Section 4: speculative execution shares the
+ * paged cache with normal execution; its Figure 3: accepted speculation continues, rejected
+ * speculation is re-executed).
+ *
+ * spx_kv_append writes the K/V of every request's k_r+1 new positions into their pages BEFORE
+ * attention: row q_indptr[r]+j of new_k/new_v ([TQ, num_kv_heads, head_dim], contiguous, same
+ * dtype as the pools) goes to logical token L_r-(k_r+1)+j of request r, i.e. page
+ * block_table[r][t/page_size], slot t%page_size (seq_lens already counts the new positions).
+ * Values are copied bit for bit; no other slot is touched.  Requests with an invalid length or
+ * page id set SPX_DEV_BAD_LEN / SPX_DEV_BAD_PAGE and are skipped.  Pools and strides as in
+ * spx_attn_args_t; head_dim * element size must be a multiple of 16 bytes.
+ *
+ * spx_kv_rollback computes, AFTER sampling, the lengths that drop the rejected drafts:
+ * new_seq_lens[r] = seq_lens[r] - (k_r - accepted_len[r]) (position 0 and the accepted drafts
+ * stay; the emitted token is the next step's position 0 and is not cached yet).  An accepted
+ * length outside [0, k_r] sets SPX_DEV_BAD_LEN and writes -1.  new_seq_lens may alias seq_lens.
+ */
+typedef struct {
+  int32_t batch, total_q;
+  int32_t num_kv_heads, head_dim, page_size, num_pages, max_pages_per_req;
+  spx_dtype_t kv_dtype;
+  const void *new_k, *new_v;          /* [TQ, num_kv_heads, head_dim]                         */
+  void *k_cache, *v_cache;            /* pools, written                                       */
+  int64_t kv_stride_page, kv_stride_head, kv_stride_token;
+  const int32_t *block_table;         /* [B, max_pages_per_req]                               */
+  const int32_t *seq_lens;            /* [B], counts the new positions                        */
+  const int32_t *q_indptr;            /* [B+1]                                                */
+} spx_kv_append_args_t;
+
+spx_status_t spx_kv_append(const spx_kv_append_args_t *args, int32_t *dev_status, void *cuda_stream);
+spx_status_t spx_kv_rollback(int32_t batch, const int32_t *seq_lens, const int32_t *q_indptr,
+                             const int32_t *accepted_len, int32_t *new_seq_lens, int32_t *dev_status,
+                             void *cuda_stream);
+
+/*
  * Convenience for callers whose data lives on the HOST: every pointer in the two structs is a
  * host pointer (pinned memory recommended); device staging buffers, the workspace and the
  * status word are carved from `dev_arena` (device memory, `arena_bytes` >=

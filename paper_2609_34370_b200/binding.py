@@ -16,7 +16,7 @@ BF16, F32 = 0, 1
 
 EXPORTS = ("spx_workspace_size", "spx_verify_attention", "spx_rejection_sample", "spx_verify_step",
            "spx_host_step_arena_size", "spx_verify_step_host", "spx_status_string", "spx_last_launch_count",
-           "spx_set_timing_events", "spx_rejection_sample_static")
+           "spx_set_timing_events", "spx_rejection_sample_static", "spx_kv_append", "spx_kv_rollback")
 
 
 class AttnArgs(C.Structure):
@@ -39,6 +39,17 @@ class SampleArgs(C.Structure):
         ("target_logits", C.c_void_p), ("draft_logits", C.c_void_p), ("draft_token_ids", C.c_void_p),
         ("q_indptr", C.c_void_p), ("u_accept", C.c_void_p), ("u_sample", C.c_void_p),
         ("accepted_len", C.c_void_p), ("out_tokens", C.c_void_p), ("diag_ratio", C.c_void_p),
+    ]
+
+
+class KvAppendArgs(C.Structure):
+    _fields_ = [
+        ("batch", C.c_int32), ("total_q", C.c_int32),
+        ("num_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("page_size", C.c_int32), ("num_pages", C.c_int32),
+        ("max_pages_per_req", C.c_int32), ("kv_dtype", C.c_int),
+        ("new_k", C.c_void_p), ("new_v", C.c_void_p), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+        ("kv_stride_page", C.c_int64), ("kv_stride_head", C.c_int64), ("kv_stride_token", C.c_int64),
+        ("block_table", C.c_void_p), ("seq_lens", C.c_void_p), ("q_indptr", C.c_void_p),
     ]
 
 
@@ -82,6 +93,10 @@ def load_library():
         lib.spx_last_launch_count.restype = C.c_int32
         lib.spx_rejection_sample_static.restype = C.c_int
         lib.spx_rejection_sample_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.spx_kv_append.restype = C.c_int
+        lib.spx_kv_append.argtypes = [C.POINTER(KvAppendArgs), C.c_void_p, C.c_void_p]
+        lib.spx_kv_rollback.restype = C.c_int
+        lib.spx_kv_rollback.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.spx_set_timing_events.restype = None
         lib.spx_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
         _lib = lib
@@ -284,3 +299,38 @@ def rejection_sample_static(target_logits, draft_logits, draft_ids, q_indptr, u_
                          None, vocab)
     _check(lib.spx_rejection_sample_static(C.byref(s), status.data_ptr(), _stream(dev)))
     return accepted, tokens, status
+
+
+def kv_append(new_k, new_v, k_cache, v_cache, kv_strides, block_table, seq_lens, q_indptr, page_size, num_pages,
+              status: Optional[torch.Tensor] = None):
+    """spx_kv_append on the current stream: the new positions' K/V go into their pages, in place."""
+    _require_cuda(new_k, new_v, k_cache, v_cache, block_table, seq_lens, q_indptr)
+    lib = load_library()
+    dev = new_k.device
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    a = KvAppendArgs()
+    a.batch, a.total_q = seq_lens.numel(), new_k.shape[0]
+    a.num_kv_heads, a.head_dim, a.page_size, a.num_pages = new_k.shape[1], new_k.shape[2], page_size, num_pages
+    a.max_pages_per_req = block_table.shape[1]
+    a.kv_dtype = _dtype_code(new_k)
+    a.new_k, a.new_v, a.k_cache, a.v_cache = _ptr(new_k), _ptr(new_v), _ptr(k_cache), _ptr(v_cache)
+    a.kv_stride_page, a.kv_stride_head, a.kv_stride_token = (int(x) for x in kv_strides)
+    a.block_table, a.seq_lens, a.q_indptr = _ptr(block_table), _ptr(seq_lens), q_indptr.data_ptr()
+    _check(lib.spx_kv_append(C.byref(a), status.data_ptr(), _stream(dev)))
+    return status
+
+
+def kv_rollback(seq_lens, q_indptr, accepted_len, out: Optional[torch.Tensor] = None,
+                status: Optional[torch.Tensor] = None):
+    """spx_kv_rollback on the current stream.  Returns (new_seq_lens, status)."""
+    _require_cuda(seq_lens, q_indptr, accepted_len)
+    lib = load_library()
+    dev = seq_lens.device
+    if out is None:
+        out = torch.empty_like(seq_lens)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    _check(lib.spx_kv_rollback(seq_lens.numel(), seq_lens.data_ptr(), q_indptr.data_ptr(), accepted_len.data_ptr(),
+                               out.data_ptr(), status.data_ptr(), _stream(dev)))
+    return out, status

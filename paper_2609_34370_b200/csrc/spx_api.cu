@@ -11,6 +11,7 @@
 #include "attn_tc.cuh"
 #include "attn_tc4.cuh"
 #include "common.cuh"
+#include "kv_cache.cuh"
 #include "plan.cuh"
 #include "sampler.cuh"
 #include "spx.h"
@@ -549,6 +550,48 @@ spx_status_t spx_verify_step_host(const spx_attn_args_t *attn, const spx_sample_
   d2h(attn->out, L.out, L.out_bytes); d2h(attn->lse, L.lse, L.lse_bytes);
   d2h(sample->accepted_len, L.acc, B * 4); d2h(sample->out_tokens, L.tok, TQ * 4); d2h(dev_status_host, L.status, 4);
   return ok ? SPX_OK : SPX_ERR_CUDA;
+}
+
+// ---- cache maintenance ------------------------------------------------------------------------
+spx_status_t spx_kv_append(const spx_kv_append_args_t *a, int32_t *dev_status, void *cuda_stream) {
+  t_launches = 0;
+  if (!a || !dev_status) return SPX_ERR_INVALID_ARG;
+  if (a->batch < 0 || a->total_q < a->batch || a->num_kv_heads <= 0 || a->head_dim <= 0 || a->page_size <= 0 ||
+      a->num_pages < 0 || a->max_pages_per_req < 0)
+    return SPX_ERR_INVALID_ARG;
+  if (a->kv_dtype != SPX_BF16 && a->kv_dtype != SPX_F32) return SPX_ERR_INVALID_ARG;
+  if ((a->page_size & (a->page_size - 1)) != 0) return SPX_ERR_UNSUPPORTED;
+  const int es = a->kv_dtype == SPX_BF16 ? 2 : 4;
+  if ((a->head_dim * es) % 16 != 0) return SPX_ERR_UNSUPPORTED;
+  if (a->kv_stride_page < 0 || a->kv_stride_head < 0 || a->kv_stride_token < a->head_dim) return SPX_ERR_INVALID_ARG;
+  if (a->batch == 0) return SPX_OK;
+  if (!a->new_k || !a->new_v || !a->k_cache || !a->v_cache || !a->block_table || !a->seq_lens || !a->q_indptr)
+    return SPX_ERR_INVALID_ARG;
+  if (((uintptr_t)a->new_k | (uintptr_t)a->new_v | (uintptr_t)a->k_cache | (uintptr_t)a->v_cache) & 15) return SPX_ERR_INVALID_ARG;
+  if (((a->kv_stride_page * es) | (a->kv_stride_head * es) | (a->kv_stride_token * es)) & 15) return SPX_ERR_INVALID_ARG;
+  KvAppendParams p{};
+  p.batch = a->batch; p.total_q = a->total_q; p.Hkv = a->num_kv_heads; p.D = a->head_dim; p.P = a->page_size;
+  while ((1 << p.log2P) < p.P) ++p.log2P;
+  p.num_pages = a->num_pages; p.max_pages_per_req = a->max_pages_per_req; p.elem_size = es;
+  p.new_k = static_cast<const unsigned char *>(a->new_k); p.new_v = static_cast<const unsigned char *>(a->new_v);
+  p.k_cache = static_cast<unsigned char *>(a->k_cache); p.v_cache = static_cast<unsigned char *>(a->v_cache);
+  p.stride_page = a->kv_stride_page; p.stride_head = a->kv_stride_head; p.stride_token = a->kv_stride_token;
+  p.block_table = a->block_table; p.seq_lens = a->seq_lens; p.q_indptr = a->q_indptr; p.dev_status = dev_status;
+  kv_append_kernel<<<a->batch, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p);
+  ++t_launches;
+  return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
+}
+
+spx_status_t spx_kv_rollback(int32_t batch, const int32_t *seq_lens, const int32_t *q_indptr, const int32_t *accepted_len,
+                             int32_t *new_seq_lens, int32_t *dev_status, void *cuda_stream) {
+  t_launches = 0;
+  if (batch < 0 || !dev_status) return SPX_ERR_INVALID_ARG;
+  if (batch == 0) return SPX_OK;
+  if (!seq_lens || !q_indptr || !accepted_len || !new_seq_lens) return SPX_ERR_INVALID_ARG;
+  kv_rollback_kernel<<<(batch + 127) / 128, 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(batch, seq_lens, q_indptr,
+                                                                                               accepted_len, new_seq_lens, dev_status);
+  ++t_launches;
+  return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
 }
 
 // ---- sampling without caller-provided scratch ------------------------------------------------
