@@ -11,6 +11,7 @@ float64 / int32 CPU tensors.
 from __future__ import annotations
 
 import ctypes
+import ctypes as c
 import os
 import subprocess
 from dataclasses import dataclass
@@ -23,7 +24,7 @@ _SRC = os.path.join(_HERE, "spx_oracle.c")
 _LIB_PATH = os.path.join(_HERE, "libspx_oracle.so")
 
 BF16, F32 = 0, 1
-OK, ERR_ARG, ERR_LEN, ERR_PAGE, ERR_TOKEN, ERR_ALLOC = 0, 1, 2, 3, 4, 5
+OK, ERR_ARG, ERR_LEN, ERR_PAGE, ERR_TOKEN, ERR_ALLOC, ERR_PARAM = 0, 1, 2, 3, 4, 5, 6
 FLAG_DEGENERATE = 1
 
 _lib = None
@@ -142,13 +143,27 @@ def verify_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tens
     return out, lse
 
 
-def softmax_row(logits_row: torch.Tensor) -> torch.Tensor:
-    """Step 1 of the sampling rule: float64 softmax of one stored logits row."""
+def softmax_row(logits_row: torch.Tensor, tau: Optional[float] = None) -> torch.Tensor:
+    """Step 1 of the sampling rule: float64 softmax of one stored logits row (at temperature tau)."""
     lib = _load()
     row = _cpu(logits_row).contiguous()
     p = torch.empty(row.numel(), dtype=torch.float64)
-    lib.oracle_softmax_row(_ptr(row), _dtype_code(row), 0, row.numel(), _ptr(p))
+    if tau is None:
+        lib.oracle_softmax_row(_ptr(row), _dtype_code(row), 0, row.numel(), _ptr(p))
+    else:
+        lib.oracle_softmax_row_tau.restype = None
+        lib.oracle_softmax_row_tau.argtypes = [c.c_void_p, c.c_int32, c.c_int64, c.c_int64, c.c_double, c.c_void_p]
+        lib.oracle_softmax_row_tau(_ptr(row), _dtype_code(row), 0, row.numel(), float(tau), _ptr(p))
     return p
+
+
+def argmax_row(logits_row: torch.Tensor) -> int:
+    """Greedy choice of one stored logits row: the lowest id attaining the maximum."""
+    lib = _load()
+    row = _cpu(logits_row).contiguous()
+    lib.oracle_argmax_row.restype = c.c_int64
+    lib.oracle_argmax_row.argtypes = [c.c_void_p, c.c_int32, c.c_int64, c.c_int64]
+    return int(lib.oracle_argmax_row(_ptr(row), _dtype_code(row), 0, row.numel()))
 
 
 def residual(p: torch.Tensor, q: torch.Tensor):
@@ -177,13 +192,15 @@ class SampleResult:
     cdf_lo: torch.Tensor         # [B] float64
     cdf_hi: torch.Tensor         # [B] float64
     flags: torch.Tensor          # [B] int32
-    status: int                  # OK or ERR_TOKEN
+    status: int                  # OK, ERR_TOKEN or ERR_PARAM
 
 
 def rejection_sample(target_logits: torch.Tensor, draft_logits: torch.Tensor,
                      draft_ids: torch.Tensor, q_indptr: torch.Tensor, u_accept: torch.Tensor,
-                     u_sample: torch.Tensor, vocab: Optional[int] = None) -> SampleResult:
-    """Speculative rejection sampling for the whole batch, in float64, one request at a time."""
+                     u_sample: torch.Tensor, vocab: Optional[int] = None,
+                     temperature: Optional[torch.Tensor] = None) -> SampleResult:
+    """Speculative rejection sampling for the whole batch, in float64, one request at a time.
+    ``temperature`` ([B] float32, optional): > 0 verifies at that temperature, 0 verifies greedily."""
     lib = _load()
     tl = _cpu(target_logits)
     dl = _cpu(draft_logits)
@@ -211,18 +228,28 @@ def rejection_sample(target_logits: torch.Tensor, draft_logits: torch.Tensor,
         cdf_hi=torch.empty(B, dtype=torch.float64),
         flags=torch.empty(B, dtype=torch.int32),
         status=OK)
-    st = lib.oracle_rejection_sample(
-        B, V, row_stride, dt, _ptr(tl), _ptr(dl), _ptr(ids), _ptr(qi), _ptr(ua), _ptr(us),
-        _ptr(res.accepted_len), _ptr(res.out_tokens), _ptr(res.rho), _ptr(res.resid_mass),
-        _ptr(res.cdf_lo), _ptr(res.cdf_hi), _ptr(res.flags))
-    if st not in (OK, ERR_TOKEN):
+    if temperature is None:
+        st = lib.oracle_rejection_sample(
+            B, V, row_stride, dt, _ptr(tl), _ptr(dl), _ptr(ids), _ptr(qi), _ptr(ua), _ptr(us),
+            _ptr(res.accepted_len), _ptr(res.out_tokens), _ptr(res.rho), _ptr(res.resid_mass),
+            _ptr(res.cdf_lo), _ptr(res.cdf_hi), _ptr(res.flags))
+    else:
+        tau = _cpu(temperature, torch.float32).contiguous()
+        assert tau.numel() == B
+        lib.oracle_rejection_sample_tau.restype = c.c_int
+        lib.oracle_rejection_sample_tau.argtypes = [c.c_int32, c.c_int64, c.c_int64, c.c_int32] + [c.c_void_p] * 14
+        st = lib.oracle_rejection_sample_tau(
+            B, V, row_stride, dt, _ptr(tl), _ptr(dl), _ptr(ids), _ptr(qi), _ptr(ua), _ptr(us), _ptr(tau),
+            _ptr(res.accepted_len), _ptr(res.out_tokens), _ptr(res.rho), _ptr(res.resid_mass),
+            _ptr(res.cdf_lo), _ptr(res.cdf_hi), _ptr(res.flags))
+    if st not in (OK, ERR_TOKEN, ERR_PARAM):
         raise OracleError(st)
     res.status = st
     return res
 
 
 def emit_cdf(r: int, n: int, target_logits: torch.Tensor, draft_logits: torch.Tensor,
-             q_indptr: torch.Tensor, vocab: Optional[int] = None):
+             q_indptr: torch.Tensor, vocab: Optional[int] = None, tau: float = 1.0):
     """Inclusive cumulative distribution request ``r``'s emitted token was drawn from, and R."""
     lib = _load()
     tl = _cpu(target_logits)
@@ -230,8 +257,11 @@ def emit_cdf(r: int, n: int, target_logits: torch.Tensor, draft_logits: torch.Te
     V = int(vocab if vocab is not None else tl.shape[1])
     qi = _cpu(q_indptr, torch.int32).contiguous()
     cdf = torch.empty(V, dtype=torch.float64)
-    R = lib.oracle_emit_cdf(int(r), int(n), V, tl.stride(0), _dtype_code(tl), _ptr(tl), _ptr(dl),
-                            _ptr(qi), _ptr(cdf))
+    lib.oracle_emit_cdf_tau.restype = c.c_double
+    lib.oracle_emit_cdf_tau.argtypes = [c.c_int32, c.c_int32, c.c_int64, c.c_int64, c.c_int32, c.c_void_p, c.c_void_p,
+                                        c.c_void_p, c.c_double, c.c_void_p]
+    R = lib.oracle_emit_cdf_tau(int(r), int(n), V, tl.stride(0), _dtype_code(tl), _ptr(tl), _ptr(dl),
+                                _ptr(qi), float(tau), _ptr(cdf))
     return cdf, float(R)
 
 

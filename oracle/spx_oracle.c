@@ -33,7 +33,12 @@
  * rates, special cases, and interval-arithmetic brute force on tiny vocabularies; for the
  * cache maintenance (tests/test_oracle_kv.py) torch's indexed scatter on the un-paged view,
  * bit-identity of every untouched slot, append-then-attend against attending a cache that was
- * filled directly, and the closed form of the rolled-back lengths.
+ * filled directly, and the closed form of the rolled-back lengths; for the verification
+ * variants (tests/test_oracle_variants.py; the paper fixes no sampling parameters, so these are
+ * this build's reading: the same temperature divides target and draft logits, temperature 0
+ * verifies greedily) the output law against softmax(target / tau), the closed form
+ * tau*ln(w) -> w / sum w, exact invariance under doubling logits and temperature together,
+ * numpy's argmax on rows with ties, and the tau -> 0 limit meeting the greedy branch.
  */
 #include <math.h>
 #include <stdint.h>
@@ -51,7 +56,8 @@ enum {
   ORACLE_ERR_LEN = 2,      /* some L_r < k_r + 1                                     */
   ORACLE_ERR_PAGE = 3,     /* a needed block-table entry is outside [0, num_pages)   */
   ORACLE_ERR_TOKEN = 4,    /* a draft token id is outside [0, V)                     */
-  ORACLE_ERR_ALLOC = 5
+  ORACLE_ERR_ALLOC = 5,
+  ORACLE_ERR_PARAM = 6     /* a per-request sampling parameter is not a temperature  */
 };
 
 /* Bit flags written per request by the sampler. */
@@ -212,9 +218,13 @@ int oracle_verify_attention(int32_t batch, int32_t Hq, int32_t Hkv, int32_t D, i
 /* (B) speculative rejection sampling                                                    */
 /* ------------------------------------------------------------------------------------ */
 
-/* Step 1: p = softmax(row) over the full vocabulary at temperature 1, max subtracted. */
-void oracle_softmax_row(const void *logits, int32_t dtype, int64_t row_offset, int64_t V,
-                        double *p) {
+/*
+ * Step 1: p = softmax(row / tau) over the full vocabulary, max subtracted:
+ * p(v) = exp((x_v - max) / tau) / sum_w exp((x_w - max) / tau), tau > 0.  The paper does not fix
+ * the sampling temperature; tau = 1 is the base case (the division is then exact).
+ */
+void oracle_softmax_row_tau(const void *logits, int32_t dtype, int64_t row_offset, int64_t V,
+                            double tau, double *p) {
   double mx = -INFINITY;
   for (int64_t v = 0; v < V; ++v) {
     const double x = widen(logits, dtype, row_offset + v);
@@ -222,10 +232,26 @@ void oracle_softmax_row(const void *logits, int32_t dtype, int64_t row_offset, i
   }
   double denom = 0.0;
   for (int64_t v = 0; v < V; ++v) {
-    p[v] = exp(widen(logits, dtype, row_offset + v) - mx);
+    p[v] = exp((widen(logits, dtype, row_offset + v) - mx) / tau);
     denom += p[v];
   }
   for (int64_t v = 0; v < V; ++v) p[v] /= denom;
+}
+
+void oracle_softmax_row(const void *logits, int32_t dtype, int64_t row_offset, int64_t V,
+                        double *p) {
+  oracle_softmax_row_tau(logits, dtype, row_offset, V, 1.0, p);
+}
+
+/* Greedy choice of a row: the lowest token id that attains the row maximum. */
+int64_t oracle_argmax_row(const void *logits, int32_t dtype, int64_t row_offset, int64_t V) {
+  int64_t best = 0;
+  double mx = widen(logits, dtype, row_offset);
+  for (int64_t v = 1; v < V; ++v) {
+    const double x = widen(logits, dtype, row_offset + v);
+    if (x > mx) { mx = x; best = v; }
+  }
+  return best;
 }
 
 /* Step 3 (first half): r(v) = max(0, p(v) - q(v)); returns R = sum_v r(v), ascending v. */
@@ -283,7 +309,7 @@ static int sample_one(int r, int32_t dtype, int64_t V, int64_t row_stride,
                       const int32_t *draft_ids, const int32_t *q_indptr, const float *u_accept,
                       const float *u_sample, int32_t *accepted_len, int32_t *out_tokens,
                       double *rho_out, double *resid_mass, double *cdf_lo, double *cdf_hi,
-                      int32_t *flags, double *p, double *q, double *res) {
+                      int32_t *flags, double *p, double *q, double *res, double tau) {
   const int64_t t0 = q_indptr[r];          /* first target row / first output slot */
   const int64_t d0 = (int64_t)q_indptr[r] - r; /* first draft row */
   const int k = q_indptr[r + 1] - q_indptr[r] - 1;
@@ -303,11 +329,36 @@ static int sample_one(int r, int32_t dtype, int64_t V, int64_t row_stride,
   }
   if (rho_out) for (int i = 0; i < k; ++i) rho_out[d0 + i] = NAN; /* rows after n: not consulted */
 
+  if (!(tau >= 0.0) || isinf(tau)) {
+    /* not a temperature: the request emits nothing */
+    accepted_len[r] = 0;
+    for (int i = 0; i <= k; ++i) out_tokens[t0 + i] = -1;
+    if (resid_mass) resid_mass[r] = NAN;
+    if (cdf_lo) cdf_lo[r] = NAN;
+    if (cdf_hi) cdf_hi[r] = NAN;
+    return ORACLE_ERR_PARAM;
+  }
+  if (tau == 0.0) {
+    /* Greedy verification, the tau -> 0 limit with a greedy draft: draft i is accepted iff it is
+     * the target's greedy choice at position i; the first mismatch is replaced by that choice;
+     * with no mismatch the bonus token is the greedy choice of row k.  No uniforms are used. */
+    for (int i = 0; i < k; ++i)
+      if (draft_ids[d0 + i] != oracle_argmax_row(target_logits, dtype, (t0 + i) * row_stride, V)) { n = i; break; }
+    accepted_len[r] = n;
+    for (int i = 0; i < n; ++i) out_tokens[t0 + i] = draft_ids[d0 + i];
+    out_tokens[t0 + n] = (int32_t)oracle_argmax_row(target_logits, dtype, (t0 + n) * row_stride, V);
+    for (int i = n + 1; i <= k; ++i) out_tokens[t0 + i] = -1;
+    if (resid_mass) resid_mass[r] = NAN;
+    if (cdf_lo) cdf_lo[r] = NAN;
+    if (cdf_hi) cdf_hi[r] = NAN;
+    return ORACLE_OK;
+  }
+
   /* step 2: sequential accept tests */
   for (int i = 0; i < k; ++i) {
     const int64_t x = draft_ids[d0 + i];
-    oracle_softmax_row(target_logits, dtype, (t0 + i) * row_stride, V, p);
-    oracle_softmax_row(draft_logits, dtype, (d0 + i) * row_stride, V, q);
+    oracle_softmax_row_tau(target_logits, dtype, (t0 + i) * row_stride, V, tau, p);
+    oracle_softmax_row_tau(draft_logits, dtype, (d0 + i) * row_stride, V, tau, q);
     const double rho = (q[x] == 0.0) ? INFINITY : p[x] / q[x];
     if (rho_out) rho_out[d0 + i] = rho;
     if (!((double)u_accept[d0 + i] < rho)) { n = i; break; }
@@ -326,7 +377,7 @@ static int sample_one(int r, int32_t dtype, int64_t V, int64_t row_stride,
     y = oracle_inverse_cdf(res, V, R, (double)u_sample[r], &lo, &hi);
   } else {
     /* step 4: bonus token from target row k */
-    oracle_softmax_row(target_logits, dtype, (t0 + k) * row_stride, V, p);
+    oracle_softmax_row_tau(target_logits, dtype, (t0 + k) * row_stride, V, tau, p);
     R = 0.0;
     for (int64_t v = 0; v < V; ++v) R += p[v];
     y = oracle_inverse_cdf(p, V, R, (double)u_sample[r], &lo, &hi);
@@ -349,13 +400,20 @@ static int sample_one(int r, int32_t dtype, int64_t V, int64_t row_stride,
  * used), cdf_lo/cdf_hi [B] (cumulative sums bracketing the emitted token), flags [B].
  * Returns ORACLE_ERR_TOKEN if some request carried an invalid draft id (that request emits
  * n = 0 and -1 tokens; the others are unaffected).
+ *
+ * temperature (NULL, or [B]) selects the verification variant per request: tau_r > 0 verifies
+ * against softmax(target / tau_r) with the draft distribution softmax(draft / tau_r) (the draft
+ * was sampled at the request's temperature); tau_r = 0 is greedy verification; anything else
+ * (negative, NaN, infinite) makes that request emit n = 0 and -1 tokens and the call return
+ * ORACLE_ERR_PARAM.  NULL means tau = 1 everywhere.
  */
-int oracle_rejection_sample(int32_t batch, int64_t V, int64_t row_stride, int32_t dtype,
-                            const void *target_logits, const void *draft_logits,
-                            const int32_t *draft_ids, const int32_t *q_indptr,
-                            const float *u_accept, const float *u_sample,
-                            int32_t *accepted_len, int32_t *out_tokens, double *rho_out,
-                            double *resid_mass, double *cdf_lo, double *cdf_hi, int32_t *flags) {
+int oracle_rejection_sample_tau(int32_t batch, int64_t V, int64_t row_stride, int32_t dtype,
+                                const void *target_logits, const void *draft_logits,
+                                const int32_t *draft_ids, const int32_t *q_indptr,
+                                const float *u_accept, const float *u_sample,
+                                const float *temperature, int32_t *accepted_len,
+                                int32_t *out_tokens, double *rho_out, double *resid_mass,
+                                double *cdf_lo, double *cdf_hi, int32_t *flags) {
   if (batch < 0 || V <= 0 || row_stride < V) return ORACLE_ERR_ARG;
   if (dtype != ORACLE_BF16 && dtype != ORACLE_F32) return ORACLE_ERR_ARG;
   for (int r = 0; r < batch; ++r)
@@ -375,7 +433,8 @@ int oracle_rejection_sample(int32_t batch, int64_t V, int64_t row_stride, int32_
       if (!p || !q || !res) continue;
       const int st = sample_one(r, dtype, V, row_stride, target_logits, draft_logits, draft_ids,
                                 q_indptr, u_accept, u_sample, accepted_len, out_tokens, rho_out,
-                                resid_mass, cdf_lo, cdf_hi, flags, p, q, res);
+                                resid_mass, cdf_lo, cdf_hi, flags, p, q, res,
+                                temperature ? (double)temperature[r] : 1.0);
       if (st != ORACLE_OK) {
 #pragma omp atomic write
         status = st;
@@ -386,14 +445,25 @@ int oracle_rejection_sample(int32_t batch, int64_t V, int64_t row_stride, int32_
   return status;
 }
 
+int oracle_rejection_sample(int32_t batch, int64_t V, int64_t row_stride, int32_t dtype,
+                            const void *target_logits, const void *draft_logits,
+                            const int32_t *draft_ids, const int32_t *q_indptr,
+                            const float *u_accept, const float *u_sample,
+                            int32_t *accepted_len, int32_t *out_tokens, double *rho_out,
+                            double *resid_mass, double *cdf_lo, double *cdf_hi, int32_t *flags) {
+  return oracle_rejection_sample_tau(batch, V, row_stride, dtype, target_logits, draft_logits,
+                                     draft_ids, q_indptr, u_accept, u_sample, NULL, accepted_len,
+                                     out_tokens, rho_out, resid_mass, cdf_lo, cdf_hi, flags);
+}
+
 /*
  * The distribution the emitted token of request r was drawn from, as the oracle computed it:
  * cdf[0..V) = inclusive cumulative sum of the residual at row n (n < k) or of the target
  * row k (n == k).  n is passed in (the oracle's accepted_len[r]).  Returns R.
  */
-double oracle_emit_cdf(int32_t r, int32_t n, int64_t V, int64_t row_stride, int32_t dtype,
-                       const void *target_logits, const void *draft_logits,
-                       const int32_t *q_indptr, double *cdf) {
+double oracle_emit_cdf_tau(int32_t r, int32_t n, int64_t V, int64_t row_stride, int32_t dtype,
+                           const void *target_logits, const void *draft_logits,
+                           const int32_t *q_indptr, double tau, double *cdf) {
   const int64_t t0 = q_indptr[r];
   const int64_t d0 = (int64_t)q_indptr[r] - r;
   const int k = q_indptr[r + 1] - q_indptr[r] - 1;
@@ -401,9 +471,9 @@ double oracle_emit_cdf(int32_t r, int32_t n, int64_t V, int64_t row_stride, int3
   double *q = (double *)malloc(sizeof(double) * (size_t)V);
   double R = NAN;
   if (p && q) {
-    oracle_softmax_row(target_logits, dtype, (t0 + n) * row_stride, V, p);
+    oracle_softmax_row_tau(target_logits, dtype, (t0 + n) * row_stride, V, tau, p);
     if (n < k) {
-      oracle_softmax_row(draft_logits, dtype, (d0 + n) * row_stride, V, q);
+      oracle_softmax_row_tau(draft_logits, dtype, (d0 + n) * row_stride, V, tau, q);
       R = oracle_residual(p, q, V, q);
       if (R == 0.0) { R = 0.0; for (int64_t v = 0; v < V; ++v) { q[v] = p[v]; R += p[v]; } }
       oracle_cumsum(q, V, cdf);
@@ -415,6 +485,12 @@ double oracle_emit_cdf(int32_t r, int32_t n, int64_t V, int64_t row_stride, int3
   }
   free(p); free(q);
   return R;
+}
+
+double oracle_emit_cdf(int32_t r, int32_t n, int64_t V, int64_t row_stride, int32_t dtype,
+                       const void *target_logits, const void *draft_logits,
+                       const int32_t *q_indptr, double *cdf) {
+  return oracle_emit_cdf_tau(r, n, V, row_stride, dtype, target_logits, draft_logits, q_indptr, 1.0, cdf);
 }
 
 /* ------------------------------------------------------------------------------------ */
