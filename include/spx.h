@@ -56,7 +56,8 @@ enum {
   SPX_DEV_BAD_TOKEN = 2,  /* a draft token id was outside [0, vocab)                          */
   SPX_DEV_BAD_LEN = 4,    /* seq_len < k+1, k+1 outside [1, max_q_len], or too many pages     */
   SPX_DEV_TIMEOUT = 8,    /* a bounded wait inside a kernel gave up                           */
-  SPX_DEV_DEGENERATE = 16 /* residual mass was zero; the target row was sampled instead       */
+  SPX_DEV_DEGENERATE = 16,/* residual mass was zero; the target row was sampled instead       */
+  SPX_DEV_BAD_PARAM = 32  /* a per-request temperature was negative, NaN or infinite          */
 };
 
 typedef enum { SPX_BF16 = 0, SPX_F32 = 1 } spx_dtype_t;
@@ -112,6 +113,14 @@ typedef struct {
  * Logits rows after n are never needed.  Arithmetic: fp32 exponentials and in-segment sums,
  * float64 across segments and for the accept ratio.
  *
+ * Verification variants (the paper fixes no sampling parameters; temperature == NULL is the
+ * rule above).  temperature[r] = tau > 0: p_i = softmax(T_i / tau), q_i = softmax(D_i / tau) (the
+ * draft was sampled at the request's temperature), everything else unchanged.  temperature[r] = 0:
+ * greedy verification - x_i is accepted iff it is the lowest token id attaining the maximum of
+ * T_i; y is that id for row n; no uniforms are read and diag_ratio stays NaN.  Any other value
+ * sets SPX_DEV_BAD_PARAM and the request emits n = 0 and -1 tokens.  Requests of one batch may mix
+ * all three.
+ *
  * Supported: vocab >= 1; logits_row_stride >= vocab and a multiple of 8 (BF16) or 4 (F32)
  * elements; both logits pointers 16-byte aligned.
  */
@@ -130,6 +139,7 @@ typedef struct {
   int32_t *accepted_len;       /* [B], written                                                */
   int32_t *out_tokens;         /* [TQ], written                                               */
   float *diag_ratio;           /* optional [TD]: p/q of each consulted draft (NaN otherwise)  */
+  const float *temperature;    /* optional [B]: see "Verification variants"; NULL = all 1     */
 } spx_sample_args_t;
 
 /*

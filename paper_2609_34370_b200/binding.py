@@ -11,7 +11,7 @@ import torch
 from .build import LIB_PATH
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = 0, 1, 2, 3, 4
-DEV_BAD_PAGE, DEV_BAD_TOKEN, DEV_BAD_LEN, DEV_TIMEOUT, DEV_DEGENERATE = 1, 2, 4, 8, 16
+DEV_BAD_PAGE, DEV_BAD_TOKEN, DEV_BAD_LEN, DEV_TIMEOUT, DEV_DEGENERATE, DEV_BAD_PARAM = 1, 2, 4, 8, 16, 32
 BF16, F32 = 0, 1
 
 EXPORTS = ("spx_workspace_size", "spx_verify_attention", "spx_rejection_sample", "spx_verify_step",
@@ -39,6 +39,7 @@ class SampleArgs(C.Structure):
         ("target_logits", C.c_void_p), ("draft_logits", C.c_void_p), ("draft_token_ids", C.c_void_p),
         ("q_indptr", C.c_void_p), ("u_accept", C.c_void_p), ("u_sample", C.c_void_p),
         ("accepted_len", C.c_void_p), ("out_tokens", C.c_void_p), ("diag_ratio", C.c_void_p),
+        ("temperature", C.c_void_p),
     ]
 
 
@@ -154,7 +155,7 @@ def make_attn_args(q, k_cache, v_cache, kv_strides, block_table, seq_lens, q_ind
 
 
 def make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, accepted_len,
-                     out_tokens, diag_ratio=None, vocab=None) -> SampleArgs:
+                     out_tokens, diag_ratio=None, vocab=None, temperature=None) -> SampleArgs:
     s = SampleArgs()
     s.batch = q_indptr.numel() - 1
     s.total_q = target_logits.shape[0]
@@ -165,6 +166,7 @@ def make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept,
     s.draft_token_ids, s.q_indptr = _ptr(draft_ids), q_indptr.data_ptr()
     s.u_accept, s.u_sample = _ptr(u_accept), _ptr(u_sample)
     s.accepted_len, s.out_tokens, s.diag_ratio = _ptr(accepted_len), _ptr(out_tokens), _ptr(diag_ratio)
+    s.temperature = _ptr(temperature)
     return s
 
 
@@ -215,9 +217,12 @@ def verify_attention(q, k_cache, v_cache, kv_strides, block_table, seq_lens, q_i
 
 
 def rejection_sample(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, vocab=None,
-                     want_ratio=False, ws: Optional[Workspace] = None):
-    """spx_rejection_sample on the current stream.  Returns (accepted_len, out_tokens, ratio, ws)."""
+                     want_ratio=False, ws: Optional[Workspace] = None, temperature=None):
+    """spx_rejection_sample on the current stream.  Returns (accepted_len, out_tokens, ratio, ws).
+    ``temperature`` ([B] float32 on the device, optional) selects the verification variant per request."""
     _require_cuda(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample)
+    if temperature is not None:
+        _require_cuda(temperature)
     lib = load_library()
     dev = target_logits.device
     B = q_indptr.numel() - 1
@@ -226,7 +231,7 @@ def rejection_sample(target_logits, draft_logits, draft_ids, q_indptr, u_accept,
     tokens = torch.empty(TQ, dtype=torch.int32, device=dev)
     ratio = torch.empty(TQ - B, dtype=torch.float32, device=dev) if want_ratio else None
     s = make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, accepted, tokens,
-                         ratio, vocab)
+                         ratio, vocab, temperature)
     need = workspace_size(None, s)
     if ws is None:
         ws = Workspace.allocate(need, dev)

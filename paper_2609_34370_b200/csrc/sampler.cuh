@@ -41,46 +41,49 @@ struct SampleParams {
   float4 *req_norm;    // [B]  (Mt, 1/St, Md, 1/Sd) of row n, log2 domain maxima; Md = NaN => bonus
   int32_t *req_done;   // [B]  segments of row n finished (zeroed by accept_kernel)
   int32_t *dev_status;
+  // verification variants (both NULL: temperature 1 everywhere)
+  const float *temperature;  // [B]  > 0: sample at that temperature; 0: greedy
+  float *row_scale;          // [(TQ+TD)] workspace: log2(e)/tau of the row's request; 0 = row not needed
 };
 
 // 16-byte vector of logits -> floats, scaled into the log2 domain
 template <typename T> struct Vec;
 template <> struct Vec<__nv_bfloat16> {
   static constexpr int N = 8;
-  __device__ static __forceinline__ void load(const __nv_bfloat16 *p, float (&f)[8]) {
+  __device__ static __forceinline__ void load(const __nv_bfloat16 *p, float (&f)[8], float c) {
     const uint4 u = __ldg(reinterpret_cast<const uint4 *>(p));
     const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      f[2 * i] = __uint_as_float(w[i] << 16) * kLog2e;
-      f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u) * kLog2e;
+      f[2 * i] = __uint_as_float(w[i] << 16) * c;
+      f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u) * c;
     }
   }
 };
 template <> struct Vec<float> {
   static constexpr int N = 4;
-  __device__ static __forceinline__ void load(const float *p, float (&f)[4]) {
+  __device__ static __forceinline__ void load(const float *p, float (&f)[4], float c) {
     const float4 u = __ldg(reinterpret_cast<const float4 *>(p));
-    f[0] = u.x * kLog2e; f[1] = u.y * kLog2e; f[2] = u.z * kLog2e; f[3] = u.w * kLog2e;
+    f[0] = u.x * c; f[1] = u.y * c; f[2] = u.z * c; f[3] = u.w * c;
   }
 };
 
 // Load the kElemsPerThread consecutive tokens [v0, v0+32) of a row that this thread owns into
-// x[] (log2 domain); tokens >= vocab become -inf.
+// x[] (log2 domain: logit * scale, scale = log2(e) / temperature); tokens >= vocab become -inf.
 template <typename T>
-__device__ __forceinline__ void load_thread_span(const T *row, int v0, int vocab, float (&x)[kElemsPerThread]) {
+__device__ __forceinline__ void load_thread_span(const T *row, int v0, int vocab, float (&x)[kElemsPerThread], float scale) {
   constexpr int N = Vec<T>::N;
 #pragma unroll
   for (int c = 0; c < kElemsPerThread / N; ++c) {
     const int v = v0 + c * N;
     if (v + N <= vocab) {
       float f[N];
-      Vec<T>::load(row + v, f);
+      Vec<T>::load(row + v, f, scale);
 #pragma unroll
       for (int i = 0; i < N; ++i) x[c * N + i] = f[i];
     } else {
 #pragma unroll
-      for (int i = 0; i < N; ++i) x[c * N + i] = (v + i < vocab) ? ld_as_float(row, v + i) * kLog2e : -INFINITY;
+      for (int i = 0; i < N; ++i) x[c * N + i] = (v + i < vocab) ? ld_as_float(row, v + i) * scale : -INFINITY;
     }
   }
 }
@@ -123,7 +126,7 @@ struct SubSlice {
 // thread-local (max, sum 2^(x*log2e - max)) of a slice; the maximum is returned in the log2 domain.
 // Four independent maxima and four independent partial sums keep the dependency chains short
 // (the reduction order is fixed, so results do not depend on scheduling).
-__device__ __forceinline__ void slice_stats(const SubSlice<__nv_bfloat16> &sl, float &m, float &s) {
+__device__ __forceinline__ void slice_stats(const SubSlice<__nv_bfloat16> &sl, float &m, float &s, float scale) {
   constexpr int NV = SubSlice<__nv_bfloat16>::NV;
   // packed bf16 maximum: one instruction per two tokens
   __nv_bfloat162 mx[4];
@@ -136,7 +139,7 @@ __device__ __forceinline__ void slice_stats(const SubSlice<__nv_bfloat16> &sl, f
     for (int i = 0; i < 4; ++i) mx[i] = __hmax2(mx[i], *reinterpret_cast<const __nv_bfloat162 *>(&w[i]));
   }
   const __nv_bfloat162 mm = __hmax2(__hmax2(mx[0], mx[1]), __hmax2(mx[2], mx[3]));
-  m = fmaxf(__low2float(mm), __high2float(mm)) * kLog2e;
+  m = fmaxf(__low2float(mm), __high2float(mm)) * scale;
   s = 0.f;
   if (m == -INFINITY) return;
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -145,28 +148,28 @@ __device__ __forceinline__ void slice_stats(const SubSlice<__nv_bfloat16> &sl, f
     const uint32_t w[4] = {sl.raw[c].x, sl.raw[c].y, sl.raw[c].z, sl.raw[c].w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      acc[i] += fast_exp2(fmaf(__uint_as_float(w[i] << 16), kLog2e, -m));
-      acc[i] += fast_exp2(fmaf(__uint_as_float(w[i] & 0xffff0000u), kLog2e, -m));
+      acc[i] += fast_exp2(fmaf(__uint_as_float(w[i] << 16), scale, -m));
+      acc[i] += fast_exp2(fmaf(__uint_as_float(w[i] & 0xffff0000u), scale, -m));
     }
   }
   s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
 }
-__device__ __forceinline__ void slice_stats(const SubSlice<float> &sl, float &m, float &s) {
+__device__ __forceinline__ void slice_stats(const SubSlice<float> &sl, float &m, float &s, float scale) {
   constexpr int NV = SubSlice<float>::NV;
   float mx = -INFINITY;
 #pragma unroll
   for (int c = 0; c < NV; ++c)
     mx = fmaxf(fmaxf(mx, fmaxf(__uint_as_float(sl.raw[c].x), __uint_as_float(sl.raw[c].y))),
                fmaxf(__uint_as_float(sl.raw[c].z), __uint_as_float(sl.raw[c].w)));
-  m = mx * kLog2e;
+  m = mx * scale;
   s = 0.f;
   if (m == -INFINITY) return;
 #pragma unroll
   for (int c = 0; c < NV; ++c) {
-    s += fast_exp2(fmaf(__uint_as_float(sl.raw[c].x), kLog2e, -m));
-    s += fast_exp2(fmaf(__uint_as_float(sl.raw[c].y), kLog2e, -m));
-    s += fast_exp2(fmaf(__uint_as_float(sl.raw[c].z), kLog2e, -m));
-    s += fast_exp2(fmaf(__uint_as_float(sl.raw[c].w), kLog2e, -m));
+    s += fast_exp2(fmaf(__uint_as_float(sl.raw[c].x), scale, -m));
+    s += fast_exp2(fmaf(__uint_as_float(sl.raw[c].y), scale, -m));
+    s += fast_exp2(fmaf(__uint_as_float(sl.raw[c].z), scale, -m));
+    s += fast_exp2(fmaf(__uint_as_float(sl.raw[c].w), scale, -m));
   }
 }
 
@@ -174,7 +177,7 @@ __device__ __forceinline__ void slice_stats(const SubSlice<float> &sl, float &m,
 // (Skipping the rows after a request's first rejection inside this pass was tried - rows walked
 // position-major, completion counters, a steering accept test - and measured slower: the
 // bookkeeping cost more than the 22 % of bytes it saved.)
-template <typename T>
+template <typename T, bool kScaled>
 __global__ void __launch_bounds__(kSampThreads) row_stats_kernel(SampleParams p, int n_units) {
   const int lane = threadIdx.x & 31;
   const int warp_global = (blockIdx.x * kSampThreads + threadIdx.x) >> 5;
@@ -184,20 +187,33 @@ __global__ void __launch_bounds__(kSampThreads) row_stats_kernel(SampleParams p,
     return (row < p.total_q) ? reinterpret_cast<const T *>(p.target) + (int64_t)row * p.row_stride
                              : reinterpret_cast<const T *>(p.draft) + (int64_t)(row - p.total_q) * p.row_stride;
   };
+  // per-row scale of the variants; a scale of 0 marks a row nobody will read (draft rows of greedy
+  // requests, rows of requests with an invalid temperature)
+  auto row_scale = [&](int u) -> float { return kScaled ? p.row_scale[u / p.nsub] : kLog2e; };
   SubSlice<T> cur, nxt;
   int u = warp_global;
-  if (u < n_units) cur.issue(row_base(u), u % p.nsub, p.vocab, lane);
+  float sc_cur = kLog2e, sc_nxt = kLog2e;
+  if (u < n_units) {
+    sc_cur = row_scale(u);
+    if (sc_cur != 0.f) cur.issue(row_base(u), u % p.nsub, p.vocab, lane);
+  }
   for (; u < n_units; u += n_warps) {
     const int un = u + n_warps;
-    if (un < n_units) nxt.issue(row_base(un), un % p.nsub, p.vocab, lane);
-    float m, s;
-    slice_stats(cur, m, s);
-    // warp merge: one exponential per lane (rescale to the warp maximum), then a plain sum
-    const float M = warp_max(m);
-    if (M > -INFINITY) s *= fast_exp2(m - M);
-    const float S = warp_sum(s);
-    if (lane == 0) p.seg_stats[u] = make_float2(M, S);
+    if (un < n_units) {
+      sc_nxt = row_scale(un);
+      if (sc_nxt != 0.f) nxt.issue(row_base(un), un % p.nsub, p.vocab, lane);
+    }
+    if (sc_cur != 0.f) {
+      float m, s;
+      slice_stats(cur, m, s, sc_cur);
+      // warp merge: one exponential per lane (rescale to the warp maximum), then a plain sum
+      const float M = warp_max(m);
+      if (M > -INFINITY) s *= fast_exp2(m - M);
+      const float S = warp_sum(s);
+      if (lane == 0) p.seg_stats[u] = make_float2(M, S);
+    }
     cur = nxt;
+    sc_cur = sc_nxt;
   }
 }
 
@@ -236,6 +252,7 @@ __device__ __forceinline__ bool ring_wait(uint64_t *bar, uint32_t parity, volati
   }
 }
 
+template <bool kScaled>
 __global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleParams p, int chunks_per_row, int n_chunks) {
   extern __shared__ __align__(1024) unsigned char ring_smem[];
   unsigned char *stages = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(ring_smem) + 1023) & ~uintptr_t(1023));
@@ -273,6 +290,11 @@ __global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleP
         const int elems = min(kRingStageElems, p.vocab - e0);
         const uint32_t bytes = (uint32_t)((elems * 2 + 15) & ~15);  // stays inside the row: its stride is a multiple of 16 bytes
         const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&full[s]);
+        if (kScaled && p.row_scale[row] == 0.f) {
+          // a row nobody will read: hand the stage over empty, the consumers release it at once
+          asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+          continue;
+        }
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                      ::"r"((uint32_t)__cvta_generic_to_shared(stages + (size_t)s * kRingStageElems * 2)), "l"(src), "r"(bytes), "r"(bar)
@@ -292,7 +314,8 @@ __global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleP
       int row, e0;
       chunk_src(g, row, e0);
       const int v_sub = e0 + wsub * kSubElems;  // first token of this warp's sub-segment
-      if (v_sub < p.vocab) {
+      const float scale = kScaled ? p.row_scale[row] : kLog2e;
+      if (v_sub < p.vocab && scale != 0.f) {
         SubSlice<__nv_bfloat16> sl;
         const uint4 *src = reinterpret_cast<const uint4 *>(stages + (size_t)s * kRingStageElems * 2 + (size_t)wsub * kSubElems * 2);
 #pragma unroll
@@ -314,7 +337,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleP
         __syncwarp();
         if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"((uint32_t)__cvta_generic_to_shared(&empty[s])) : "memory");
         float m, sum;
-        slice_stats(sl, m, sum);
+        slice_stats(sl, m, sum, scale);
         const float M = warp_max(m);
         if (M > -INFINITY) sum *= fast_exp2(m - M);
         const float S = warp_sum(sum);
@@ -327,11 +350,103 @@ __global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleP
   }
 }
 
+// Verification variants, step 0: the scale log2(e)/tau of every logits row.  One thread per request.
+// Greedy requests (tau = 0) need only the maxima of their target rows (scale log2(e)); their draft
+// rows, and every row of a request whose temperature is not one, are marked 0 = skip.
+__global__ void row_scale_kernel(SampleParams p) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= p.batch) return;
+  const int t0 = p.q_indptr[r];
+  const int k = p.q_indptr[r + 1] - t0 - 1;
+  if (k < 0 || k > SPX_MAX_K || t0 < 0 || t0 + k + 1 > p.total_q) return;  // reported by accept_kernel
+  const float tau = p.temperature[r];
+  const bool valid = tau >= 0.f && tau != INFINITY;
+  const float st = !valid ? 0.f : (tau == 0.f ? kLog2e : kLog2e / tau);
+  const float sd = (valid && tau > 0.f) ? st : 0.f;
+  for (int i = 0; i <= k; ++i) p.row_scale[t0 + i] = st;
+  for (int i = 0; i < k; ++i) p.row_scale[p.total_q + t0 - r + i] = sd;
+}
+
+// Greedy verification (tau = 0): one block per request, warp i finds the greedy choice of target
+// row i - the lowest token id that attains the row maximum, compared on the stored values - from
+// the sub-segment maxima of the statistics pass (scaling is monotone, so the row maximum lies in a
+// sub-segment whose scaled maximum equals the row's) and one scan of those sub-segments.  Thread 0
+// then accepts drafts while they equal the greedy choice and emits the choice of row n.
+template <typename T>
+__global__ void __launch_bounds__(32 * (SPX_MAX_K + 1)) greedy_kernel(SampleParams p) {
+  const int r = blockIdx.x;
+  if (!(p.temperature[r] == 0.f)) return;
+  const int t0 = p.q_indptr[r];
+  const int k = p.q_indptr[r + 1] - t0 - 1;
+  if (k < 0 || k > SPX_MAX_K || t0 < 0 || t0 + k + 1 > p.total_q) return;  // reported by accept_kernel
+  const int d0 = t0 - r;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __shared__ int s_arg[SPX_MAX_K + 1];
+  __shared__ int s_bad;
+  if (threadIdx.x == 0) s_bad = 0;
+  __syncthreads();
+  if (threadIdx.x < k) {
+    const int x = p.draft_ids[d0 + threadIdx.x];
+    if (x < 0 || x >= p.vocab) s_bad = 1;
+  }
+  __syncthreads();
+  if (s_bad) return;  // reported by accept_kernel, which also wrote the outputs
+  if (warp <= k) {
+    constexpr int N = Vec<T>::N;
+    const float2 *st = p.seg_stats + (int64_t)(t0 + warp) * p.nsub;
+    const T *row = reinterpret_cast<const T *>(p.target) + (int64_t)(t0 + warp) * p.row_stride;
+    float M = -INFINITY;
+    for (int j = lane; j < p.nsub; j += 32) M = fmaxf(M, st[j].x);
+    M = warp_max(M);
+    float best = -INFINITY;
+    int best_i = 0x7fffffff;
+    auto consider = [&](float v, int i) {
+      if (v > best || (v == best && i < best_i)) { best = v; best_i = i; }
+    };
+    for (int j0 = 0; j0 < p.nsub; j0 += 32) {
+      const int j = j0 + lane;
+      uint32_t cand = __ballot_sync(0xffffffffu, j < p.nsub && st[j].x == M);
+      while (cand) {
+        const int sub = j0 + __ffs(cand) - 1;
+        cand &= cand - 1;
+        for (int c = 0; c < kSubElems / 32 / N; ++c) {
+          const int v = sub * kSubElems + (c * 32 + lane) * N;
+          if (v + N <= p.vocab) {
+            union { uint4 u; T e[N]; } tmp;
+            tmp.u = __ldg(reinterpret_cast<const uint4 *>(row + v));
+#pragma unroll
+            for (int i = 0; i < N; ++i) consider(ld_as_float(tmp.e, i), v + i);
+          } else {
+            for (int i = 0; i < N && v + i < p.vocab; ++i) consider(ld_as_float(row, v + i), v + i);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+      consider(ov, oi);
+    }
+    if (lane == 0) s_arg[warp] = best_i;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int n = k;
+    for (int i = 0; i < k; ++i)
+      if (p.draft_ids[d0 + i] != s_arg[i]) { n = i; break; }
+    p.accepted_len[r] = n;
+    for (int i = 0; i < n; ++i) p.out_tokens[t0 + i] = s_arg[i];
+    p.out_tokens[t0 + n] = s_arg[n] == 0x7fffffff ? -1 : s_arg[n];
+    for (int i = n + 1; i <= k; ++i) p.out_tokens[t0 + i] = -1;
+  }
+}
+
 // One warp per request, lane = row (lanes 0..k: target rows, lanes k+1..2k: draft rows).  Each lane
 // merges its row's segment pairs (fp32 exponentials, float64 sum); the accept ratios of all
 // drafts are evaluated in parallel in float64 and the first failure fixes n.  Writes
 // accepted_len, the accepted ids and the -1 padding; slot n is left for resid_select_kernel.
-template <typename T>
+template <typename T, bool kScaled>
 __global__ void __launch_bounds__(128) accept_kernel(SampleParams p) {
   const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
@@ -367,6 +482,24 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p) {
     if (lane <= k) p.out_tokens[t0 + lane] = -1;
     return;
   }
+  double scale = (double)kLog2e;
+  if (kScaled) {
+    const float tau = p.temperature[r];
+    if (!(tau >= 0.f) || tau == INFINITY) {
+      if (lane == 0) {
+        atomicOr(p.dev_status, SPX_DEV_BAD_PARAM);
+        p.accepted_len[r] = 0;
+        p.req_norm[r] = make_float4(nanf_, nanf_, nanf_, -1.f);
+      }
+      if (lane <= k) p.out_tokens[t0 + lane] = -1;
+      return;
+    }
+    if (tau == 0.f) {  // greedy: decided by greedy_kernel, nothing for the residual pass
+      if (lane == 0) p.req_norm[r] = make_float4(nanf_, nanf_, nanf_, -1.f);
+      return;
+    }
+    scale = (double)p.row_scale[t0];
+  }
   // row normalisers: M (log2 domain) and S = sum 2^(x - M)
   float M = -INFINITY;
   double S = 0.0;
@@ -381,8 +514,14 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p) {
   const double Sd = __shfl_sync(0xffffffffu, S, (k + 1 + lane) & 31);
   bool reject = false;
   if (lane < k) {
-    const double tx = (double)(ld_as_float(target, (int64_t)(t0 + lane) * p.row_stride + x) * kLog2e);
-    const double dx = (double)(ld_as_float(draft, (int64_t)(d0 + lane) * p.row_stride + x) * kLog2e);
+    double tx, dx;
+    if (kScaled) {
+      tx = (double)ld_as_float(target, (int64_t)(t0 + lane) * p.row_stride + x) * scale;
+      dx = (double)ld_as_float(draft, (int64_t)(d0 + lane) * p.row_stride + x) * scale;
+    } else {
+      tx = (double)(ld_as_float(target, (int64_t)(t0 + lane) * p.row_stride + x) * kLog2e);
+      dx = (double)(ld_as_float(draft, (int64_t)(d0 + lane) * p.row_stride + x) * kLog2e);
+    }
     // rho = p(x)/q(x) = 2^(tx-Mt)/St * Sd/2^(dx-Md)
     const double rho = exp2((tx - (double)M) - (dx - (double)Md)) * (Sd / S);
     reject = !((double)p.u_accept[d0 + lane] < rho);
@@ -409,14 +548,20 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p) {
 // last (bonus requests need no residual pass: their block 0 draws at once).  grid = (nseg, B).
 // Segment choice in float64 over the segment masses, token choice by an fp32 scan of the chosen
 // segment (thread t owns tokens [32t, 32t+32) of it).
-template <typename T>
+template <typename T, bool kScaled>
 __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams p) {
   const int seg_mine = blockIdx.x, r = blockIdx.y;
   const float4 nm = p.req_norm[r];
-  if (nm.w < 0.f) return;  // invalid request
+  if (nm.w < 0.f) return;  // invalid request, or one that another kernel decides (greedy)
   const bool bonus = (nm.z != nm.z);
   if (bonus && seg_mine != 0) return;
   const int t0 = p.q_indptr[r];
+  // the variants keep the stored logit and scale it inside one fused multiply-add with the
+  // maximum (a separately rounded product would cost |x * scale| * 2^-24 of relative accuracy,
+  // which matters at low temperature); the base rule scales at load time
+  const float scale = kScaled ? p.row_scale[t0] : kLog2e;
+  const float load_scale = kScaled ? 1.f : kLog2e;
+  auto ex = [&](float x, float M) -> float { return kScaled ? fast_exp2(fmaf(x, scale, -M)) : fast_exp2(x - M); };
   const int n = p.accepted_len[r];
   const T *trow = reinterpret_cast<const T *>(p.target) + (int64_t)(t0 + n) * p.row_stride;
   const T *drow = reinterpret_cast<const T *>(p.draft) + (int64_t)(t0 - r + n) * p.row_stride;
@@ -426,12 +571,12 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
   if (!bonus) {
     const int v0 = seg_mine * kSegElems + threadIdx.x * kElemsPerThread;
     float xt[kElemsPerThread], xd[kElemsPerThread];
-    load_thread_span(trow, v0, p.vocab, xt);
-    load_thread_span(drow, v0, p.vocab, xd);
+    load_thread_span(trow, v0, p.vocab, xt, load_scale);
+    load_thread_span(drow, v0, p.vocab, xd, load_scale);
     float acc = 0.f;
 #pragma unroll
     for (int i = 0; i < kElemsPerThread; ++i)
-      acc += fmaxf(0.f, fast_exp2(xt[i] - nm.x) * nm.y - fast_exp2(xd[i] - nm.z) * nm.w);
+      acc += fmaxf(0.f, ex(xt[i], nm.x) * nm.y - ex(xd[i], nm.z) * nm.w);
     acc = warp_sum(acc);
     if (lane == 0) s_w[warp] = acc;
     __syncthreads();
@@ -503,16 +648,16 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
   float w[kElemsPerThread];
   {
     float xt[kElemsPerThread];
-    load_thread_span(trow, v0, p.vocab, xt);
+    load_thread_span(trow, v0, p.vocab, xt, load_scale);
     if (use_target) {
 #pragma unroll
-      for (int i = 0; i < kElemsPerThread; ++i) w[i] = fast_exp2(xt[i] - nm.x) * nm.y;
+      for (int i = 0; i < kElemsPerThread; ++i) w[i] = ex(xt[i], nm.x) * nm.y;
     } else {
       float xd[kElemsPerThread];
-      load_thread_span(drow, v0, p.vocab, xd);
+      load_thread_span(drow, v0, p.vocab, xd, load_scale);
 #pragma unroll
       for (int i = 0; i < kElemsPerThread; ++i)
-        w[i] = fmaxf(0.f, fast_exp2(xt[i] - nm.x) * nm.y - fast_exp2(xd[i] - nm.z) * nm.w);
+        w[i] = fmaxf(0.f, ex(xt[i], nm.x) * nm.y - ex(xd[i], nm.z) * nm.w);
     }
   }
   float tsum = 0.f;

@@ -118,7 +118,7 @@ static AttnWs attn_ws_layout(const spx_attn_args_t *a) {
 }
 
 struct SampleWs {
-  size_t seg_stats, seg_resid, req_norm, req_done, total;
+  size_t seg_stats, seg_resid, req_norm, req_done, row_scale, total;
   int32_t nseg, nsub;
 };
 
@@ -148,6 +148,8 @@ static SampleWs sample_ws_layout(const spx_sample_args_t *s) {
   w.seg_resid = off; off = align_up(off + sizeof(float) * (size_t)s->batch * w.nseg, 256);
   w.req_norm = off; off = align_up(off + sizeof(float4) * (size_t)s->batch, 256);
   w.req_done = off; off = align_up(off + sizeof(int32_t) * (size_t)s->batch, 256);
+  w.row_scale = off;
+  if (s->temperature) off = align_up(off + sizeof(float) * rows, 256);
   w.total = off;
   return w;
 }
@@ -337,33 +339,44 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
   return e == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
 }
 
-template <typename T>
+template <typename T, bool kScaled>
 static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream, int num_sms, int phases) {
   const int rows = p.total_q + p.total_d;
   const int n_units = rows * p.nsub;
   int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_stats_kernel<T>, kSampThreads, 0) != cudaSuccess) return SPX_ERR_CUDA;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_stats_kernel<T, kScaled>, kSampThreads, 0) != cudaSuccess)
+    return SPX_ERR_CUDA;
   if (per_sm < 1) per_sm = 1;
   int grid = num_sms * per_sm;
   const int max_grid = (n_units + kSampThreads / 32 - 1) / (kSampThreads / 32);
   if (grid > max_grid) grid = max_grid;
   if (phases & kPhaseStats) {
+    if constexpr (kScaled) {
+      row_scale_kernel<<<(p.batch + 127) / 128, 128, 0, stream>>>(p);
+      ++t_launches;
+    }
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
       // bf16 logits: the bulk-copy ring kernel, one CTA per SM
       static_assert(kSubElems == 2048, "the ring kernel reduces 2048-token sub-segments");
-      if (cudaFuncSetAttribute(row_stats_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmemBytes) != cudaSuccess)
+      if (cudaFuncSetAttribute(row_stats_ring_kernel<kScaled>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmemBytes) !=
+          cudaSuccess)
         return SPX_ERR_CUDA;
       const int chunks_per_row = (p.vocab + kRingStageElems - 1) / kRingStageElems;
       const int n_chunks = rows * chunks_per_row;
-      row_stats_ring_kernel<<<num_sms < n_chunks ? num_sms : n_chunks, kRingThreads, kRingSmemBytes, stream>>>(p, chunks_per_row, n_chunks);
+      row_stats_ring_kernel<kScaled><<<num_sms < n_chunks ? num_sms : n_chunks, kRingThreads, kRingSmemBytes, stream>>>(
+          p, chunks_per_row, n_chunks);
     } else {
-      row_stats_kernel<T><<<grid, kSampThreads, 0, stream>>>(p, n_units);
+      row_stats_kernel<T, kScaled><<<grid, kSampThreads, 0, stream>>>(p, n_units);
     }
     ++t_launches;
   }
   if (phases & kPhaseTail) {
-    accept_kernel<T><<<(p.batch * 32 + 127) / 128, 128, 0, stream>>>(p);
-    resid_select_kernel<T><<<dim3(p.nseg, p.batch), kSampThreads, 0, stream>>>(p);
+    accept_kernel<T, kScaled><<<(p.batch * 32 + 127) / 128, 128, 0, stream>>>(p);
+    if constexpr (kScaled) {
+      greedy_kernel<T><<<p.batch, 32 * (SPX_MAX_K + 1), 0, stream>>>(p);
+      ++t_launches;
+    }
+    resid_select_kernel<T, kScaled><<<dim3(p.nseg, p.batch), kSampThreads, 0, stream>>>(p);
     t_launches += 2;
   }
   return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
@@ -386,7 +399,14 @@ static spx_status_t launch_sampler(const spx_sample_args_t *s, unsigned char *ws
   p.req_norm = reinterpret_cast<float4 *>(ws + w.req_norm);
   p.req_done = reinterpret_cast<int32_t *>(ws + w.req_done);
   p.dev_status = dev_status;
-  return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16>(p, stream, num_sms, phases) : launch_sampler_t<float>(p, stream, num_sms, phases);
+  if (s->temperature) {
+    p.temperature = s->temperature;
+    p.row_scale = reinterpret_cast<float *>(ws + w.row_scale);
+    return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16, true>(p, stream, num_sms, phases)
+                                       : launch_sampler_t<float, true>(p, stream, num_sms, phases);
+  }
+  return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16, false>(p, stream, num_sms, phases)
+                                     : launch_sampler_t<float, false>(p, stream, num_sms, phases);
 }
 
 static spx_status_t check_ws(const void *ws, size_t ws_bytes, size_t need, const int32_t *dev_status) {
@@ -479,7 +499,7 @@ spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_
 // ---- host-buffer convenience ---------------------------------------------------------------
 namespace {
 struct HostStepLayout {
-  size_t q, k, v, bt, sl, qi, out, lse, tl, dl, ids, ua, us, acc, tok, status, ws, total;
+  size_t q, k, v, bt, sl, qi, out, lse, tl, dl, ids, ua, us, tau, acc, tok, status, ws, total;
   size_t q_bytes, kv_bytes, bt_bytes, out_bytes, lse_bytes, tl_bytes, dl_bytes, ws_bytes;
 };
 HostStepLayout host_layout(const spx_attn_args_t *a, const spx_sample_args_t *s, int64_t kv_pool_elems) {
@@ -499,6 +519,7 @@ HostStepLayout host_layout(const spx_attn_args_t *a, const spx_sample_args_t *s,
   L.q = take(L.q_bytes); L.k = take(L.kv_bytes); L.v = take(L.kv_bytes); L.bt = take(L.bt_bytes);
   L.sl = take(B * 4); L.qi = take((B + 1) * 4); L.out = take(L.out_bytes); L.lse = take(L.lse_bytes);
   L.tl = take(L.tl_bytes); L.dl = take(L.dl_bytes); L.ids = take(TD * 4); L.ua = take(TD * 4); L.us = take(B * 4);
+  L.tau = take(s->temperature ? B * 4 : 0);
   L.acc = take(B * 4); L.tok = take(TQ * 4); L.status = take(4); L.ws = take(L.ws_bytes);
   L.total = off;
   return L;
@@ -533,6 +554,7 @@ spx_status_t spx_verify_step_host(const spx_attn_args_t *attn, const spx_sample_
   h2d(L.bt, attn->block_table, L.bt_bytes); h2d(L.sl, attn->seq_lens, B * 4); h2d(L.qi, attn->q_indptr, (B + 1) * 4);
   h2d(L.tl, sample->target_logits, L.tl_bytes); h2d(L.dl, sample->draft_logits, L.dl_bytes);
   h2d(L.ids, sample->draft_token_ids, TD * 4); h2d(L.ua, sample->u_accept, TD * 4); h2d(L.us, sample->u_sample, B * 4);
+  h2d(L.tau, sample->temperature, B * 4);
   ok = ok && cudaMemsetAsync(d + L.status, 0, 4, stream) == cudaSuccess;
   if (!ok) return SPX_ERR_CUDA;
   spx_attn_args_t a = *attn;
@@ -545,6 +567,7 @@ spx_status_t spx_verify_step_host(const spx_attn_args_t *attn, const spx_sample_
   s.q_indptr = a.q_indptr; s.u_accept = reinterpret_cast<float *>(d + L.ua); s.u_sample = reinterpret_cast<float *>(d + L.us);
   s.accepted_len = reinterpret_cast<int32_t *>(d + L.acc); s.out_tokens = reinterpret_cast<int32_t *>(d + L.tok);
   s.diag_ratio = nullptr;
+  s.temperature = sample->temperature ? reinterpret_cast<float *>(d + L.tau) : nullptr;
   const spx_status_t st = spx_verify_step(&a, &s, d + L.ws, L.ws_bytes, reinterpret_cast<int32_t *>(d + L.status), cuda_stream);
   if (st != SPX_OK) return st;
   d2h(attn->out, L.out, L.out_bytes); d2h(attn->lse, L.lse, L.lse_bytes);

@@ -8,6 +8,13 @@ Tolerances (stated where they are used as well):
     draft has |p/q - u| < 1e-6 (accept-class near tie) or whose target s*R lies within 1e-6*R of
     the CDF interval of the token the GPU chose (cdf-class near tie, an fp32 scan cannot
     reproduce a float64 sequential cumulative sum bit for bit).  Both classes are counted.
+  * sampling at a temperature other than 1: the same, plus a third counted class.  At low
+    temperature p and q can both be within fp32 resolution of the same one-hot row, so the residual
+    max(0, p - q) is a difference of nearly equal fp32 numbers and its total mass R can fall below
+    what fp32 probabilities resolve at all (R ~ 1e-9 occurs at tau = 0.05).  A band relative to R is
+    then meaningless for an fp32 kernel; the class is stated in absolute probability mass instead:
+    the GPU's token is tolerated iff s*R lies within 2^-22 (four fp32 ulps of unit mass, the
+    resolution of p and q near 1) of the oracle's cumulative interval of that token.
 """
 from __future__ import annotations
 
@@ -25,6 +32,7 @@ ATTN_TOL = {
 }
 ACCEPT_BAND = 1e-6
 CDF_BAND = 1e-6
+CDF_ABS_BAND = 2.0 ** -22       # variants only: absolute probability mass
 
 
 def gpu_attention(b, ws=None, **kw):
@@ -74,15 +82,18 @@ class SampleReport:
     exact: int = 0
     accept_near_tie: int = 0
     cdf_near_tie: int = 0
+    cdf_abs_near_tie: int = 0           # requests at a temperature other than 1 only
     hard_mismatch: List[int] = field(default_factory=list)
     accept_band_eligible: int = 0       # consulted drafts inside the accept band (oracle side)
 
 
-def check_sampling(b_cpu, acc_gpu, tok_gpu, ref: Optional[oracle.SampleResult] = None) -> SampleReport:
-    """Bit-exactness of (accepted_len, out_tokens) outside the two counted near-tie classes."""
+def check_sampling(b_cpu, acc_gpu, tok_gpu, ref: Optional[oracle.SampleResult] = None,
+                   temperature: Optional[torch.Tensor] = None) -> SampleReport:
+    """Bit-exactness of (accepted_len, out_tokens) outside the two counted near-tie classes.
+    Greedy requests (temperature 0) have no near-tie class: they must match exactly."""
     if ref is None:
         ref = oracle.rejection_sample(b_cpu.target_logits, b_cpu.draft_logits, b_cpu.draft_ids, b_cpu.q_indptr,
-                                      b_cpu.u_accept, b_cpu.u_sample)
+                                      b_cpu.u_accept, b_cpu.u_sample, temperature=temperature)
     acc_gpu = acc_gpu.detach().cpu()
     tok_gpu = tok_gpu.detach().cpu()
     qi = b_cpu.q_indptr.tolist()
@@ -98,6 +109,10 @@ def check_sampling(b_cpu, acc_gpu, tok_gpu, ref: Optional[oracle.SampleResult] =
         if n_o == n_g and torch.equal(ref.out_tokens[t0:t1], tok_gpu[t0:t1]):
             rep.exact += 1
             continue
+        tau = 1.0 if temperature is None else float(temperature[r])
+        if not tau > 0.0:
+            rep.hard_mismatch.append(r)
+            continue
         upto = min(max(n_o, n_g), k - 1)
         if k > 0 and bool(near[d0:d0 + upto + 1].any()):
             rep.accept_near_tie += 1
@@ -106,12 +121,15 @@ def check_sampling(b_cpu, acc_gpu, tok_gpu, ref: Optional[oracle.SampleResult] =
                 bool((tok_gpu[t0 + n_o + 1:t1] == -1).all()):
             y_g = int(tok_gpu[t0 + n_o])
             if 0 <= y_g < b_cpu.spec.vocab:
-                cdf, R = oracle.emit_cdf(r, n_o, b_cpu.target_logits, b_cpu.draft_logits, b_cpu.q_indptr)
+                cdf, R = oracle.emit_cdf(r, n_o, b_cpu.target_logits, b_cpu.draft_logits, b_cpu.q_indptr, tau=tau)
                 target = float(b_cpu.u_sample[r]) * R
                 lo = float(cdf[y_g - 1]) if y_g > 0 else 0.0
                 hi = float(cdf[y_g])
                 if hi > lo and lo - CDF_BAND * R <= target <= hi + CDF_BAND * R:
                     rep.cdf_near_tie += 1
+                    continue
+                if tau != 1.0 and lo - CDF_ABS_BAND <= target <= hi + CDF_ABS_BAND:
+                    rep.cdf_abs_near_tie += 1
                     continue
         rep.hard_mismatch.append(r)
     return rep
