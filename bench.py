@@ -178,6 +178,59 @@ def run_reference(args):
     }))
 
 
+def time_extras(spx, binding, spec, b, attn_args, dev, iters: int = 200):
+    """Device time (CUDA events, mean of `iters` calls after 5 warm-up calls, L2 not flushed for the
+    small ones: they are launch-bound) of the calls around the step and of the verification variants."""
+    def timed(fn):
+        for _ in range(5):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters * 1e3      # microseconds
+
+    g = torch.Generator().manual_seed(spec.seed + 7)
+    shape = (b.total_q, spec.num_kv_heads, spec.head_dim)
+    new_k = torch.randn(shape, generator=g).to(b.q.dtype).to(dev)
+    new_v = torch.randn(shape, generator=g).to(b.q.dtype).to(dev)
+    k_pool, v_pool = b.k_cache.clone(), b.v_cache.clone()     # the benchmark's own pools stay untouched
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    acc = torch.empty(b.batch, dtype=torch.int32, device=dev)
+    tok = torch.empty(b.total_q, dtype=torch.int32, device=dev)
+    new_len = torch.empty_like(b.seq_lens)
+    out = {}
+    out["kv_append_us"] = timed(lambda: spx.kv_append(new_k, new_v, k_pool, v_pool, b.kv_strides, b.block_table, b.seq_lens,
+                                                      b.q_indptr, spec.page_size, b.num_pages, status=status))
+    out["kv_append_bytes"] = 2 * new_k.numel() * new_k.element_size() * 2
+    base = binding.make_sample_args(b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample, acc, tok)
+    ws = spx.Workspace.allocate(spx.workspace_size(attn_args, base), dev)
+    lib = spx.load_library()
+    import ctypes as C
+    stream = torch.cuda.current_stream(dev).cuda_stream
+
+    def sample_call(sargs):
+        return lambda: lib.spx_rejection_sample(C.byref(sargs), ws.buf.data_ptr(), ws.buf.numel(), ws.status.data_ptr(), stream)
+
+    out["sample_tau1_us"] = timed(sample_call(base))
+    out["kv_rollback_us"] = timed(lambda: spx.kv_rollback(b.seq_lens, b.q_indptr, acc, out=new_len, status=status))
+    taus = {"mixed": torch.tensor([[1.0, 0.0, 0.3, 0.7, 0.0, 1.5, 4.0, 0.05][r % 8] for r in range(b.batch)]),
+            "0.7": torch.full((b.batch,), 0.7), "greedy": torch.zeros(b.batch)}
+    for name, tau in taus.items():
+        tau_d = tau.to(dev)
+        sv = binding.make_sample_args(b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample,
+                                      acc, tok, None, None, tau_d)
+        ws.ensure(spx.workspace_size(attn_args, sv))
+        out[f"sample_tau_{name}_us"] = timed(sample_call(sv))
+        out[f"step_tau_{name}_us"] = timed(lambda: spx.verify_step(attn_args, sv, ws, dev))
+    if int(ws.status.item()) != 0 or int(status.item()) != 0:
+        out["status"] = [int(ws.status.item()), int(status.item())]
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -188,6 +241,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--extras", action="store_true",
+                    help="also time the pieces around the step: KV append / rollback, verification variants")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling captures of a smaller case)")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -277,6 +332,10 @@ def main():
     value = job_tokens * args.steps / (ms_total * 1e-3)
     ms_per_step = ms_total / args.steps
 
+    extras = None
+    if args.extras and rank == 0:
+        extras = time_extras(spx, binding, spec, b, a, dev)
+
     # ---- end to end through the host-buffer entry point (every rank, max time) ----
     b_host = None
     e2e = None
@@ -346,6 +405,8 @@ def main():
         "step_hbm": {"bytes": kv_bytes + logit_bytes, "achieved_gbs": step_gbs,
                      "frac_of_measured": step_gbs / peak, "frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS},
     }
+    if extras is not None:
+        result["extras"] = extras
     if not args.no_cpu_baseline:
         try:
             n_req = oracle_sample_size(spec)

@@ -282,7 +282,11 @@ __global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleP
     // ---- producer (one thread)
     if (lane == 0) {
       int i = 0;
+      // the scale of the next chunk's row is fetched one iteration ahead, off the issue path
+      float sc_next = (kScaled && (int)blockIdx.x < n_chunks) ? p.row_scale[blockIdx.x / chunks_per_row] : 1.f;
       for (int g = blockIdx.x; g < n_chunks; g += gridDim.x, ++i) {
+        const float sc = sc_next;
+        if (kScaled && g + (int)gridDim.x < n_chunks) sc_next = p.row_scale[(g + gridDim.x) / chunks_per_row];
         const int s = i % kRingStages;
         if (i >= kRingStages && !ring_wait(&empty[s], ((i / kRingStages) - 1) & 1, abort, p.dev_status)) break;
         int row, e0;
@@ -290,7 +294,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleP
         const int elems = min(kRingStageElems, p.vocab - e0);
         const uint32_t bytes = (uint32_t)((elems * 2 + 15) & ~15);  // stays inside the row: its stride is a multiple of 16 bytes
         const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&full[s]);
-        if (kScaled && p.row_scale[row] == 0.f) {
+        if (kScaled && sc == 0.f) {
           // a row nobody will read: hand the stage over empty, the consumers release it at once
           asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
           continue;
@@ -309,12 +313,12 @@ __global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleP
     int i = grp;
     for (int g = blockIdx.x + grp * gridDim.x; g < n_chunks; g += kRingGroups * gridDim.x, i += kRingGroups) {
       const int s = i % kRingStages;
-      const bool ok = __all_sync(0xffffffffu, ring_wait(&full[s], (i / kRingStages) & 1, abort, p.dev_status));
-      if (!ok) break;
       int row, e0;
       chunk_src(g, row, e0);
+      const float scale = kScaled ? p.row_scale[row] : kLog2e;  // in flight while the stage fills
+      const bool ok = __all_sync(0xffffffffu, ring_wait(&full[s], (i / kRingStages) & 1, abort, p.dev_status));
+      if (!ok) break;
       const int v_sub = e0 + wsub * kSubElems;  // first token of this warp's sub-segment
-      const float scale = kScaled ? p.row_scale[row] : kLog2e;
       if (v_sub < p.vocab && scale != 0.f) {
         SubSlice<__nv_bfloat16> sl;
         const uint4 *src = reinterpret_cast<const uint4 *>(stages + (size_t)s * kRingStageElems * 2 + (size_t)wsub * kSubElems * 2);
@@ -367,41 +371,41 @@ __global__ void row_scale_kernel(SampleParams p) {
   for (int i = 0; i < k; ++i) p.row_scale[p.total_q + t0 - r + i] = sd;
 }
 
-// Greedy verification (tau = 0): one block per request, warp i finds the greedy choice of target
-// row i - the lowest token id that attains the row maximum, compared on the stored values - from
-// the sub-segment maxima of the statistics pass (scaling is monotone, so the row maximum lies in a
-// sub-segment whose scaled maximum equals the row's) and one scan of those sub-segments.  Thread 0
-// then accepts drafts while they equal the greedy choice and emits the choice of row n.
+// Greedy verification (tau = 0) of one request by one block: a warp finds the greedy choice of a
+// target row - the lowest token id that attains the row maximum, compared on the stored values -
+// from the sub-segment maxima of the statistics pass (scaling is monotone, so the row maximum lies
+// in a sub-segment whose scaled maximum equals the row's) and one scan of those sub-segments.
+// Thread 0 then accepts drafts while they equal the greedy choice and emits the choice of row n.
+// Requests that are not greedy, or that the accept test reports as invalid, are left alone.
 template <typename T>
-__global__ void __launch_bounds__(32 * (SPX_MAX_K + 1)) greedy_kernel(SampleParams p) {
-  const int r = blockIdx.x;
+__device__ __forceinline__ void greedy_request(const SampleParams &p, int r) {
   if (!(p.temperature[r] == 0.f)) return;
   const int t0 = p.q_indptr[r];
   const int k = p.q_indptr[r + 1] - t0 - 1;
-  if (k < 0 || k > SPX_MAX_K || t0 < 0 || t0 + k + 1 > p.total_q) return;  // reported by accept_kernel
+  if (k < 0 || k > SPX_MAX_K || t0 < 0 || t0 + k + 1 > p.total_q) return;
   const int d0 = t0 - r;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   __shared__ int s_arg[SPX_MAX_K + 1];
   __shared__ int s_bad;
   if (threadIdx.x == 0) s_bad = 0;
   __syncthreads();
-  if (threadIdx.x < k) {
+  if ((int)threadIdx.x < k) {
     const int x = p.draft_ids[d0 + threadIdx.x];
     if (x < 0 || x >= p.vocab) s_bad = 1;
   }
   __syncthreads();
-  if (s_bad) return;  // reported by accept_kernel, which also wrote the outputs
-  if (warp <= k) {
+  if (s_bad) return;
+  for (int i = warp; i <= k; i += n_warps) {
     constexpr int N = Vec<T>::N;
-    const float2 *st = p.seg_stats + (int64_t)(t0 + warp) * p.nsub;
-    const T *row = reinterpret_cast<const T *>(p.target) + (int64_t)(t0 + warp) * p.row_stride;
+    const float2 *st = p.seg_stats + (int64_t)(t0 + i) * p.nsub;
+    const T *row = reinterpret_cast<const T *>(p.target) + (int64_t)(t0 + i) * p.row_stride;
     float M = -INFINITY;
     for (int j = lane; j < p.nsub; j += 32) M = fmaxf(M, st[j].x);
     M = warp_max(M);
     float best = -INFINITY;
     int best_i = 0x7fffffff;
-    auto consider = [&](float v, int i) {
-      if (v > best || (v == best && i < best_i)) { best = v; best_i = i; }
+    auto consider = [&](float v, int idx) {
+      if (v > best || (v == best && idx < best_i)) { best = v; best_i = idx; }
     };
     for (int j0 = 0; j0 < p.nsub; j0 += 32) {
       const int j = j0 + lane;
@@ -409,15 +413,16 @@ __global__ void __launch_bounds__(32 * (SPX_MAX_K + 1)) greedy_kernel(SamplePara
       while (cand) {
         const int sub = j0 + __ffs(cand) - 1;
         cand &= cand - 1;
+#pragma unroll
         for (int c = 0; c < kSubElems / 32 / N; ++c) {
           const int v = sub * kSubElems + (c * 32 + lane) * N;
           if (v + N <= p.vocab) {
             union { uint4 u; T e[N]; } tmp;
             tmp.u = __ldg(reinterpret_cast<const uint4 *>(row + v));
 #pragma unroll
-            for (int i = 0; i < N; ++i) consider(ld_as_float(tmp.e, i), v + i);
+            for (int e = 0; e < N; ++e) consider(ld_as_float(tmp.e, e), v + e);
           } else {
-            for (int i = 0; i < N && v + i < p.vocab; ++i) consider(ld_as_float(row, v + i), v + i);
+            for (int e = 0; e < N && v + e < p.vocab; ++e) consider(ld_as_float(row, v + e), v + e);
           }
         }
       }
@@ -428,7 +433,7 @@ __global__ void __launch_bounds__(32 * (SPX_MAX_K + 1)) greedy_kernel(SamplePara
       const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
       consider(ov, oi);
     }
-    if (lane == 0) s_arg[warp] = best_i;
+    if (lane == 0) s_arg[i] = best_i;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -447,7 +452,11 @@ __global__ void __launch_bounds__(32 * (SPX_MAX_K + 1)) greedy_kernel(SamplePara
 // drafts are evaluated in parallel in float64 and the first failure fixes n.  Writes
 // accepted_len, the accepted ids and the -1 padding; slot n is left for resid_select_kernel.
 template <typename T, bool kScaled>
-__global__ void __launch_bounds__(128) accept_kernel(SampleParams p) {
+__global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_blocks) {
+  if (kScaled && (int)blockIdx.x >= accept_blocks) {  // variants: one extra block per request for the greedy ones
+    greedy_request<T>(p, blockIdx.x - accept_blocks);
+    return;
+  }
   const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (r >= p.batch) return;
@@ -494,7 +503,7 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p) {
       if (lane <= k) p.out_tokens[t0 + lane] = -1;
       return;
     }
-    if (tau == 0.f) {  // greedy: decided by greedy_kernel, nothing for the residual pass
+    if (tau == 0.f) {  // greedy: decided by this launch's extra blocks, nothing for the residual pass
       if (lane == 0) p.req_norm[r] = make_float4(nanf_, nanf_, nanf_, -1.f);
       return;
     }
@@ -552,7 +561,7 @@ template <typename T, bool kScaled>
 __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams p) {
   const int seg_mine = blockIdx.x, r = blockIdx.y;
   const float4 nm = p.req_norm[r];
-  if (nm.w < 0.f) return;  // invalid request, or one that another kernel decides (greedy)
+  if (nm.w < 0.f) return;  // invalid request, or a greedy one (decided beside the accept test)
   const bool bonus = (nm.z != nm.z);
   if (bonus && seg_mine != 0) return;
   const int t0 = p.q_indptr[r];

@@ -371,11 +371,8 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
     ++t_launches;
   }
   if (phases & kPhaseTail) {
-    accept_kernel<T, kScaled><<<(p.batch * 32 + 127) / 128, 128, 0, stream>>>(p);
-    if constexpr (kScaled) {
-      greedy_kernel<T><<<p.batch, 32 * (SPX_MAX_K + 1), 0, stream>>>(p);
-      ++t_launches;
-    }
+    const int accept_blocks = (p.batch * 32 + 127) / 128;
+    accept_kernel<T, kScaled><<<accept_blocks + (kScaled ? p.batch : 0), 128, 0, stream>>>(p, accept_blocks);
     resid_select_kernel<T, kScaled><<<dim3(p.nseg, p.batch), kSampThreads, 0, stream>>>(p);
     t_launches += 2;
   }
