@@ -295,3 +295,42 @@ def kv_rollback(seq_lens: torch.Tensor, q_indptr: torch.Tensor, accepted_len: to
     if st != OK:
         raise OracleError(st)
     return out
+
+
+def draft_confidence(draft_logits: torch.Tensor, draft_ids: Optional[torch.Tensor], q_indptr: torch.Tensor,
+                     vocab: Optional[int] = None):
+    """Per-draft top-1 probability, probability of the drafted token (None without ids) and the
+    per-request product of the top-1 probabilities, all float64."""
+    lib = _load()
+    dl = _cpu(draft_logits)
+    qi = _cpu(q_indptr, torch.int32).contiguous()
+    B = qi.numel() - 1
+    TD = int(qi[-1]) - B
+    V = int(vocab if vocab is not None else dl.shape[1])
+    ids = _cpu(draft_ids, torch.int32).contiguous() if draft_ids is not None else None
+    cmax = torch.empty(TD, dtype=torch.float64)
+    ctok = torch.empty(TD, dtype=torch.float64) if ids is not None else None
+    creq = torch.empty(B, dtype=torch.float64)
+    lib.oracle_draft_confidence.restype = c.c_int
+    lib.oracle_draft_confidence.argtypes = [c.c_int32, c.c_int64, c.c_int64, c.c_int32] + [c.c_void_p] * 6
+    st = lib.oracle_draft_confidence(B, V, dl.stride(0) if dl.dim() == 2 and dl.numel() else V, _dtype_code(dl), _ptr(dl),
+                                     _ptr(ids), _ptr(qi), _ptr(cmax), _ptr(ctok), _ptr(creq))
+    if st not in (OK, ERR_TOKEN):
+        raise OracleError(st)
+    return cmax, ctok, creq
+
+
+def select_speculation(confidence: torch.Tensor, k_in: torch.Tensor, alpha: float):
+    """Keep-top-(1-alpha): returns (k_out [B] int32, n_drop)."""
+    lib = _load()
+    conf = _cpu(confidence, torch.float32).contiguous()
+    kin = _cpu(k_in, torch.int32).contiguous()
+    assert conf.numel() == kin.numel()
+    kout = torch.empty_like(kin)
+    nd = c.c_int32(0)
+    lib.oracle_select_speculation.restype = c.c_int
+    lib.oracle_select_speculation.argtypes = [c.c_int32, c.c_void_p, c.c_void_p, c.c_double, c.c_void_p, c.c_void_p]
+    st = lib.oracle_select_speculation(kin.numel(), _ptr(conf), _ptr(kin), float(alpha), _ptr(kout), c.byref(nd))
+    if st != OK:
+        raise OracleError(st)
+    return kout, int(nd.value)

@@ -38,7 +38,10 @@
  * this build's reading: the same temperature divides target and draft logits, temperature 0
  * verifies greedily) the output law against softmax(target / tau), the closed form
  * tau*ln(w) -> w / sum w, exact invariance under doubling logits and temperature together,
- * numpy's argmax on rows with ties, and the tau -> 0 limit meeting the greedy branch.
+ * numpy's argmax on rows with ties, and the tau -> 0 limit meeting the greedy branch; for the
+ * selective-speculation support (tests/test_oracle_select.py; Section 5.1) scipy's softmax
+ * maxima, the closed forms 1/V and w_max / sum w, numpy's lexsort on (confidence, -index),
+ * and the invariants of a keep-top-(1-alpha) selection (count, separation, alpha = 0 and 1).
  */
 #include <math.h>
 #include <stdint.h>
@@ -491,6 +494,94 @@ double oracle_emit_cdf(int32_t r, int32_t n, int64_t V, int64_t row_stride, int3
                        const void *target_logits, const void *draft_logits,
                        const int32_t *q_indptr, double *cdf) {
   return oracle_emit_cdf_tau(r, n, V, row_stride, dtype, target_logits, draft_logits, q_indptr, 1.0, cdf);
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* (E) selective speculation: draft confidence and the keep-top-(1-alpha) selection       */
+/* ------------------------------------------------------------------------------------ */
+
+/*
+ * Section 5.1 ranks drafted tokens by the draft's confidence and drops a fixed fraction alpha
+ * of the lowest-ranked ones; Section 7.4 states it per sequence ("rank the sequences in a batch
+ * by their speculation confidence and drop the lowest alpha fraction").  The paper does not
+ * define the confidence beyond citing the self-speculation works that use the draft's top
+ * probability, so this build reads it as:
+ *   conf_max[d]  = max_v softmax(D_d)(v)              (the draft's top-1 probability)
+ *   conf_tok[d]  = softmax(D_d)(x_d)                  (probability of the drafted token)
+ *   req_conf[r]  = prod_i conf_max[d0(r) + i]         (1 for k_r = 0; with one draft per
+ *                                                      sequence every reading coincides)
+ * Draft rows and ids are indexed as in the sampling half (row q_indptr[r] - r + i).
+ * conf_tok may be NULL; an id outside [0, V) gives conf_tok = NaN and ORACLE_ERR_TOKEN.
+ */
+int oracle_draft_confidence(int32_t batch, int64_t V, int64_t row_stride, int32_t dtype,
+                            const void *draft_logits, const int32_t *draft_ids,
+                            const int32_t *q_indptr, double *conf_max, double *conf_tok,
+                            double *req_conf) {
+  if (batch < 0 || V <= 0 || row_stride < V) return ORACLE_ERR_ARG;
+  if (dtype != ORACLE_BF16 && dtype != ORACLE_F32) return ORACLE_ERR_ARG;
+  int status = ORACLE_OK;
+  double *q = (double *)malloc(sizeof(double) * (size_t)V);
+  if (!q) return ORACLE_ERR_ALLOC;
+  for (int r = 0; r < batch; ++r) {
+    const int64_t d0 = (int64_t)q_indptr[r] - r;
+    const int k = q_indptr[r + 1] - q_indptr[r] - 1;
+    if (k < 0) { free(q); return ORACLE_ERR_ARG; }
+    double prod = 1.0;
+    for (int i = 0; i < k; ++i) {
+      oracle_softmax_row(draft_logits, dtype, (d0 + i) * row_stride, V, q);
+      double mx = 0.0;
+      for (int64_t v = 0; v < V; ++v) if (q[v] > mx) mx = q[v];
+      conf_max[d0 + i] = mx;
+      prod *= mx;
+      if (conf_tok) {
+        const int64_t x = draft_ids[d0 + i];
+        if (x < 0 || x >= V) { conf_tok[d0 + i] = NAN; status = ORACLE_ERR_TOKEN; }
+        else conf_tok[d0 + i] = q[x];
+      }
+    }
+    req_conf[r] = prod;
+  }
+  free(q);
+  return status;
+}
+
+/* Total order on fp32 bit patterns (-NaN < -inf < ... < -0 < +0 < ... < +inf < +NaN). */
+static uint32_t f32_order_key(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+/*
+ * Selection.  Among the requests that carry drafts (k_in[r] > 0; N of them) drop the
+ * n_drop = floor(alpha * N) with the lowest confidence; a dropped request continues without
+ * speculation (k_out = 0), the others keep k_out = k_in.  Order: the total order above on the
+ * stored fp32 confidences; among equal confidences the higher request index is dropped first.
+ * alpha outside [0, 1] (or NaN) is an argument error.  Returns n_drop through *n_drop_out.
+ * Written as the definition: repeatedly remove the lowest remaining participant.
+ */
+int oracle_select_speculation(int32_t batch, const float *confidence, const int32_t *k_in,
+                              double alpha, int32_t *k_out, int32_t *n_drop_out) {
+  if (batch < 0 || !(alpha >= 0.0 && alpha <= 1.0)) return ORACLE_ERR_ARG;
+  int64_t N = 0;
+  for (int r = 0; r < batch; ++r) {
+    if (k_in[r] < 0) return ORACLE_ERR_ARG;
+    k_out[r] = k_in[r];
+    if (k_in[r] > 0) ++N;
+  }
+  const int64_t n_drop = (int64_t)floor(alpha * (double)N);
+  for (int64_t d = 0; d < n_drop; ++d) {
+    int worst = -1;
+    for (int r = 0; r < batch; ++r) {
+      if (k_out[r] == 0) continue;   /* not a participant, or dropped already */
+      if (worst < 0) { worst = r; continue; }
+      /* r > worst here (ascending scan), so an equal confidence moves the choice to the higher index */
+      if (f32_order_key(confidence[r]) <= f32_order_key(confidence[worst])) worst = r;
+    }
+    k_out[worst] = 0;
+  }
+  if (n_drop_out) *n_drop_out = (int32_t)n_drop;
+  return ORACLE_OK;
 }
 
 /* ------------------------------------------------------------------------------------ */
