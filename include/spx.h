@@ -203,6 +203,47 @@ spx_status_t spx_kv_rollback(int32_t batch, const int32_t *seq_lens, const int32
                              void *cuda_stream);
 
 /*
+ * Selective speculation support (the paper's Section 5.1: drafted tokens are ranked by the
+ * draft's confidence and a fixed fraction alpha of the lowest-ranked is not speculated on;
+ * Section 7.4 applies it per sequence).  The paper does not define the confidence further; this
+ * library takes the draft's top-1 probability.
+ *
+ * spx_draft_confidence: for every draft row d (indexed as in the sampling half: request r owns
+ * rows q_indptr[r]-r .. +k_r-1 of draft_logits) at temperature 1
+ *   conf_max[d] = max_v softmax(D_d)(v);  conf_tok[d] = softmax(D_d)(x_d)  (optional, needs ids);
+ *   req_conf[r] = product of conf_max over the request's drafts (1 when k_r = 0).
+ * fp32 results of float64 merges of fp32 partial sums (relative error of order 1e-6).  Workspace
+ * from spx_draft_confidence_workspace (0 = invalid arguments), 256-byte aligned, caller-owned.
+ * An id outside [0, vocab) sets SPX_DEV_BAD_TOKEN and conf_tok = NaN for that draft.
+ *
+ * spx_select_speculation: among the requests with k_in[r] > 0 (N of them) the
+ * floor(alpha * N) with the lowest confidence get k_out[r] = 0, the others k_out[r] = k_in[r].
+ * Order: the IEEE total order on the stored fp32 confidences (bit patterns; -0 < +0, NaNs at the
+ * ends by sign); among equal confidences the higher index is dropped first.  Integer-exact.
+ * alpha outside [0, 1] is SPX_ERR_INVALID_ARG; a negative k_in sets SPX_DEV_BAD_LEN and counts as
+ * 0.  n_drop (device, optional) receives floor(alpha * N).  k_out may alias k_in.  One thread
+ * block: meant for batches up to a few 10^4 requests.
+ */
+typedef struct {
+  int32_t batch, total_q;            /* total_q = q_indptr[B]; draft rows TD = total_q - B      */
+  int32_t vocab;
+  int64_t logits_row_stride;         /* elements                                                */
+  spx_dtype_t logits_dtype;
+  const void *draft_logits;          /* [TD, vocab], 16-byte aligned                            */
+  const int32_t *draft_token_ids;    /* [TD]; may be NULL when conf_tok is NULL                 */
+  const int32_t *q_indptr;           /* [B+1]                                                   */
+  float *conf_max;                   /* [TD], written                                           */
+  float *conf_tok;                   /* [TD], written; optional                                 */
+  float *req_conf;                   /* [B], written                                            */
+} spx_conf_args_t;
+
+size_t spx_draft_confidence_workspace(const spx_conf_args_t *args);
+spx_status_t spx_draft_confidence(const spx_conf_args_t *args, void *workspace, size_t workspace_bytes,
+                                  int32_t *dev_status, void *cuda_stream);
+spx_status_t spx_select_speculation(int32_t batch, const float *confidence, const int32_t *k_in, double alpha,
+                                    int32_t *k_out, int32_t *n_drop, int32_t *dev_status, void *cuda_stream);
+
+/*
  * Convenience for callers whose data lives on the HOST: every pointer in the two structs is a
  * host pointer (pinned memory recommended); device staging buffers, the workspace and the
  * status word are carved from `dev_arena` (device memory, `arena_bytes` >=

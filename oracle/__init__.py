@@ -334,3 +334,76 @@ def select_speculation(confidence: torch.Tensor, k_in: torch.Tensor, alpha: floa
     if st != OK:
         raise OracleError(st)
     return kout, int(nd.value)
+
+
+# ---- the paper's scheduler numerics (Eq. 1-4, the gain G, Algorithm 1) ----
+
+def sp_recurrence(B: float, N: int, theta: float, T: int):
+    """Eq. 1 iterated from Appendix A.1's initial conditions: (s_a, s_r, n), each [T+1] float64."""
+    lib = _load()
+    sa, sr, n = (torch.empty(T + 1, dtype=torch.float64) for _ in range(3))
+    lib.oracle_sp_recurrence.restype = c.c_int
+    lib.oracle_sp_recurrence.argtypes = [c.c_double, c.c_int32, c.c_double, c.c_int32, c.c_void_p, c.c_void_p, c.c_void_p]
+    st = lib.oracle_sp_recurrence(float(B), int(N), float(theta), int(T), _ptr(sa), _ptr(sr), _ptr(n))
+    if st != OK:
+        raise OracleError(st)
+    return sa, sr, n
+
+
+def sp_effective_batch(B: float, N: int, theta: float) -> float:
+    lib = _load()
+    lib.oracle_sp_effective_batch.restype = c.c_double
+    lib.oracle_sp_effective_batch.argtypes = [c.c_double, c.c_int32, c.c_double]
+    return float(lib.oracle_sp_effective_batch(float(B), int(N), float(theta)))
+
+
+def alpha_recurrence(B: float, N: int, alpha: float, T: int) -> torch.Tensor:
+    lib = _load()
+    bt = torch.empty(T + 1, dtype=torch.float64)
+    lib.oracle_alpha_recurrence.restype = c.c_int
+    lib.oracle_alpha_recurrence.argtypes = [c.c_double, c.c_int32, c.c_double, c.c_int32, c.c_void_p]
+    st = lib.oracle_alpha_recurrence(float(B), int(N), float(alpha), int(T), _ptr(bt))
+    if st != OK:
+        raise OracleError(st)
+    return bt
+
+
+def alpha_batch(B: float, N: int, alpha: float) -> float:
+    lib = _load()
+    lib.oracle_alpha_batch.restype = c.c_double
+    lib.oracle_alpha_batch.argtypes = [c.c_double, c.c_int32, c.c_double]
+    return float(lib.oracle_alpha_batch(float(B), int(N), float(alpha)))
+
+
+def alpha_effective_batch(B: float, N: int, alpha: float, theta_alpha: float) -> float:
+    lib = _load()
+    lib.oracle_alpha_effective_batch.restype = c.c_double
+    lib.oracle_alpha_effective_batch.argtypes = [c.c_double, c.c_int32, c.c_double, c.c_double]
+    return float(lib.oracle_alpha_effective_batch(float(B), int(N), float(alpha), float(theta_alpha)))
+
+
+def delay_gain(I: float, pdr: float, bs: float, i_delay: float, i_wait: Sequence[float]) -> float:
+    lib = _load()
+    w = torch.tensor(list(i_wait), dtype=torch.float64)
+    lib.oracle_delay_gain.restype = c.c_double
+    lib.oracle_delay_gain.argtypes = [c.c_double, c.c_int32, c.c_double, c.c_double, c.c_double, c.c_void_p]
+    return float(lib.oracle_delay_gain(float(I), w.numel(), float(pdr), float(bs), float(i_delay), _ptr(w)))
+
+
+def lookahead_memory(ell: torch.Tensor, tau: torch.Tensor, prec: torch.Tensor, pp: int, theta: float,
+                     horizon: int = 64) -> torch.Tensor:
+    """Algorithm 1: estimated KV memory (tokens) at look-ahead iterations 1..horizon, float64."""
+    lib = _load()
+    ell = _cpu(ell, torch.int32).contiguous()
+    tau = _cpu(tau, torch.int32).contiguous()
+    prec = _cpu(prec, torch.float64).contiguous()
+    assert ell.numel() == tau.numel() == prec.numel()
+    M = torch.empty(horizon, dtype=torch.float64)
+    lib.oracle_lookahead_memory.restype = c.c_int
+    lib.oracle_lookahead_memory.argtypes = [c.c_int32, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int32, c.c_double,
+                                            c.c_int32, c.c_void_p]
+    st = lib.oracle_lookahead_memory(ell.numel(), _ptr(ell), _ptr(tau), _ptr(prec), int(pp), float(theta), int(horizon),
+                                     _ptr(M))
+    if st != OK:
+        raise OracleError(st)
+    return M

@@ -41,7 +41,12 @@
  * numpy's argmax on rows with ties, and the tau -> 0 limit meeting the greedy branch; for the
  * selective-speculation support (tests/test_oracle_select.py; Section 5.1) scipy's softmax
  * maxima, the closed forms 1/V and w_max / sum w, numpy's lexsort on (confidence, -index),
- * and the invariants of a keep-top-(1-alpha) selection (count, separation, alpha = 0 and 1).
+ * and the invariants of a keep-top-(1-alpha) selection (count, separation, alpha = 0 and 1);
+ * for the scheduler numerics (tests/test_oracle_model.py; Eq. 1-4, Section 5.2, Algorithm 1,
+ * Appendix A.1-A.3) conservation s^a + s^r + n = B, the recurrences' limits against the closed
+ * forms, G against throughput ratios built from the token counts and times of Appendix A.3, and
+ * Algorithm 1 against scipy's binomial pmf, its closed forms at pp = 1 and theta = 1, and a
+ * Python brute force.
  */
 #include <math.h>
 #include <stdint.h>
@@ -581,6 +586,120 @@ int oracle_select_speculation(int32_t batch, const float *confidence, const int3
     k_out[worst] = 0;
   }
   if (n_drop_out) *n_drop_out = (int32_t)n_drop;
+  return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* (F) the paper's scheduler numerics: Eq. 1-4, the gain G, Algorithm 1                   */
+/* ------------------------------------------------------------------------------------ */
+
+/*
+ * Eq. 1 with the initial conditions of Appendix A.1 (s^a_0 = s^r_0 = 0, n_0 = B, everything 0
+ * for t < 0), iterated for t = 0..T.  sa, sr, n each hold T+1 doubles.
+ *   s^a_t = (s^a_{t-1} + n_{t-1}) Theta
+ *   s^r_t = sum_{i=1}^{N-1} (s^a_{t-i} + n_{t-i}) (1 - Theta)
+ *   n_t   = (s^a_{t-N} + n_{t-N}) (1 - Theta)
+ */
+int oracle_sp_recurrence(double B, int32_t N, double theta, int32_t T, double *sa, double *sr,
+                         double *n) {
+  if (N < 1 || T < 0 || !(theta >= 0.0 && theta <= 1.0)) return ORACLE_ERR_ARG;
+  for (int t = 0; t <= T; ++t) {
+    if (t == 0) { sa[0] = 0.0; sr[0] = 0.0; n[0] = B; continue; }
+    sa[t] = (sa[t - 1] + n[t - 1]) * theta;
+    double rej = 0.0;
+    for (int i = 1; i <= N - 1; ++i)
+      if (t - i >= 0) rej += (sa[t - i] + n[t - i]) * (1.0 - theta);
+    sr[t] = rej;
+    n[t] = (t - N >= 0) ? (sa[t - N] + n[t - N]) * (1.0 - theta) : 0.0;
+  }
+  return ORACLE_OK;
+}
+
+/* Eq. 2: steady-state effective batch of speculative-parallel execution. */
+double oracle_sp_effective_batch(double B, int32_t N, double theta) {
+  return B / ((double)N - theta * (double)(N - 1));
+}
+
+/*
+ * Eq. 3 with the initial conditions of Appendix A.2 (B_i = B (1-alpha)^i for 0 <= i <= N-1):
+ * B_{t+1} = alpha B_{t+1-N} + (1-alpha) B_t, for t+1 = N..T.  Bt holds T+1 doubles.
+ */
+int oracle_alpha_recurrence(double B, int32_t N, double alpha, int32_t T, double *Bt) {
+  if (N < 1 || T < 0 || !(alpha >= 0.0 && alpha < 1.0)) return ORACLE_ERR_ARG;
+  for (int t = 0; t <= T; ++t) {
+    if (t <= N - 1) Bt[t] = B * pow(1.0 - alpha, (double)t);
+    else Bt[t] = alpha * Bt[t - N] + (1.0 - alpha) * Bt[t - 1];
+  }
+  return ORACLE_OK;
+}
+
+/* Eq. 3, limit: steady-state batch under drop ratio alpha. */
+double oracle_alpha_batch(double B, int32_t N, double alpha) {
+  return B / (1.0 + alpha * (double)(N - 1));
+}
+
+/* Eq. 4: expected effective batch under selective speculation. */
+double oracle_alpha_effective_batch(double B, int32_t N, double alpha, double theta_alpha) {
+  const double Ba = oracle_alpha_batch(B, N, alpha);
+  return alpha * Ba + (1.0 - alpha) * Ba / ((double)N - theta_alpha * (double)(N - 1));
+}
+
+/*
+ * Section 5.2, gain of delayed over aggressive admission:
+ * G = (I + (n+1)(pdr-1)) / (I + pdr - 1) * (bs + 1 - i_delay/I) / (bs + 1 - sum_k i_wait^k / I).
+ */
+double oracle_delay_gain(double I, int32_t n, double pdr, double bs, double i_delay,
+                         const double *i_wait) {
+  double wait = 0.0;
+  for (int k = 0; k < n; ++k) wait += i_wait[k];
+  const double left = (I + (double)(n + 1) * (pdr - 1.0)) / (I + pdr - 1.0);
+  const double right = (bs + 1.0 - i_delay / I) / (bs + 1.0 - wait / I);
+  return left * right;
+}
+
+/*
+ * Algorithm 1: look-ahead memory estimate (in tokens) for iterations i = 1..horizon (the paper
+ * uses 64).  Per request r: ell[r] current length, tau[r] predicted remaining length, prec[r] the
+ * precision E(tau[r]) of that prediction (the caller evaluates E).  pp pipeline depth, theta
+ * speculation accuracy.  With w rejections by iteration i:
+ *   t = i - pp w (accepted), k = t + w (generated), p = C(k, t) theta^t (1-theta)^w,
+ *   w_max = floor(i / pp);
+ *   E[L_gen] = sum_w k p;  P_fin(r) = prec[r] sum_w [k >= tau[r]] p;
+ *   E[N_fin] = sum_r P_fin(r);  E[L_fin] = sum_r ell[r] P_fin(r);
+ *   M[i-1] = L_total + (|B| - E[N_fin]) E[L_gen] - E[L_fin],  L_total = sum_r ell[r].
+ * 0^0 = 1 (theta = 0 or 1 select single terms).
+ */
+int oracle_lookahead_memory(int32_t nreq, const int32_t *ell, const int32_t *tau,
+                            const double *prec, int32_t pp, double theta, int32_t horizon,
+                            double *M) {
+  if (nreq < 0 || pp < 1 || horizon < 0 || !(theta >= 0.0 && theta <= 1.0)) return ORACLE_ERR_ARG;
+  double L_total = 0.0;
+  for (int r = 0; r < nreq; ++r) L_total += (double)ell[r];
+  for (int i = 1; i <= horizon; ++i) {
+    const int w_max = i / pp;
+    double E_gen = 0.0;
+    for (int w = 0; w <= w_max; ++w) {
+      const int t = i - pp * w, k = t + w;
+      double binom = 1.0;
+      for (int j = 1; j <= w; ++j) binom = binom * (double)(t + j) / (double)j;
+      E_gen += (double)k * binom * pow(theta, (double)t) * pow(1.0 - theta, (double)w);
+    }
+    double E_nfin = 0.0, E_lfin = 0.0;
+    for (int r = 0; r < nreq; ++r) {
+      double reach = 0.0;
+      for (int w = 0; w <= w_max; ++w) {
+        const int t = i - pp * w, k = t + w;
+        if (k < tau[r]) continue;
+        double binom = 1.0;
+        for (int j = 1; j <= w; ++j) binom = binom * (double)(t + j) / (double)j;
+        reach += binom * pow(theta, (double)t) * pow(1.0 - theta, (double)w);
+      }
+      const double P_fin = prec[r] * reach;
+      E_nfin += P_fin;
+      E_lfin += (double)ell[r] * P_fin;
+    }
+    M[i - 1] = L_total + ((double)nreq - E_nfin) * E_gen - E_lfin;
+  }
   return ORACLE_OK;
 }
 

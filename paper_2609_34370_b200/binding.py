@@ -16,7 +16,8 @@ BF16, F32 = 0, 1
 
 EXPORTS = ("spx_workspace_size", "spx_verify_attention", "spx_rejection_sample", "spx_verify_step",
            "spx_host_step_arena_size", "spx_verify_step_host", "spx_status_string", "spx_last_launch_count",
-           "spx_set_timing_events", "spx_rejection_sample_static", "spx_kv_append", "spx_kv_rollback")
+           "spx_set_timing_events", "spx_rejection_sample_static", "spx_kv_append", "spx_kv_rollback",
+           "spx_draft_confidence_workspace", "spx_draft_confidence", "spx_select_speculation")
 
 
 class AttnArgs(C.Structure):
@@ -51,6 +52,15 @@ class KvAppendArgs(C.Structure):
         ("new_k", C.c_void_p), ("new_v", C.c_void_p), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
         ("kv_stride_page", C.c_int64), ("kv_stride_head", C.c_int64), ("kv_stride_token", C.c_int64),
         ("block_table", C.c_void_p), ("seq_lens", C.c_void_p), ("q_indptr", C.c_void_p),
+    ]
+
+
+class ConfArgs(C.Structure):
+    _fields_ = [
+        ("batch", C.c_int32), ("total_q", C.c_int32), ("vocab", C.c_int32), ("logits_row_stride", C.c_int64),
+        ("logits_dtype", C.c_int),
+        ("draft_logits", C.c_void_p), ("draft_token_ids", C.c_void_p), ("q_indptr", C.c_void_p),
+        ("conf_max", C.c_void_p), ("conf_tok", C.c_void_p), ("req_conf", C.c_void_p),
     ]
 
 
@@ -98,6 +108,13 @@ def load_library():
         lib.spx_kv_append.argtypes = [C.POINTER(KvAppendArgs), C.c_void_p, C.c_void_p]
         lib.spx_kv_rollback.restype = C.c_int
         lib.spx_kv_rollback.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.spx_draft_confidence_workspace.restype = C.c_size_t
+        lib.spx_draft_confidence_workspace.argtypes = [C.POINTER(ConfArgs)]
+        lib.spx_draft_confidence.restype = C.c_int
+        lib.spx_draft_confidence.argtypes = [C.POINTER(ConfArgs), C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        lib.spx_select_speculation.restype = C.c_int
+        lib.spx_select_speculation.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_double, C.c_void_p, C.c_void_p,
+                                               C.c_void_p, C.c_void_p]
         lib.spx_set_timing_events.restype = None
         lib.spx_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
         _lib = lib
@@ -339,3 +356,46 @@ def kv_rollback(seq_lens, q_indptr, accepted_len, out: Optional[torch.Tensor] = 
     _check(lib.spx_kv_rollback(seq_lens.numel(), seq_lens.data_ptr(), q_indptr.data_ptr(), accepted_len.data_ptr(),
                                out.data_ptr(), status.data_ptr(), _stream(dev)))
     return out, status
+
+
+def draft_confidence(draft_logits, draft_ids, q_indptr, vocab=None, want_token_conf=True, ws: Optional[Workspace] = None):
+    """spx_draft_confidence on the current stream.  Returns (conf_max, conf_tok or None, req_conf, ws)."""
+    _require_cuda(draft_logits, q_indptr)
+    lib = load_library()
+    dev = q_indptr.device
+    B = q_indptr.numel() - 1
+    TD = draft_logits.shape[0]
+    a = ConfArgs()
+    a.batch, a.total_q = B, TD + B
+    a.vocab = int(vocab if vocab is not None else draft_logits.shape[1])
+    a.logits_row_stride = draft_logits.stride(0) if TD else a.vocab + (-a.vocab) % 8
+    a.logits_dtype = _dtype_code(draft_logits)
+    conf_max = torch.empty(TD, dtype=torch.float32, device=dev)
+    conf_tok = torch.empty(TD, dtype=torch.float32, device=dev) if want_token_conf and draft_ids is not None else None
+    req_conf = torch.empty(B, dtype=torch.float32, device=dev)
+    a.draft_logits, a.draft_token_ids, a.q_indptr = _ptr(draft_logits), _ptr(draft_ids), q_indptr.data_ptr()
+    a.conf_max, a.conf_tok, a.req_conf = _ptr(conf_max), _ptr(conf_tok), _ptr(req_conf)
+    need = int(lib.spx_draft_confidence_workspace(C.byref(a)))
+    if need == 0:
+        raise SpxError(ERR_INVALID_ARG, "invalid arguments for workspace sizing")
+    if ws is None:
+        ws = Workspace.allocate(need, dev)
+    ws.ensure(need)
+    _check(lib.spx_draft_confidence(C.byref(a), ws.buf.data_ptr(), ws.buf.numel(), ws.status.data_ptr(), _stream(dev)))
+    return conf_max, conf_tok, req_conf, ws
+
+
+def select_speculation(confidence, k_in, alpha: float, out: Optional[torch.Tensor] = None,
+                       status: Optional[torch.Tensor] = None):
+    """spx_select_speculation on the current stream.  Returns (k_out, n_drop [1] int32 on the device, status)."""
+    _require_cuda(confidence, k_in)
+    lib = load_library()
+    dev = k_in.device
+    if out is None:
+        out = torch.empty_like(k_in)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    n_drop = torch.zeros(1, dtype=torch.int32, device=dev)
+    _check(lib.spx_select_speculation(k_in.numel(), _ptr(confidence), _ptr(k_in), float(alpha), _ptr(out),
+                                      n_drop.data_ptr(), status.data_ptr(), _stream(dev)))
+    return out, n_drop, status

@@ -12,6 +12,7 @@
 #include "attn_tc4.cuh"
 #include "common.cuh"
 #include "kv_cache.cuh"
+#include "select.cuh"
 #include "plan.cuh"
 #include "sampler.cuh"
 #include "spx.h"
@@ -610,6 +611,79 @@ spx_status_t spx_kv_rollback(int32_t batch, const int32_t *seq_lens, const int32
   if (!seq_lens || !q_indptr || !accepted_len || !new_seq_lens) return SPX_ERR_INVALID_ARG;
   kv_rollback_kernel<<<(batch + 127) / 128, 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(batch, seq_lens, q_indptr,
                                                                                                accepted_len, new_seq_lens, dev_status);
+  ++t_launches;
+  return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
+}
+
+// ---- selective speculation support ------------------------------------------------------------
+static spx_status_t check_conf(const spx_conf_args_t *c, bool need_ptrs) {
+  if (!c) return SPX_ERR_INVALID_ARG;
+  if (c->batch < 0 || c->total_q < c->batch || c->vocab <= 0 || c->logits_row_stride < c->vocab) return SPX_ERR_INVALID_ARG;
+  if (c->logits_dtype != SPX_BF16 && c->logits_dtype != SPX_F32) return SPX_ERR_INVALID_ARG;
+  if (c->logits_row_stride % (c->logits_dtype == SPX_BF16 ? 8 : 4) != 0) return SPX_ERR_INVALID_ARG;
+  if ((int64_t)c->total_q - c->batch > (int64_t)c->batch * SPX_MAX_K) return SPX_ERR_INVALID_ARG;
+  if (need_ptrs && c->batch > 0) {
+    if (!c->q_indptr || !c->req_conf) return SPX_ERR_INVALID_ARG;
+    if (c->total_q > c->batch && (!c->draft_logits || !c->conf_max || ((uintptr_t)c->draft_logits & 15))) return SPX_ERR_INVALID_ARG;
+    if (c->conf_tok && c->total_q > c->batch && !c->draft_token_ids) return SPX_ERR_INVALID_ARG;
+  }
+  return SPX_OK;
+}
+
+size_t spx_draft_confidence_workspace(const spx_conf_args_t *c) {
+  if (check_conf(c, false) != SPX_OK) return 0;
+  const size_t nsub = (c->vocab + kSubElems - 1) / kSubElems;
+  return align_up(sizeof(float2) * (size_t)(c->total_q - c->batch) * nsub + 256, 256);
+}
+
+spx_status_t spx_draft_confidence(const spx_conf_args_t *c, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                  void *cuda_stream) {
+  t_launches = 0;
+  const spx_status_t st = check_conf(c, true);
+  if (st != SPX_OK) return st;
+  if (!dev_status) return SPX_ERR_INVALID_ARG;
+  if (c->batch == 0) return SPX_OK;
+  const size_t need = spx_draft_confidence_workspace(c);
+  if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return SPX_ERR_WORKSPACE;
+  DeviceInfo info;
+  if (!get_device_info(&info)) return SPX_ERR_CUDA;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const int td = c->total_q - c->batch;
+  const int nsub = (c->vocab + kSubElems - 1) / kSubElems;
+  if ((int64_t)td * nsub > 0x7fffffff) return SPX_ERR_UNSUPPORTED;
+  if (td > 0) {
+    // the statistics pass of the sampling half, over the draft rows only
+    SampleParams p{};
+    p.batch = c->batch; p.total_q = td; p.total_d = 0; p.vocab = c->vocab; p.nsub = nsub;
+    p.nseg = (c->vocab + kSegElems - 1) / kSegElems;
+    p.row_stride = c->logits_row_stride;
+    p.target = c->draft_logits; p.draft = c->draft_logits;
+    p.seg_stats = static_cast<float2 *>(workspace);
+    p.dev_status = dev_status;
+    const spx_status_t ls = c->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16, false>(p, stream, info.num_sms, kPhaseStats)
+                                                        : launch_sampler_t<float, false>(p, stream, info.num_sms, kPhaseStats);
+    if (ls != SPX_OK) return ls;
+  }
+  ConfParams q{};
+  q.batch = c->batch; q.total_d = td; q.vocab = c->vocab; q.nsub = nsub; q.row_stride = c->logits_row_stride;
+  q.draft = c->draft_logits; q.draft_ids = c->draft_token_ids; q.q_indptr = c->q_indptr;
+  q.seg_stats = static_cast<const float2 *>(workspace);
+  q.conf_max = c->conf_max; q.conf_tok = c->conf_tok; q.req_conf = c->req_conf; q.dev_status = dev_status;
+  const int blocks = (c->batch * 32 + 127) / 128;
+  if (c->logits_dtype == SPX_BF16) confidence_kernel<__nv_bfloat16><<<blocks, 128, 0, stream>>>(q);
+  else confidence_kernel<float><<<blocks, 128, 0, stream>>>(q);
+  ++t_launches;
+  return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
+}
+
+spx_status_t spx_select_speculation(int32_t batch, const float *confidence, const int32_t *k_in, double alpha, int32_t *k_out,
+                                    int32_t *n_drop, int32_t *dev_status, void *cuda_stream) {
+  t_launches = 0;
+  if (batch < 0 || !dev_status || !(alpha >= 0.0 && alpha <= 1.0)) return SPX_ERR_INVALID_ARG;
+  if (batch == 0) return SPX_OK;
+  if (!confidence || !k_in || !k_out) return SPX_ERR_INVALID_ARG;
+  select_kernel<<<1, kSelThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(batch, confidence, k_in, alpha, k_out, n_drop,
+                                                                               dev_status);
   ++t_launches;
   return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
 }
