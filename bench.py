@@ -226,8 +226,26 @@ def time_extras(spx, binding, spec, b, attn_args, dev, iters: int = 200):
         ws.ensure(spx.workspace_size(attn_args, sv))
         out[f"sample_tau_{name}_us"] = timed(sample_call(sv))
         out[f"step_tau_{name}_us"] = timed(lambda: spx.verify_step(attn_args, sv, ws, dev))
-    if int(ws.status.item()) != 0 or int(status.item()) != 0:
-        out["status"] = [int(ws.status.item()), int(status.item())]
+    # selective-speculation support and Algorithm 1
+    cws = spx.Workspace.allocate(1 << 20, dev)
+    out["draft_confidence_us"] = timed(lambda: spx.draft_confidence(b.draft_logits, b.draft_ids, b.q_indptr, ws=cws))
+    out["draft_confidence_bytes"] = b.draft_logits.numel() * b.draft_logits.element_size()
+    conf = spx.draft_confidence(b.draft_logits, b.draft_ids, b.q_indptr, ws=cws)[2]
+    k_in = torch.tensor(b.k_host, dtype=torch.int32, device=dev)
+    k_out = torch.empty_like(k_in)
+    n_drop = torch.zeros(1, dtype=torch.int32, device=dev)
+    out["select_speculation_us"] = timed(lambda: spx.select_speculation(conf, k_in, 0.3, out=k_out, status=status, n_drop=n_drop))
+    big = 16384
+    conf_big = torch.rand(big, device=dev)
+    k_big = torch.ones(big, dtype=torch.int32, device=dev)
+    k_big_out = torch.empty_like(k_big)
+    out["select_speculation_16k_us"] = timed(lambda: spx.select_speculation(conf_big, k_big, 0.3, out=k_big_out, status=status, n_drop=n_drop))
+    ell = b.seq_lens.to(torch.int32)
+    tau = torch.full((b.batch,), 32, dtype=torch.int32, device=dev)
+    prec = torch.full((b.batch,), 0.83, dtype=torch.float64, device=dev)
+    out["lookahead_memory_us"] = timed(lambda: spx.lookahead_memory(ell, tau, prec, 2, 0.7))
+    if int(ws.status.item()) != 0 or int(status.item()) != 0 or int(cws.status.item()) != 0:
+        out["status"] = [int(ws.status.item()), int(status.item()), int(cws.status.item())]
     return out
 
 

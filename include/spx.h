@@ -244,6 +244,33 @@ spx_status_t spx_select_speculation(int32_t batch, const float *confidence, cons
                                     int32_t *k_out, int32_t *n_drop, int32_t *dev_status, void *cuda_stream);
 
 /*
+ * The paper's scheduler numerics.
+ *
+ * spx_lookahead_memory is its Algorithm 1 ("look-ahead memory estimation over future
+ * iterations"): for i = 1..horizon (the paper uses 64), with pipeline depth pp and speculation
+ * accuracy theta, w counting a request's rejected speculations,
+ *   t = i - pp w,  k = t + w,  p = C(k, t) theta^t (1 - theta)^w,  w = 0..floor(i / pp),
+ *   E[L_gen] = sum_w k p,   P_fin(r) = prec[r] * sum_w [k >= tau[r]] p,
+ *   M[i-1] = sum_r ell[r] + (nreq - sum_r P_fin(r)) E[L_gen] - sum_r ell[r] P_fin(r),
+ * where ell[r] is the request's current length, tau[r] its predicted remaining length and
+ * prec[r] the precision of that prediction (the caller evaluates the predictor's precision
+ * table).  All device pointers; float64 arithmetic; 0^0 = 1.  Supported: 1 <= horizon <= 256,
+ * pp >= 1, theta in [0, 1]; otherwise SPX_ERR_INVALID_ARG.
+ *
+ * The closed forms run on the host (they are scalar): Eq. 2 (steady-state effective batch of
+ * speculative-parallel execution, B / (N - theta (N - 1))), Eq. 3's limit (steady-state batch
+ * under drop ratio alpha, B / (1 + alpha (N - 1))), Eq. 4 (effective batch under selective
+ * speculation), and the gain G of delayed over aggressive admission (Section 5.2).
+ */
+spx_status_t spx_lookahead_memory(int32_t nreq, const int32_t *ell, const int32_t *tau, const double *prec, int32_t pp,
+                                  double theta, int32_t horizon, double *mem_estimate, void *cuda_stream);
+double spx_sp_effective_batch(double batch, int32_t stages, double theta);
+double spx_selective_batch(double batch, int32_t stages, double alpha);
+double spx_selective_effective_batch(double batch, int32_t stages, double alpha, double theta_alpha);
+double spx_delay_gain(double iterations, int32_t n_evictions, double pdr, double running, double i_delay,
+                      const double *i_wait /* host, [n_evictions] */);
+
+/*
  * Convenience for callers whose data lives on the HOST: every pointer in the two structs is a
  * host pointer (pinned memory recommended); device staging buffers, the workspace and the
  * status word are carved from `dev_arena` (device memory, `arena_bytes` >=

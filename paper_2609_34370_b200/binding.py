@@ -17,7 +17,9 @@ BF16, F32 = 0, 1
 EXPORTS = ("spx_workspace_size", "spx_verify_attention", "spx_rejection_sample", "spx_verify_step",
            "spx_host_step_arena_size", "spx_verify_step_host", "spx_status_string", "spx_last_launch_count",
            "spx_set_timing_events", "spx_rejection_sample_static", "spx_kv_append", "spx_kv_rollback",
-           "spx_draft_confidence_workspace", "spx_draft_confidence", "spx_select_speculation")
+           "spx_draft_confidence_workspace", "spx_draft_confidence", "spx_select_speculation",
+           "spx_lookahead_memory", "spx_sp_effective_batch", "spx_selective_batch", "spx_selective_effective_batch",
+           "spx_delay_gain")
 
 
 class AttnArgs(C.Structure):
@@ -115,6 +117,15 @@ def load_library():
         lib.spx_select_speculation.restype = C.c_int
         lib.spx_select_speculation.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_double, C.c_void_p, C.c_void_p,
                                                C.c_void_p, C.c_void_p]
+        lib.spx_lookahead_memory.restype = C.c_int
+        lib.spx_lookahead_memory.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_double, C.c_int32,
+                                             C.c_void_p, C.c_void_p]
+        for name, nargs in (("spx_sp_effective_batch", 0), ("spx_selective_batch", 0), ("spx_selective_effective_batch", 1)):
+            fn = getattr(lib, name)
+            fn.restype = C.c_double
+            fn.argtypes = [C.c_double, C.c_int32, C.c_double] + [C.c_double] * nargs
+        lib.spx_delay_gain.restype = C.c_double
+        lib.spx_delay_gain.argtypes = [C.c_double, C.c_int32, C.c_double, C.c_double, C.c_double, C.POINTER(C.c_double)]
         lib.spx_set_timing_events.restype = None
         lib.spx_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
         _lib = lib
@@ -386,7 +397,7 @@ def draft_confidence(draft_logits, draft_ids, q_indptr, vocab=None, want_token_c
 
 
 def select_speculation(confidence, k_in, alpha: float, out: Optional[torch.Tensor] = None,
-                       status: Optional[torch.Tensor] = None):
+                       status: Optional[torch.Tensor] = None, n_drop: Optional[torch.Tensor] = None):
     """spx_select_speculation on the current stream.  Returns (k_out, n_drop [1] int32 on the device, status)."""
     _require_cuda(confidence, k_in)
     lib = load_library()
@@ -395,7 +406,35 @@ def select_speculation(confidence, k_in, alpha: float, out: Optional[torch.Tenso
         out = torch.empty_like(k_in)
     if status is None:
         status = torch.zeros(1, dtype=torch.int32, device=dev)
-    n_drop = torch.zeros(1, dtype=torch.int32, device=dev)
+    if n_drop is None:
+        n_drop = torch.zeros(1, dtype=torch.int32, device=dev)
     _check(lib.spx_select_speculation(k_in.numel(), _ptr(confidence), _ptr(k_in), float(alpha), _ptr(out),
                                       n_drop.data_ptr(), status.data_ptr(), _stream(dev)))
     return out, n_drop, status
+
+
+def lookahead_memory(ell, tau, prec, pp: int, theta: float, horizon: int = 64):
+    """spx_lookahead_memory on the current stream: [horizon] float64 on the device."""
+    _require_cuda(ell, tau, prec)
+    lib = load_library()
+    out = torch.empty(horizon, dtype=torch.float64, device=ell.device)
+    _check(lib.spx_lookahead_memory(ell.numel(), _ptr(ell), _ptr(tau), _ptr(prec), int(pp), float(theta), int(horizon),
+                                    out.data_ptr(), _stream(ell.device)))
+    return out
+
+
+def sp_effective_batch(batch: float, stages: int, theta: float) -> float:
+    return float(load_library().spx_sp_effective_batch(float(batch), int(stages), float(theta)))
+
+
+def selective_batch(batch: float, stages: int, alpha: float) -> float:
+    return float(load_library().spx_selective_batch(float(batch), int(stages), float(alpha)))
+
+
+def selective_effective_batch(batch: float, stages: int, alpha: float, theta_alpha: float) -> float:
+    return float(load_library().spx_selective_effective_batch(float(batch), int(stages), float(alpha), float(theta_alpha)))
+
+
+def delay_gain(iterations: float, pdr: float, running: float, i_delay: float, i_wait) -> float:
+    w = (C.c_double * len(i_wait))(*[float(x) for x in i_wait])
+    return float(load_library().spx_delay_gain(float(iterations), len(i_wait), float(pdr), float(running), float(i_delay), w))

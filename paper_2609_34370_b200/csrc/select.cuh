@@ -115,6 +115,27 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(int32_t batch, cons
     for (int r = tid; r < batch; r += kSelThreads) k_out[r] = k_in[r] > 0 ? k_in[r] : 0;
     return;
   }
+  if (batch <= kSelThreads) {
+    // small batch: rank by counting.  rank(r) = number of participants that are dropped before r
+    // (lower key, or equal key at a higher index); r is dropped iff rank(r) < n_drop.
+    __shared__ uint32_t s_key[kSelThreads];
+    __shared__ int s_part[kSelThreads];
+    int k = 0;
+    uint32_t key = 0;
+    if (tid < batch) {
+      k = k_in[tid];
+      if (k > 0) key = order_key(confidence[tid]);
+      s_key[tid] = key;
+      s_part[tid] = k > 0;
+    }
+    __syncthreads();
+    if (tid < batch) {
+      int rank = 0;
+      for (int j = 0; j < batch; ++j) rank += (s_part[j] && (s_key[j] < key || (s_key[j] == key && j > tid))) ? 1 : 0;
+      k_out[tid] = (k > 0 && rank >= n_drop) ? k : 0;
+    }
+    return;
+  }
   // radix select, most significant byte first
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
@@ -128,11 +149,25 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(int32_t batch, cons
       if ((key & mask) == prefix) atomicAdd(&s_hist[(key >> shift) & 255], 1);
     }
     __syncthreads();
-    if (tid == 0) {
-      int rank = s_rank, b = 0;
-      while (b < 255 && rank > s_hist[b]) { rank -= s_hist[b]; ++b; }
-      s_prefix = prefix | ((uint32_t)b << shift);
-      s_rank = rank;
+    if (warp == 0) {
+      // lane l owns bins 8l..8l+7: exclusive prefix over lanes, then the owner of the crossing bin walks its 8
+      int mine = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) mine += s_hist[8 * lane + j];
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int nb = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += nb;
+      }
+      const int excl = incl - mine;
+      const int rank = s_rank;
+      if (rank > excl && rank <= incl) {
+        int left = rank - excl, b = 8 * lane;
+        while (left > s_hist[b]) { left -= s_hist[b]; ++b; }
+        s_prefix = prefix | ((uint32_t)b << shift);
+        s_rank = left;
+      }
     }
     __syncthreads();
   }

@@ -13,6 +13,7 @@
 #include "common.cuh"
 #include "kv_cache.cuh"
 #include "select.cuh"
+#include "lookahead.cuh"
 #include "plan.cuh"
 #include "sampler.cuh"
 #include "spx.h"
@@ -686,6 +687,35 @@ spx_status_t spx_select_speculation(int32_t batch, const float *confidence, cons
                                                                                dev_status);
   ++t_launches;
   return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
+}
+
+// ---- the paper's scheduler numerics -----------------------------------------------------------
+spx_status_t spx_lookahead_memory(int32_t nreq, const int32_t *ell, const int32_t *tau, const double *prec, int32_t pp,
+                                  double theta, int32_t horizon, double *mem_estimate, void *cuda_stream) {
+  t_launches = 0;
+  if (nreq < 0 || pp < 1 || horizon < 1 || horizon > kLookMaxHorizon || !(theta >= 0.0 && theta <= 1.0) || !mem_estimate)
+    return SPX_ERR_INVALID_ARG;
+  if (nreq > 0 && (!ell || !tau || !prec)) return SPX_ERR_INVALID_ARG;
+  lookahead_kernel<<<horizon, kLookThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(nreq, ell, tau, prec, pp, theta,
+                                                                                         mem_estimate);
+  ++t_launches;
+  return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
+}
+
+double spx_sp_effective_batch(double batch, int32_t stages, double theta) {
+  return batch / ((double)stages - theta * (double)(stages - 1));
+}
+double spx_selective_batch(double batch, int32_t stages, double alpha) { return batch / (1.0 + alpha * (double)(stages - 1)); }
+double spx_selective_effective_batch(double batch, int32_t stages, double alpha, double theta_alpha) {
+  const double ba = spx_selective_batch(batch, stages, alpha);
+  return alpha * ba + (1.0 - alpha) * spx_sp_effective_batch(ba, stages, theta_alpha);
+}
+double spx_delay_gain(double iterations, int32_t n_evictions, double pdr, double running, double i_delay, const double *i_wait) {
+  double waited = 0.0;
+  for (int k = 0; k < n_evictions; ++k) waited += i_wait[k];
+  const double recompute = (iterations + (double)(n_evictions + 1) * (pdr - 1.0)) / (iterations + pdr - 1.0);
+  const double idle = (running + 1.0 - i_delay / iterations) / (running + 1.0 - waited / iterations);
+  return recompute * idle;
 }
 
 // ---- sampling without caller-provided scratch ------------------------------------------------
