@@ -193,12 +193,14 @@ class SampleResult:
     cdf_hi: torch.Tensor         # [B] float64
     flags: torch.Tensor          # [B] int32
     status: int                  # OK, ERR_TOKEN or ERR_PARAM
+    margin: Optional[torch.Tensor] = None   # [B] float64: smallest top-p decision margin (filtered calls only)
 
 
 def rejection_sample(target_logits: torch.Tensor, draft_logits: torch.Tensor,
                      draft_ids: torch.Tensor, q_indptr: torch.Tensor, u_accept: torch.Tensor,
                      u_sample: torch.Tensor, vocab: Optional[int] = None,
-                     temperature: Optional[torch.Tensor] = None) -> SampleResult:
+                     temperature: Optional[torch.Tensor] = None, top_k: Optional[torch.Tensor] = None,
+                     top_p: Optional[torch.Tensor] = None) -> SampleResult:
     """Speculative rejection sampling for the whole batch, in float64, one request at a time.
     ``temperature`` ([B] float32, optional): > 0 verifies at that temperature, 0 verifies greedily."""
     lib = _load()
@@ -228,7 +230,18 @@ def rejection_sample(target_logits: torch.Tensor, draft_logits: torch.Tensor,
         cdf_hi=torch.empty(B, dtype=torch.float64),
         flags=torch.empty(B, dtype=torch.int32),
         status=OK)
-    if temperature is None:
+    if top_k is not None or top_p is not None:
+        tau = _cpu(temperature, torch.float32).contiguous() if temperature is not None else None
+        tk = _cpu(top_k, torch.int32).contiguous() if top_k is not None else None
+        tp = _cpu(top_p, torch.float32).contiguous() if top_p is not None else None
+        res.margin = torch.empty(B, dtype=torch.float64)
+        lib.oracle_rejection_sample_filtered.restype = c.c_int
+        lib.oracle_rejection_sample_filtered.argtypes = [c.c_int32, c.c_int64, c.c_int64, c.c_int32] + [c.c_void_p] * 17
+        st = lib.oracle_rejection_sample_filtered(
+            B, V, row_stride, dt, _ptr(tl), _ptr(dl), _ptr(ids), _ptr(qi), _ptr(ua), _ptr(us), _ptr(tau), _ptr(tk),
+            _ptr(tp), _ptr(res.accepted_len), _ptr(res.out_tokens), _ptr(res.rho), _ptr(res.resid_mass),
+            _ptr(res.cdf_lo), _ptr(res.cdf_hi), _ptr(res.flags), _ptr(res.margin))
+    elif temperature is None:
         st = lib.oracle_rejection_sample(
             B, V, row_stride, dt, _ptr(tl), _ptr(dl), _ptr(ids), _ptr(qi), _ptr(ua), _ptr(us),
             _ptr(res.accepted_len), _ptr(res.out_tokens), _ptr(res.rho), _ptr(res.resid_mass),
@@ -249,7 +262,8 @@ def rejection_sample(target_logits: torch.Tensor, draft_logits: torch.Tensor,
 
 
 def emit_cdf(r: int, n: int, target_logits: torch.Tensor, draft_logits: torch.Tensor,
-             q_indptr: torch.Tensor, vocab: Optional[int] = None, tau: float = 1.0):
+             q_indptr: torch.Tensor, vocab: Optional[int] = None, tau: float = 1.0, top_k: int = 0,
+             top_p: float = 1.0):
     """Inclusive cumulative distribution request ``r``'s emitted token was drawn from, and R."""
     lib = _load()
     tl = _cpu(target_logits)
@@ -257,11 +271,11 @@ def emit_cdf(r: int, n: int, target_logits: torch.Tensor, draft_logits: torch.Te
     V = int(vocab if vocab is not None else tl.shape[1])
     qi = _cpu(q_indptr, torch.int32).contiguous()
     cdf = torch.empty(V, dtype=torch.float64)
-    lib.oracle_emit_cdf_tau.restype = c.c_double
-    lib.oracle_emit_cdf_tau.argtypes = [c.c_int32, c.c_int32, c.c_int64, c.c_int64, c.c_int32, c.c_void_p, c.c_void_p,
-                                        c.c_void_p, c.c_double, c.c_void_p]
-    R = lib.oracle_emit_cdf_tau(int(r), int(n), V, tl.stride(0), _dtype_code(tl), _ptr(tl), _ptr(dl),
-                                _ptr(qi), float(tau), _ptr(cdf))
+    lib.oracle_emit_cdf_filtered.restype = c.c_double
+    lib.oracle_emit_cdf_filtered.argtypes = [c.c_int32, c.c_int32, c.c_int64, c.c_int64, c.c_int32, c.c_void_p, c.c_void_p,
+                                             c.c_void_p, c.c_double, c.c_int32, c.c_double, c.c_void_p]
+    R = lib.oracle_emit_cdf_filtered(int(r), int(n), V, tl.stride(0), _dtype_code(tl), _ptr(tl), _ptr(dl),
+                                     _ptr(qi), float(tau), int(top_k), float(top_p), _ptr(cdf))
     return cdf, float(R)
 
 
@@ -407,3 +421,19 @@ def lookahead_memory(ell: torch.Tensor, tau: torch.Tensor, prec: torch.Tensor, p
     if st != OK:
         raise OracleError(st)
     return M
+
+
+def filtered_row(logits_row: torch.Tensor, tau: float = 1.0, top_k: int = 0, top_p: float = 1.0):
+    """Step 1 under top-k / top-p: (p [V] float64, kept count, top-p decision margin)."""
+    lib = _load()
+    row = _cpu(logits_row).contiguous()
+    V = row.numel()
+    p = torch.empty(V, dtype=torch.float64)
+    scratch = torch.empty(V, dtype=torch.float64)
+    m = c.c_double(0.0)
+    lib.oracle_filtered_row.restype = c.c_int64
+    lib.oracle_filtered_row.argtypes = [c.c_void_p, c.c_int32, c.c_int64, c.c_int64, c.c_double, c.c_int32, c.c_double,
+                                        c.c_void_p, c.c_void_p, c.c_void_p]
+    kept = lib.oracle_filtered_row(_ptr(row), _dtype_code(row), 0, V, float(tau), int(top_k), float(top_p), _ptr(p),
+                                   _ptr(scratch), c.byref(m))
+    return p, int(kept), float(m.value)

@@ -38,7 +38,10 @@
  * this build's reading: the same temperature divides target and draft logits, temperature 0
  * verifies greedily) the output law against softmax(target / tau), the closed form
  * tau*ln(w) -> w / sum w, exact invariance under doubling logits and temperature together,
- * numpy's argmax on rows with ties, and the tau -> 0 limit meeting the greedy branch; for the
+ * numpy's argmax on rows with ties, and the tau -> 0 limit meeting the greedy branch; for top-k /
+ * top-p filtering (tests/test_oracle_filters.py) a numpy restatement by argsort, unique and
+ * cumulative sums, hand-worked rows (0.5, 0.3, 0.15, 0.05), the limits that switch a filter off,
+ * ties kept together, and the output law of speculative sampling under filtering; for the
  * selective-speculation support (tests/test_oracle_select.py; Section 5.1) scipy's softmax
  * maxima, the closed forms 1/V and w_max / sum w, numpy's lexsort on (confidence, -index),
  * and the invariants of a keep-top-(1-alpha) selection (count, separation, alpha = 0 and 1);
@@ -262,6 +265,85 @@ int64_t oracle_argmax_row(const void *logits, int32_t dtype, int64_t row_offset,
   return best;
 }
 
+static int cmp_desc(const void *a, const void *b) {
+  const double x = *(const double *)a, y = *(const double *)b;
+  return (x < y) - (x > y);
+}
+
+/*
+ * Step 1 with top-k / top-p filtering (the paper fixes no sampling parameters; this is the usual
+ * serving rule, stated on values so that it does not depend on how ties are ordered):
+ *   top-k (1 <= top_k < V): keep every token whose logit is >= the top_k-th largest logit of the
+ *     row (tokens tying that value are all kept);
+ *   top-p (top_p < 1), applied to the survivors' distribution pi = softmax(x / tau) restricted to
+ *     them: walk the distinct logit values downwards, adding the mass of each value's group; the
+ *     first value at which the running mass reaches top_p is the last one kept;
+ *   p = softmax(x / tau) renormalised over the kept tokens, 0 elsewhere.
+ * sorted is scratch for V doubles.  *margin (may be NULL) receives how far, in units of the
+ * survivors' mass, the top-p crossing was from tipping to a neighbouring value (+inf when top-p is
+ * off): the decision is a floating-point comparison and an fp32 evaluation may legitimately differ
+ * when this is tiny.  Returns the number of kept tokens.
+ */
+int64_t oracle_filtered_row(const void *logits, int32_t dtype, int64_t row_offset, int64_t V,
+                            double tau, int32_t top_k, double top_p, double *p, double *sorted,
+                            double *margin) {
+  for (int64_t v = 0; v < V; ++v) sorted[v] = widen(logits, dtype, row_offset + v);
+  qsort(sorted, (size_t)V, sizeof(double), cmp_desc);
+  const double mx = sorted[0];
+  double thr = -INFINITY;
+  if (top_k >= 1 && (int64_t)top_k < V) thr = sorted[top_k - 1];
+  if (margin) *margin = INFINITY;
+  if (top_p < 1.0) {
+    /* survivors' mass, group by group in descending order (the same order as the walk below) */
+    double Zk = 0.0;
+    for (int64_t j = 0; j < V && sorted[j] >= thr;) {
+      int64_t g = j;
+      double gm = 0.0;
+      while (g < V && sorted[g] == sorted[j]) { gm += exp((sorted[g] - mx) / tau); ++g; }
+      Zk += gm;
+      j = g;
+    }
+    double cum = 0.0;
+    for (int64_t j = 0; j < V && sorted[j] >= thr;) {
+      int64_t g = j;
+      double gm = 0.0;
+      while (g < V && sorted[g] == sorted[j]) { gm += exp((sorted[g] - mx) / tau); ++g; }
+      const double before = cum;
+      cum += gm;
+      if (cum >= top_p * Zk) {
+        thr = sorted[j];
+        if (margin) {
+          const double over = (cum - top_p * Zk) / Zk, under = (top_p * Zk - before) / Zk;
+          *margin = over < under ? over : under;
+        }
+        break;
+      }
+      j = g;
+    }
+  }
+  double Z = 0.0;
+  int64_t kept = 0;
+  for (int64_t v = 0; v < V; ++v) {
+    const double x = widen(logits, dtype, row_offset + v);
+    if (x >= thr) { p[v] = exp((x - mx) / tau); Z += p[v]; ++kept; }
+    else p[v] = 0.0;
+  }
+  for (int64_t v = 0; v < V; ++v) p[v] /= Z;
+  return kept;
+}
+
+/* The distribution of one row under a request's sampling parameters. */
+typedef struct { double tau; int32_t top_k; double top_p; double *sorted; double margin; } row_params_t;
+
+static void row_dist(const void *logits, int32_t dtype, int64_t row_offset, int64_t V,
+                     row_params_t *rp, double *p) {
+  const int filtered = (rp->top_k >= 1 && (int64_t)rp->top_k < V) || rp->top_p < 1.0;
+  if (!filtered) { oracle_softmax_row_tau(logits, dtype, row_offset, V, rp->tau, p); return; }
+  double m;
+  oracle_filtered_row(logits, dtype, row_offset, V, rp->tau, rp->top_k, rp->top_p, p, rp->sorted, &m);
+  if (m < rp->margin) rp->margin = m;
+}
+
 /* Step 3 (first half): r(v) = max(0, p(v) - q(v)); returns R = sum_v r(v), ascending v. */
 double oracle_residual(const double *p, const double *q, int64_t V, double *r) {
   double R = 0.0;
@@ -317,7 +399,9 @@ static int sample_one(int r, int32_t dtype, int64_t V, int64_t row_stride,
                       const int32_t *draft_ids, const int32_t *q_indptr, const float *u_accept,
                       const float *u_sample, int32_t *accepted_len, int32_t *out_tokens,
                       double *rho_out, double *resid_mass, double *cdf_lo, double *cdf_hi,
-                      int32_t *flags, double *p, double *q, double *res, double tau) {
+                      int32_t *flags, double *p, double *q, double *res, row_params_t *rp) {
+  const double tau = rp->tau;
+  const int filtered = (rp->top_k >= 1 && (int64_t)rp->top_k < V) || rp->top_p < 1.0;
   const int64_t t0 = q_indptr[r];          /* first target row / first output slot */
   const int64_t d0 = (int64_t)q_indptr[r] - r; /* first draft row */
   const int k = q_indptr[r + 1] - q_indptr[r] - 1;
@@ -337,8 +421,8 @@ static int sample_one(int r, int32_t dtype, int64_t V, int64_t row_stride,
   }
   if (rho_out) for (int i = 0; i < k; ++i) rho_out[d0 + i] = NAN; /* rows after n: not consulted */
 
-  if (!(tau >= 0.0) || isinf(tau)) {
-    /* not a temperature: the request emits nothing */
+  if (!(tau >= 0.0) || isinf(tau) || !(rp->top_p > 0.0 && rp->top_p <= 1.0)) {
+    /* not a temperature, or not a nucleus mass: the request emits nothing */
     accepted_len[r] = 0;
     for (int i = 0; i <= k; ++i) out_tokens[t0 + i] = -1;
     if (resid_mass) resid_mass[r] = NAN;
@@ -365,9 +449,10 @@ static int sample_one(int r, int32_t dtype, int64_t V, int64_t row_stride,
   /* step 2: sequential accept tests */
   for (int i = 0; i < k; ++i) {
     const int64_t x = draft_ids[d0 + i];
-    oracle_softmax_row_tau(target_logits, dtype, (t0 + i) * row_stride, V, tau, p);
-    oracle_softmax_row_tau(draft_logits, dtype, (d0 + i) * row_stride, V, tau, q);
-    const double rho = (q[x] == 0.0) ? INFINITY : p[x] / q[x];
+    row_dist(target_logits, dtype, (t0 + i) * row_stride, V, rp, p);
+    row_dist(draft_logits, dtype, (d0 + i) * row_stride, V, rp, q);
+    /* with filtering a draft token can have target probability 0: it is rejected whatever q says */
+    const double rho = (filtered && p[x] == 0.0) ? 0.0 : ((q[x] == 0.0) ? INFINITY : p[x] / q[x]);
     if (rho_out) rho_out[d0 + i] = rho;
     if (!((double)u_accept[d0 + i] < rho)) { n = i; break; }
   }
@@ -385,7 +470,7 @@ static int sample_one(int r, int32_t dtype, int64_t V, int64_t row_stride,
     y = oracle_inverse_cdf(res, V, R, (double)u_sample[r], &lo, &hi);
   } else {
     /* step 4: bonus token from target row k */
-    oracle_softmax_row_tau(target_logits, dtype, (t0 + k) * row_stride, V, tau, p);
+    row_dist(target_logits, dtype, (t0 + k) * row_stride, V, rp, p);
     R = 0.0;
     for (int64_t v = 0; v < V; ++v) R += p[v];
     y = oracle_inverse_cdf(p, V, R, (double)u_sample[r], &lo, &hi);
@@ -414,14 +499,22 @@ static int sample_one(int r, int32_t dtype, int64_t V, int64_t row_stride,
  * was sampled at the request's temperature); tau_r = 0 is greedy verification; anything else
  * (negative, NaN, infinite) makes that request emit n = 0 and -1 tokens and the call return
  * ORACLE_ERR_PARAM.  NULL means tau = 1 everywhere.
+ *
+ * top_k (NULL, or [B] int32; values < 1 or >= V switch it off) and top_p (NULL, or [B] float;
+ * 1 switches it off, values outside (0, 1] are ORACLE_ERR_PARAM like a bad temperature) filter
+ * both the target and the draft rows of the request as oracle_filtered_row states (the draft was
+ * sampled under the request's parameters); greedy requests ignore them.  margin_out (NULL, or
+ * [B]) receives the smallest top-p decision margin over the rows the request consulted.
  */
-int oracle_rejection_sample_tau(int32_t batch, int64_t V, int64_t row_stride, int32_t dtype,
-                                const void *target_logits, const void *draft_logits,
-                                const int32_t *draft_ids, const int32_t *q_indptr,
-                                const float *u_accept, const float *u_sample,
-                                const float *temperature, int32_t *accepted_len,
-                                int32_t *out_tokens, double *rho_out, double *resid_mass,
-                                double *cdf_lo, double *cdf_hi, int32_t *flags) {
+int oracle_rejection_sample_filtered(int32_t batch, int64_t V, int64_t row_stride, int32_t dtype,
+                                     const void *target_logits, const void *draft_logits,
+                                     const int32_t *draft_ids, const int32_t *q_indptr,
+                                     const float *u_accept, const float *u_sample,
+                                     const float *temperature, const int32_t *top_k,
+                                     const float *top_p, int32_t *accepted_len,
+                                     int32_t *out_tokens, double *rho_out, double *resid_mass,
+                                     double *cdf_lo, double *cdf_hi, int32_t *flags,
+                                     double *margin_out) {
   if (batch < 0 || V <= 0 || row_stride < V) return ORACLE_ERR_ARG;
   if (dtype != ORACLE_BF16 && dtype != ORACLE_F32) return ORACLE_ERR_ARG;
   for (int r = 0; r < batch; ++r)
@@ -432,25 +525,45 @@ int oracle_rejection_sample_tau(int32_t batch, int64_t V, int64_t row_stride, in
     double *p = (double *)malloc(sizeof(double) * (size_t)V);
     double *q = (double *)malloc(sizeof(double) * (size_t)V);
     double *res = (double *)malloc(sizeof(double) * (size_t)V);
-    if (!p || !q || !res) {
+    double *sorted = (double *)malloc(sizeof(double) * (size_t)V);
+    if (!p || !q || !res || !sorted) {
 #pragma omp atomic write
       status = ORACLE_ERR_ALLOC;
     }
 #pragma omp for schedule(dynamic, 1)
     for (int r = 0; r < batch; ++r) {
-      if (!p || !q || !res) continue;
+      if (!p || !q || !res || !sorted) continue;
+      row_params_t rp;
+      rp.tau = temperature ? (double)temperature[r] : 1.0;
+      rp.top_k = top_k ? top_k[r] : 0;
+      rp.top_p = top_p ? (double)top_p[r] : 1.0;
+      rp.sorted = sorted;
+      rp.margin = INFINITY;
       const int st = sample_one(r, dtype, V, row_stride, target_logits, draft_logits, draft_ids,
                                 q_indptr, u_accept, u_sample, accepted_len, out_tokens, rho_out,
-                                resid_mass, cdf_lo, cdf_hi, flags, p, q, res,
-                                temperature ? (double)temperature[r] : 1.0);
+                                resid_mass, cdf_lo, cdf_hi, flags, p, q, res, &rp);
+      if (margin_out) margin_out[r] = rp.margin;
       if (st != ORACLE_OK) {
 #pragma omp atomic write
         status = st;
       }
     }
-    free(p); free(q); free(res);
+    free(p); free(q); free(res); free(sorted);
   }
   return status;
+}
+
+int oracle_rejection_sample_tau(int32_t batch, int64_t V, int64_t row_stride, int32_t dtype,
+                                const void *target_logits, const void *draft_logits,
+                                const int32_t *draft_ids, const int32_t *q_indptr,
+                                const float *u_accept, const float *u_sample,
+                                const float *temperature, int32_t *accepted_len,
+                                int32_t *out_tokens, double *rho_out, double *resid_mass,
+                                double *cdf_lo, double *cdf_hi, int32_t *flags) {
+  return oracle_rejection_sample_filtered(batch, V, row_stride, dtype, target_logits, draft_logits,
+                                          draft_ids, q_indptr, u_accept, u_sample, temperature, NULL,
+                                          NULL, accepted_len, out_tokens, rho_out, resid_mass, cdf_lo,
+                                          cdf_hi, flags, NULL);
 }
 
 int oracle_rejection_sample(int32_t batch, int64_t V, int64_t row_stride, int32_t dtype,
@@ -469,19 +582,22 @@ int oracle_rejection_sample(int32_t batch, int64_t V, int64_t row_stride, int32_
  * cdf[0..V) = inclusive cumulative sum of the residual at row n (n < k) or of the target
  * row k (n == k).  n is passed in (the oracle's accepted_len[r]).  Returns R.
  */
-double oracle_emit_cdf_tau(int32_t r, int32_t n, int64_t V, int64_t row_stride, int32_t dtype,
-                           const void *target_logits, const void *draft_logits,
-                           const int32_t *q_indptr, double tau, double *cdf) {
+double oracle_emit_cdf_filtered(int32_t r, int32_t n, int64_t V, int64_t row_stride, int32_t dtype,
+                                const void *target_logits, const void *draft_logits,
+                                const int32_t *q_indptr, double tau, int32_t top_k, double top_p,
+                                double *cdf) {
   const int64_t t0 = q_indptr[r];
   const int64_t d0 = (int64_t)q_indptr[r] - r;
   const int k = q_indptr[r + 1] - q_indptr[r] - 1;
   double *p = (double *)malloc(sizeof(double) * (size_t)V);
   double *q = (double *)malloc(sizeof(double) * (size_t)V);
+  double *sorted = (double *)malloc(sizeof(double) * (size_t)V);
   double R = NAN;
-  if (p && q) {
-    oracle_softmax_row_tau(target_logits, dtype, (t0 + n) * row_stride, V, tau, p);
+  if (p && q && sorted) {
+    row_params_t rp = {tau, top_k, top_p, sorted, INFINITY};
+    row_dist(target_logits, dtype, (t0 + n) * row_stride, V, &rp, p);
     if (n < k) {
-      oracle_softmax_row_tau(draft_logits, dtype, (d0 + n) * row_stride, V, tau, q);
+      row_dist(draft_logits, dtype, (d0 + n) * row_stride, V, &rp, q);
       R = oracle_residual(p, q, V, q);
       if (R == 0.0) { R = 0.0; for (int64_t v = 0; v < V; ++v) { q[v] = p[v]; R += p[v]; } }
       oracle_cumsum(q, V, cdf);
@@ -491,8 +607,15 @@ double oracle_emit_cdf_tau(int32_t r, int32_t n, int64_t V, int64_t row_stride, 
       oracle_cumsum(p, V, cdf);
     }
   }
-  free(p); free(q);
+  free(p); free(q); free(sorted);
   return R;
+}
+
+double oracle_emit_cdf_tau(int32_t r, int32_t n, int64_t V, int64_t row_stride, int32_t dtype,
+                           const void *target_logits, const void *draft_logits,
+                           const int32_t *q_indptr, double tau, double *cdf) {
+  return oracle_emit_cdf_filtered(r, n, V, row_stride, dtype, target_logits, draft_logits, q_indptr,
+                                  tau, 0, 1.0, cdf);
 }
 
 double oracle_emit_cdf(int32_t r, int32_t n, int64_t V, int64_t row_stride, int32_t dtype,
