@@ -121,6 +121,20 @@ typedef struct {
  * sets SPX_DEV_BAD_PARAM and the request emits n = 0 and -1 tokens.  Requests of one batch may mix
  * all three.
  *
+ * top_k / top_p (each NULL = off, else [B]) filter the target AND the draft rows of a request
+ * before the rule is applied (the draft was sampled under the request's parameters):
+ *   top_k[r] = K with 1 <= K < vocab: keep every token whose logit is >= the K-th largest logit of
+ *     the row (tokens tying that value are all kept); other values switch it off;
+ *   top_p[r] = P < 1, applied to the survivors' distribution softmax(x / tau): going down the
+ *     distinct logit values, the first value at which the running mass reaches P is the last one
+ *     kept; P = 1 switches it off; P outside (0, 1] sets SPX_DEV_BAD_PARAM like a bad temperature;
+ *   p and q are softmax(x / tau) renormalised over the kept tokens and 0 elsewhere.  A drafted
+ *   token with p(x) = 0 is rejected; one with q(x) = 0 < p(x) is accepted.
+ * The top-p comparison is made on sums of fp32 exponentials (2^-44 fixed point, order
+ * independent); it can differ from an exact evaluation when the running mass comes within about
+ * 1e-6 of P.  Greedy requests ignore both filters.  The workspace is larger when temperature,
+ * top_k or top_p is given: size it with the same pointers set.
+ *
  * Supported: vocab >= 1; logits_row_stride >= vocab and a multiple of 8 (BF16) or 4 (F32)
  * elements; both logits pointers 16-byte aligned.
  */
@@ -140,6 +154,8 @@ typedef struct {
   int32_t *out_tokens;         /* [TQ], written                                               */
   float *diag_ratio;           /* optional [TD]: p/q of each consulted draft (NaN otherwise)  */
   const float *temperature;    /* optional [B]: see "Verification variants"; NULL = all 1     */
+  const int32_t *top_k;        /* optional [B]                                                */
+  const float *top_p;          /* optional [B]                                                */
 } spx_sample_args_t;
 
 /*

@@ -42,7 +42,7 @@ class SampleArgs(C.Structure):
         ("target_logits", C.c_void_p), ("draft_logits", C.c_void_p), ("draft_token_ids", C.c_void_p),
         ("q_indptr", C.c_void_p), ("u_accept", C.c_void_p), ("u_sample", C.c_void_p),
         ("accepted_len", C.c_void_p), ("out_tokens", C.c_void_p), ("diag_ratio", C.c_void_p),
-        ("temperature", C.c_void_p),
+        ("temperature", C.c_void_p), ("top_k", C.c_void_p), ("top_p", C.c_void_p),
     ]
 
 
@@ -183,7 +183,7 @@ def make_attn_args(q, k_cache, v_cache, kv_strides, block_table, seq_lens, q_ind
 
 
 def make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, accepted_len,
-                     out_tokens, diag_ratio=None, vocab=None, temperature=None) -> SampleArgs:
+                     out_tokens, diag_ratio=None, vocab=None, temperature=None, top_k=None, top_p=None) -> SampleArgs:
     s = SampleArgs()
     s.batch = q_indptr.numel() - 1
     s.total_q = target_logits.shape[0]
@@ -194,7 +194,7 @@ def make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept,
     s.draft_token_ids, s.q_indptr = _ptr(draft_ids), q_indptr.data_ptr()
     s.u_accept, s.u_sample = _ptr(u_accept), _ptr(u_sample)
     s.accepted_len, s.out_tokens, s.diag_ratio = _ptr(accepted_len), _ptr(out_tokens), _ptr(diag_ratio)
-    s.temperature = _ptr(temperature)
+    s.temperature, s.top_k, s.top_p = _ptr(temperature), _ptr(top_k), _ptr(top_p)
     return s
 
 
@@ -245,12 +245,13 @@ def verify_attention(q, k_cache, v_cache, kv_strides, block_table, seq_lens, q_i
 
 
 def rejection_sample(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, vocab=None,
-                     want_ratio=False, ws: Optional[Workspace] = None, temperature=None):
+                     want_ratio=False, ws: Optional[Workspace] = None, temperature=None, top_k=None, top_p=None):
     """spx_rejection_sample on the current stream.  Returns (accepted_len, out_tokens, ratio, ws).
     ``temperature`` ([B] float32 on the device, optional) selects the verification variant per request."""
     _require_cuda(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample)
-    if temperature is not None:
-        _require_cuda(temperature)
+    for extra in (temperature, top_k, top_p):
+        if extra is not None:
+            _require_cuda(extra)
     lib = load_library()
     dev = target_logits.device
     B = q_indptr.numel() - 1
@@ -259,7 +260,7 @@ def rejection_sample(target_logits, draft_logits, draft_ids, q_indptr, u_accept,
     tokens = torch.empty(TQ, dtype=torch.int32, device=dev)
     ratio = torch.empty(TQ - B, dtype=torch.float32, device=dev) if want_ratio else None
     s = make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, accepted, tokens,
-                         ratio, vocab, temperature)
+                         ratio, vocab, temperature, top_k, top_p)
     need = workspace_size(None, s)
     if ws is None:
         ws = Workspace.allocate(need, dev)

@@ -42,8 +42,16 @@ struct SampleParams {
   int32_t *req_done;   // [B]  segments of row n finished (zeroed by accept_kernel)
   int32_t *dev_status;
   // verification variants (both NULL: temperature 1 everywhere)
-  const float *temperature;  // [B]  > 0: sample at that temperature; 0: greedy
+  const float *temperature;  // [B]  > 0: sample at that temperature; 0: greedy (NULL with filters: 1)
   float *row_scale;          // [(TQ+TD)] workspace: log2(e)/tau of the row's request; 0 = row not needed
+  // top-k / top-p filtering (all NULL unless one of top_k / top_p is given)
+  const int32_t *top_k;      // [B]  < 1 or >= vocab: off
+  const float *top_p;        // [B]  1: off
+  int32_t *row_req;          // [(TQ+TD)] request whose filter applies to the row, -1 = none
+  uint32_t *row_thresh;      // [(TQ+TD)] order key of the lowest kept logit (0 = everything kept)
+  double *row_z;             // [(TQ+TD)] kept mass sum 2^(x*scale - M); < 0 = unfiltered, use the statistics
+  uint2 *req_thresh;         // [B]  thresholds of rows n (target, draft)
+  float *seg_pmass;          // [B][nseg] kept target mass of each segment of row n
 };
 
 // 16-byte vector of logits -> floats, scaled into the log2 domain
@@ -354,6 +362,199 @@ __global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleP
   }
 }
 
+// Total order on fp32 bit patterns, as an unsigned key (larger logit -> larger key).
+__device__ __forceinline__ uint32_t order_key32(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// top-k / top-p thresholds of one logits row per block (kFilterThreads threads).
+//
+// The kept set is {v : key(x_v) >= T}.  T is found by a byte-wise radix descent from the top of
+// the key space: each level builds a 256-bin histogram (count, mass) of the elements that match
+// the prefix chosen so far and warp 0 picks the bin where the running count reaches top_k, or the
+// running mass reaches top_p times the survivors' mass.  Masses are sums of 2^(x*scale - M) in
+// 2^-44 fixed point: integer atomics make every sum exact and independent of the order of
+// arrival, so the result is reproducible and the cumulative mass at the top-k threshold equals
+// the survivors' mass bit for bit.  Histograms are private to each warp (shared-memory atomics
+// only collide inside a warp) and summed per level.  bf16 keys have 16 significant bits (2
+// levels), fp32 keys 32 (4 levels).  After the first pass the row is re-read out of L2.
+constexpr int kFilterThreads = 1024;
+constexpr int kFilterWarps = kFilterThreads / 32;
+constexpr float kMassScale = 17592186044416.f;  // 2^44
+constexpr int kFilterSmemBytes = kFilterWarps * 256 * (8 + 4) + 256 * (8 + 4) * 2 + 64;
+
+template <typename T>
+__global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SampleParams p) {
+  extern __shared__ __align__(16) unsigned char fsm[];
+  unsigned long long *w_mass = reinterpret_cast<unsigned long long *>(fsm);                    // [warps][256]
+  unsigned long long *s_mass = w_mass + kFilterWarps * 256;                                    // [256] level sums
+  unsigned long long *s_mass1 = s_mass + 256;                                                  // [256] level-1 copy
+  uint32_t *w_cnt = reinterpret_cast<uint32_t *>(s_mass1 + 256);                               // [warps][256]
+  uint32_t *s_cnt = w_cnt + kFilterWarps * 256;
+  uint32_t *s_cnt1 = s_cnt + 256;
+  __shared__ uint32_t s_bin;
+  __shared__ unsigned long long s_above_mass, s_bin_mass;
+  __shared__ uint32_t s_above_cnt;
+  const int row = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int r = p.row_req[row];
+  if (r < 0) {
+    if (tid == 0) { p.row_thresh[row] = 0; p.row_z[row] = -1.0; }
+    return;
+  }
+  constexpr int kLevels = sizeof(T) == 2 ? 2 : 4;
+  constexpr int kKeyShift = sizeof(T) == 2 ? 16 : 0;  // bf16: the low 16 bits of the fp32 key are zero
+  constexpr int N = Vec<T>::N;
+  const int tk_raw = p.top_k ? p.top_k[r] : 0;
+  const bool use_k = tk_raw >= 1 && tk_raw < p.vocab;
+  const float tp = p.top_p ? p.top_p[r] : 1.f;
+  const bool use_p = tp < 1.f;
+  const float scale = p.row_scale[row];
+  const T *base = row < p.total_q ? reinterpret_cast<const T *>(p.target) + (int64_t)row * p.row_stride
+                                  : reinterpret_cast<const T *>(p.draft) + (int64_t)(row - p.total_q) * p.row_stride;
+  float M = -INFINITY;
+  {
+    const float2 *st = p.seg_stats + (int64_t)row * p.nsub;
+    for (int j = 0; j < p.nsub; ++j) M = fmaxf(M, st[j].x);
+  }
+
+  // one histogram pass: elements whose key matches `prefix` in the bits above `shift + 8`
+  auto hist_pass = [&](uint32_t prefix, int level) {
+    const int shift = kKeyShift + 8 * (kLevels - 1 - level);
+    for (int i = tid; i < kFilterWarps * 256; i += kFilterThreads) { w_cnt[i] = 0; w_mass[i] = 0ull; }
+    __syncthreads();
+    uint32_t *my_cnt = w_cnt + warp * 256;
+    unsigned long long *my_mass = w_mass + warp * 256;
+    auto add = [&](float x) {
+      const uint32_t key = order_key32(x);
+      if (level > 0 && (key >> (shift + 8)) != (prefix >> (shift + 8))) return;
+      const uint32_t bin = (key >> shift) & 255u;
+      atomicAdd(&my_cnt[bin], 1u);
+      const float e = fast_exp2(fmaf(x, scale, -M));
+      atomicAdd(&my_mass[bin], __float2ull_rn(e * kMassScale));
+    };
+    for (int v = tid * N; v < p.vocab; v += kFilterThreads * N) {
+      if (v + N <= p.vocab) {
+        union { uint4 u; T e[N]; } tmp;
+        tmp.u = __ldg(reinterpret_cast<const uint4 *>(base + v));
+#pragma unroll
+        for (int i = 0; i < N; ++i) add(ld_as_float(tmp.e, i));
+      } else {
+        for (int i = 0; i < N && v + i < p.vocab; ++i) add(ld_as_float(base, v + i));
+      }
+    }
+    __syncthreads();
+    if (tid < 256) {
+      uint32_t c = 0;
+      unsigned long long m = 0ull;
+      for (int w = 0; w < kFilterWarps; ++w) { c += w_cnt[w * 256 + tid]; m += w_mass[w * 256 + tid]; }
+      s_cnt[tid] = c;
+      s_mass[tid] = m;
+    }
+    __syncthreads();
+  };
+
+  // warp 0: the highest bin b such that (count or mass of bins >= b, plus what lies above the
+  // prefix) reaches the target; leaves the bin, and count / mass of the bins above it, in shared memory
+  auto pick = [&](bool by_count, uint32_t need_cnt, double need_mass, unsigned long long mass_above_prefix) {
+    if (warp == 0) {
+      // lane l owns bins 255-8l .. 248-8l (descending)
+      uint32_t c8 = 0;
+      unsigned long long m8 = 0ull;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { c8 += s_cnt[255 - 8 * lane - j]; m8 += s_mass[255 - 8 * lane - j]; }
+      uint32_t ci = c8;
+      unsigned long long mi = m8;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t cn = __shfl_up_sync(0xffffffffu, ci, o);
+        const unsigned long long mn = __shfl_up_sync(0xffffffffu, mi, o);
+        if (lane >= o) { ci += cn; mi += mn; }
+      }
+      const bool reached = by_count ? (ci >= need_cnt) : ((double)(mass_above_prefix + mi) >= need_mass);
+      const uint32_t bal = __ballot_sync(0xffffffffu, reached);
+      // rounding could leave the mass criterion unmet even at the last bin: take the lowest occupied bin then
+      const int owner = bal ? __ffs(bal) - 1 : 31;
+      if (lane == owner) {
+        uint32_t cc = ci - c8;
+        unsigned long long mm = mi - m8;
+        int b = 255 - 8 * lane, chosen = -1;
+        for (int j = 0; j < 8; ++j, --b) {
+          const bool hit = by_count ? (cc + s_cnt[b] >= need_cnt) : ((double)(mass_above_prefix + mm + s_mass[b]) >= need_mass);
+          if (hit) { chosen = b; break; }
+          cc += s_cnt[b];
+          mm += s_mass[b];
+        }
+        if (chosen < 0) {  // only without a crossing: lowest occupied bin of the whole level
+          cc = 0; mm = 0ull; chosen = 0;
+          for (int bb = 255; bb >= 0; --bb) if (s_cnt[bb]) chosen = bb;
+          for (int bb = 255; bb > chosen; --bb) { cc += s_cnt[bb]; mm += s_mass[bb]; }
+        }
+        s_bin = (uint32_t)chosen;
+        s_above_cnt = cc;
+        s_above_mass = mm;
+        s_bin_mass = s_mass[chosen];
+      }
+    }
+    __syncthreads();
+  };
+
+  // level 0 serves both descents
+  hist_pass(0u, 0);
+  if (tid < 256) { s_cnt1[tid] = s_cnt[tid]; s_mass1[tid] = s_mass[tid]; }
+  __syncthreads();
+  unsigned long long total = 0ull;
+  for (int b = 0; b < 256; ++b) total += s_mass1[b];   // every thread: 256 broadcast reads
+
+  uint32_t Tk = 0;
+  unsigned long long Zk = total;
+  if (use_k) {
+    uint32_t prefix = 0, need = (uint32_t)tk_raw;
+    unsigned long long above = 0ull;
+    for (int level = 0; level < kLevels; ++level) {
+      if (level > 0) hist_pass(prefix, level);
+      pick(true, need, 0.0, 0ull);
+      const int shift = kKeyShift + 8 * (kLevels - 1 - level);
+      prefix |= s_bin << shift;
+      need -= s_above_cnt;
+      above += s_above_mass;
+      if (level == kLevels - 1) Zk = above + s_bin_mass;
+      __syncthreads();
+    }
+    Tk = prefix;
+  }
+  uint32_t Tf = Tk;
+  unsigned long long Zf = Zk;
+  if (use_p) {
+    const double need_mass = (double)tp * (double)Zk;
+    uint32_t prefix = 0;
+    unsigned long long above = 0ull;
+    for (int level = 0; level < kLevels; ++level) {
+      if (level == 0) {
+        if (use_k) {  // the level-0 histogram was overwritten by the top-k descent: restore it
+          if (tid < 256) { s_cnt[tid] = s_cnt1[tid]; s_mass[tid] = s_mass1[tid]; }
+          __syncthreads();
+        }
+      } else {
+        hist_pass(prefix, level);
+      }
+      pick(false, 0u, need_mass, above);
+      const int shift = kKeyShift + 8 * (kLevels - 1 - level);
+      prefix |= s_bin << shift;
+      above += s_above_mass;
+      if (level == kLevels - 1) Zf = above + s_bin_mass;
+      __syncthreads();
+    }
+    Tf = prefix;
+    if (Tf < Tk) { Tf = Tk; Zf = Zk; }  // cannot happen with exact sums; keeps the sets nested regardless
+  }
+  if (tid == 0) {
+    p.row_thresh[row] = Tf;
+    p.row_z[row] = (double)Zf / (double)kMassScale;
+  }
+}
+
 // Verification variants, step 0: the scale log2(e)/tau of every logits row.  One thread per request.
 // Greedy requests (tau = 0) need only the maxima of their target rows (scale log2(e)); their draft
 // rows, and every row of a request whose temperature is not one, are marked 0 = skip.
@@ -363,12 +564,19 @@ __global__ void row_scale_kernel(SampleParams p) {
   const int t0 = p.q_indptr[r];
   const int k = p.q_indptr[r + 1] - t0 - 1;
   if (k < 0 || k > SPX_MAX_K || t0 < 0 || t0 + k + 1 > p.total_q) return;  // reported by accept_kernel
-  const float tau = p.temperature[r];
-  const bool valid = tau >= 0.f && tau != INFINITY;
+  const float tau = p.temperature ? p.temperature[r] : 1.f;
+  const float tp = p.top_p ? p.top_p[r] : 1.f;
+  const int tk = p.top_k ? p.top_k[r] : 0;
+  const bool valid = tau >= 0.f && tau != INFINITY && tp > 0.f && tp <= 1.f;
   const float st = !valid ? 0.f : (tau == 0.f ? kLog2e : kLog2e / tau);
   const float sd = (valid && tau > 0.f) ? st : 0.f;
   for (int i = 0; i <= k; ++i) p.row_scale[t0 + i] = st;
   for (int i = 0; i < k; ++i) p.row_scale[p.total_q + t0 - r + i] = sd;
+  if (p.row_req) {
+    const bool filtered = valid && tau > 0.f && ((tk >= 1 && tk < p.vocab) || tp < 1.f);
+    for (int i = 0; i <= k; ++i) p.row_req[t0 + i] = filtered ? r : -1;
+    for (int i = 0; i < k; ++i) p.row_req[p.total_q + t0 - r + i] = filtered ? r : -1;
+  }
 }
 
 // Greedy verification (tau = 0) of one request by one block: a warp finds the greedy choice of a
@@ -379,7 +587,7 @@ __global__ void row_scale_kernel(SampleParams p) {
 // Requests that are not greedy, or that the accept test reports as invalid, are left alone.
 template <typename T>
 __device__ __forceinline__ void greedy_request(const SampleParams &p, int r) {
-  if (!(p.temperature[r] == 0.f)) return;
+  if (!p.temperature || !(p.temperature[r] == 0.f)) return;
   const int t0 = p.q_indptr[r];
   const int k = p.q_indptr[r + 1] - t0 - 1;
   if (k < 0 || k > SPX_MAX_K || t0 < 0 || t0 + k + 1 > p.total_q) return;
@@ -451,7 +659,7 @@ __device__ __forceinline__ void greedy_request(const SampleParams &p, int r) {
 // merges its row's segment pairs (fp32 exponentials, float64 sum); the accept ratios of all
 // drafts are evaluated in parallel in float64 and the first failure fixes n.  Writes
 // accepted_len, the accepted ids and the -1 padding; slot n is left for resid_select_kernel.
-template <typename T, bool kScaled>
+template <typename T, bool kScaled, bool kFiltered>
 __global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_blocks) {
   if (kScaled && (int)blockIdx.x >= accept_blocks) {  // variants: one extra block per request for the greedy ones
     greedy_request<T>(p, blockIdx.x - accept_blocks);
@@ -493,8 +701,9 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_
   }
   double scale = (double)kLog2e;
   if (kScaled) {
-    const float tau = p.temperature[r];
-    if (!(tau >= 0.f) || tau == INFINITY) {
+    const float tau = p.temperature ? p.temperature[r] : 1.f;
+    const float tp = (kFiltered && p.top_p) ? p.top_p[r] : 1.f;
+    if (!(tau >= 0.f) || tau == INFINITY || !(tp > 0.f && tp <= 1.f)) {
       if (lane == 0) {
         atomicOr(p.dev_status, SPX_DEV_BAD_PARAM);
         p.accepted_len[r] = 0;
@@ -512,15 +721,21 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_
   // row normalisers: M (log2 domain) and S = sum 2^(x - M)
   float M = -INFINITY;
   double S = 0.0;
+  uint32_t thr = 0;  // filtering: order key of the row's lowest kept logit
   if (lane < 2 * k + 1) {
     const int row = lane <= k ? t0 + lane : p.total_q + d0 + (lane - k - 1);
     const float2 *st = p.seg_stats + (int64_t)row * p.nsub;
     for (int i = 0; i < p.nsub; ++i) M = fmaxf(M, st[i].x);
     for (int i = 0; i < p.nsub; ++i) S += (double)(st[i].y * fast_exp2(st[i].x - M));
+    if (kFiltered) {
+      const double z = p.row_z[row];
+      if (z >= 0.0) { S = z; thr = p.row_thresh[row]; }
+    }
   }
   // lane i < k pairs target row i (its own) with draft row i (lane k+1+i)
   const float Md = __shfl_sync(0xffffffffu, M, (k + 1 + lane) & 31);
   const double Sd = __shfl_sync(0xffffffffu, S, (k + 1 + lane) & 31);
+  const uint32_t thr_d = __shfl_sync(0xffffffffu, thr, (k + 1 + lane) & 31);
   bool reject = false;
   if (lane < k) {
     double tx, dx;
@@ -532,7 +747,15 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_
       dx = (double)(ld_as_float(draft, (int64_t)(d0 + lane) * p.row_stride + x) * kLog2e);
     }
     // rho = p(x)/q(x) = 2^(tx-Mt)/St * Sd/2^(dx-Md)
-    const double rho = exp2((tx - (double)M) - (dx - (double)Md)) * (Sd / S);
+    double rho = exp2((tx - (double)M) - (dx - (double)Md)) * (Sd / S);
+    if (kFiltered) {
+      // a drafted token outside the target's kept set is rejected; one outside the draft's own kept
+      // set (it cannot have been drafted) is accepted when the target keeps it
+      const bool p_in = order_key32(ld_as_float(target, (int64_t)(t0 + lane) * p.row_stride + x)) >= thr;
+      const bool q_in = order_key32(ld_as_float(draft, (int64_t)(d0 + lane) * p.row_stride + x)) >= thr_d;
+      if (!p_in) rho = 0.0;
+      else if (!q_in) rho = (double)INFINITY;
+    }
     reject = !((double)p.u_accept[d0 + lane] < rho);
     if (p.diag_ratio) p.diag_ratio[d0 + lane] = (float)rho;
   }
@@ -551,19 +774,30 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_
     if (n < k) p.req_norm[r] = make_float4(Mt_n, (float)(1.0 / St_n), Md_n, (float)(1.0 / Sd_n));
     else p.req_norm[r] = make_float4(Mt_n, (float)(1.0 / St_n), nanf_, 0.f);
   }
+  if (kFiltered) {
+    const uint32_t tt = __shfl_sync(0xffffffffu, thr, n);
+    const uint32_t td = __shfl_sync(0xffffffffu, thr, (k + 1 + n) & 31);
+    if (lane == 0) p.req_thresh[r] = make_uint2(tt, n < k ? td : 0u);
+  }
 }
 
 // Residual mass per segment of row n, then the final draw by the block that finishes the request
 // last (bonus requests need no residual pass: their block 0 draws at once).  grid = (nseg, B).
 // Segment choice in float64 over the segment masses, token choice by an fp32 scan of the chosen
 // segment (thread t owns tokens [32t, 32t+32) of it).
-template <typename T, bool kScaled>
+template <typename T, bool kScaled, bool kFiltered>
 __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams p) {
   const int seg_mine = blockIdx.x, r = blockIdx.y;
   const float4 nm = p.req_norm[r];
   if (nm.w < 0.f) return;  // invalid request, or a greedy one (decided beside the accept test)
   const bool bonus = (nm.z != nm.z);
-  if (bonus && seg_mine != 0) return;
+  // filtering: tokens below the row's threshold carry no mass.  A masked request always takes the
+  // full pass (the statistics of the unfiltered row are of no use to it), a bonus draw as a residual
+  // against a draft term of zero.
+  uint2 thr = make_uint2(0u, 0u);
+  if (kFiltered) thr = p.req_thresh[r];
+  const bool masked = kFiltered && (thr.x != 0u || thr.y != 0u);
+  if (bonus && !masked && seg_mine != 0) return;
   const int t0 = p.q_indptr[r];
   // the variants keep the stored logit and scale it inside one fused multiply-add with the
   // maximum (a separately rounded product would cost |x * scale| * 2^-24 of relative accuracy,
@@ -571,28 +805,51 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
   const float scale = kScaled ? p.row_scale[t0] : kLog2e;
   const float load_scale = kScaled ? 1.f : kLog2e;
   auto ex = [&](float x, float M) -> float { return kScaled ? fast_exp2(fmaf(x, scale, -M)) : fast_exp2(x - M); };
+  // probability terms of one token (xt, xd are stored logits whenever kFiltered)
+  auto pt_of = [&](float xt) -> float {
+    const float v = ex(xt, nm.x) * nm.y;
+    return (kFiltered && order_key32(xt) < thr.x) ? 0.f : v;
+  };
+  auto qd_of = [&](float xd) -> float {
+    if (kFiltered && (bonus || order_key32(xd) < thr.y)) return 0.f;
+    return ex(xd, nm.z) * nm.w;
+  };
   const int n = p.accepted_len[r];
   const T *trow = reinterpret_cast<const T *>(p.target) + (int64_t)(t0 + n) * p.row_stride;
   const T *drow = reinterpret_cast<const T *>(p.draft) + (int64_t)(t0 - r + n) * p.row_stride;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   __shared__ float s_w[kSampThreads / 32];
   __shared__ int s_last;
-  if (!bonus) {
+  __shared__ float s_wp[kSampThreads / 32];
+  if (!bonus || masked) {
     const int v0 = seg_mine * kSegElems + threadIdx.x * kElemsPerThread;
     float xt[kElemsPerThread], xd[kElemsPerThread];
     load_thread_span(trow, v0, p.vocab, xt, load_scale);
-    load_thread_span(drow, v0, p.vocab, xd, load_scale);
-    float acc = 0.f;
+    if (!bonus) load_thread_span(drow, v0, p.vocab, xd, load_scale);
+    float acc = 0.f, accp = 0.f;
 #pragma unroll
-    for (int i = 0; i < kElemsPerThread; ++i)
-      acc += fmaxf(0.f, ex(xt[i], nm.x) * nm.y - ex(xd[i], nm.z) * nm.w);
+    for (int i = 0; i < kElemsPerThread; ++i) {
+      if (kFiltered) {
+        const float pt = pt_of(xt[i]);
+        acc += fmaxf(0.f, pt - (bonus ? 0.f : qd_of(xd[i])));
+        accp += pt;
+      } else {
+        acc += fmaxf(0.f, ex(xt[i], nm.x) * nm.y - ex(xd[i], nm.z) * nm.w);
+      }
+    }
     acc = warp_sum(acc);
-    if (lane == 0) s_w[warp] = acc;
+    if (kFiltered) accp = warp_sum(accp);
+    if (lane == 0) { s_w[warp] = acc; if (kFiltered) s_wp[warp] = accp; }
     __syncthreads();
     if (threadIdx.x == 0) {
       float tot = 0.f;
       for (int w = 0; w < kSampThreads / 32; ++w) tot += s_w[w];
       p.seg_resid[(int64_t)r * p.nseg + seg_mine] = tot;
+      if (kFiltered) {
+        float totp = 0.f;
+        for (int w = 0; w < kSampThreads / 32; ++w) totp += s_wp[w];
+        p.seg_pmass[(int64_t)r * p.nseg + seg_mine] = totp;
+      }
       __threadfence();
       s_last = (atomicAdd(&p.req_done[r], 1) == p.nseg - 1);
     }
@@ -604,6 +861,7 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
   const float2 *tstats = p.seg_stats + (int64_t)(t0 + n) * p.nsub;
   // probability mass of segment i of the target row, from its sub-segment statistics
   auto target_mass = [&](int i) -> double {
+    if (masked) return (double)reinterpret_cast<const volatile float *>(p.seg_pmass)[(int64_t)r * p.nseg + i];
     double acc = 0.0;
     for (int j = i * kSubPerSeg; j < min((i + 1) * kSubPerSeg, p.nsub); ++j)
       acc += (double)(tstats[j].y * fast_exp2(tstats[j].x - nm.x));
@@ -619,11 +877,11 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
     const volatile float *resid = p.seg_resid + (int64_t)r * p.nseg;
     double R = 0.0;
     int degenerate = 0;
-    if (!bonus) {
+    if (!bonus || masked) {
       for (int i = 0; i < p.nseg; ++i) R += (double)resid[i];
       if (!(R > 0.0)) degenerate = 1;
     }
-    const bool use_target = bonus || degenerate;
+    const bool use_target = (bonus && !masked) || degenerate;
     if (use_target) {
       R = 0.0;
       for (int i = 0; i < p.nseg; ++i) R += target_mass(i);
@@ -651,22 +909,22 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
     if (threadIdx.x == 0) p.out_tokens[t0 + n] = -1;
     return;
   }
-  const bool use_target = bonus || s_degenerate;
+  const bool use_target = (bonus && !masked) || s_degenerate;
   const float target = s_target;
   const int v0 = seg * kSegElems + threadIdx.x * kElemsPerThread;
   float w[kElemsPerThread];
   {
     float xt[kElemsPerThread];
     load_thread_span(trow, v0, p.vocab, xt, load_scale);
-    if (use_target) {
+    if (use_target || (kFiltered && bonus)) {
 #pragma unroll
-      for (int i = 0; i < kElemsPerThread; ++i) w[i] = ex(xt[i], nm.x) * nm.y;
+      for (int i = 0; i < kElemsPerThread; ++i) w[i] = kFiltered ? pt_of(xt[i]) : ex(xt[i], nm.x) * nm.y;
     } else {
       float xd[kElemsPerThread];
       load_thread_span(drow, v0, p.vocab, xd, load_scale);
 #pragma unroll
       for (int i = 0; i < kElemsPerThread; ++i)
-        w[i] = fmaxf(0.f, ex(xt[i], nm.x) * nm.y - ex(xd[i], nm.z) * nm.w);
+        w[i] = kFiltered ? fmaxf(0.f, pt_of(xt[i]) - qd_of(xd[i])) : fmaxf(0.f, ex(xt[i], nm.x) * nm.y - ex(xd[i], nm.z) * nm.w);
     }
   }
   float tsum = 0.f;

@@ -120,7 +120,7 @@ static AttnWs attn_ws_layout(const spx_attn_args_t *a) {
 }
 
 struct SampleWs {
-  size_t seg_stats, seg_resid, req_norm, req_done, row_scale, total;
+  size_t seg_stats, seg_resid, req_norm, req_done, row_scale, row_req, row_thresh, row_z, req_thresh, seg_pmass, total;
   int32_t nseg, nsub;
 };
 
@@ -151,7 +151,15 @@ static SampleWs sample_ws_layout(const spx_sample_args_t *s) {
   w.req_norm = off; off = align_up(off + sizeof(float4) * (size_t)s->batch, 256);
   w.req_done = off; off = align_up(off + sizeof(int32_t) * (size_t)s->batch, 256);
   w.row_scale = off;
-  if (s->temperature) off = align_up(off + sizeof(float) * rows, 256);
+  const bool filtered = s->top_k || s->top_p;
+  if (s->temperature || filtered) off = align_up(off + sizeof(float) * rows, 256);
+  if (filtered) {
+    w.row_req = off; off = align_up(off + sizeof(int32_t) * rows, 256);
+    w.row_thresh = off; off = align_up(off + sizeof(uint32_t) * rows, 256);
+    w.row_z = off; off = align_up(off + sizeof(double) * rows, 256);
+    w.req_thresh = off; off = align_up(off + sizeof(uint2) * (size_t)s->batch, 256);
+    w.seg_pmass = off; off = align_up(off + sizeof(float) * (size_t)s->batch * w.nseg, 256);
+  }
   w.total = off;
   return w;
 }
@@ -341,7 +349,7 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
   return e == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
 }
 
-template <typename T, bool kScaled>
+template <typename T, bool kScaled, bool kFiltered = false>
 static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream, int num_sms, int phases) {
   const int rows = p.total_q + p.total_d;
   const int n_units = rows * p.nsub;
@@ -373,9 +381,15 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
     ++t_launches;
   }
   if (phases & kPhaseTail) {
+    if constexpr (kFiltered) {
+      if (cudaFuncSetAttribute(filter_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFilterSmemBytes) != cudaSuccess)
+        return SPX_ERR_CUDA;
+      filter_rows_kernel<T><<<rows, kFilterThreads, kFilterSmemBytes, stream>>>(p);
+      ++t_launches;
+    }
     const int accept_blocks = (p.batch * 32 + 127) / 128;
-    accept_kernel<T, kScaled><<<accept_blocks + (kScaled ? p.batch : 0), 128, 0, stream>>>(p, accept_blocks);
-    resid_select_kernel<T, kScaled><<<dim3(p.nseg, p.batch), kSampThreads, 0, stream>>>(p);
+    accept_kernel<T, kScaled, kFiltered><<<accept_blocks + (kScaled ? p.batch : 0), 128, 0, stream>>>(p, accept_blocks);
+    resid_select_kernel<T, kScaled, kFiltered><<<dim3(p.nseg, p.batch), kSampThreads, 0, stream>>>(p);
     t_launches += 2;
   }
   return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
@@ -398,6 +412,17 @@ static spx_status_t launch_sampler(const spx_sample_args_t *s, unsigned char *ws
   p.req_norm = reinterpret_cast<float4 *>(ws + w.req_norm);
   p.req_done = reinterpret_cast<int32_t *>(ws + w.req_done);
   p.dev_status = dev_status;
+  if (s->top_k || s->top_p) {
+    p.temperature = s->temperature; p.top_k = s->top_k; p.top_p = s->top_p;
+    p.row_scale = reinterpret_cast<float *>(ws + w.row_scale);
+    p.row_req = reinterpret_cast<int32_t *>(ws + w.row_req);
+    p.row_thresh = reinterpret_cast<uint32_t *>(ws + w.row_thresh);
+    p.row_z = reinterpret_cast<double *>(ws + w.row_z);
+    p.req_thresh = reinterpret_cast<uint2 *>(ws + w.req_thresh);
+    p.seg_pmass = reinterpret_cast<float *>(ws + w.seg_pmass);
+    return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16, true, true>(p, stream, num_sms, phases)
+                                       : launch_sampler_t<float, true, true>(p, stream, num_sms, phases);
+  }
   if (s->temperature) {
     p.temperature = s->temperature;
     p.row_scale = reinterpret_cast<float *>(ws + w.row_scale);
@@ -498,7 +523,7 @@ spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_
 // ---- host-buffer convenience ---------------------------------------------------------------
 namespace {
 struct HostStepLayout {
-  size_t q, k, v, bt, sl, qi, out, lse, tl, dl, ids, ua, us, tau, acc, tok, status, ws, total;
+  size_t q, k, v, bt, sl, qi, out, lse, tl, dl, ids, ua, us, tau, topk, topp, acc, tok, status, ws, total;
   size_t q_bytes, kv_bytes, bt_bytes, out_bytes, lse_bytes, tl_bytes, dl_bytes, ws_bytes;
 };
 HostStepLayout host_layout(const spx_attn_args_t *a, const spx_sample_args_t *s, int64_t kv_pool_elems) {
@@ -518,7 +543,7 @@ HostStepLayout host_layout(const spx_attn_args_t *a, const spx_sample_args_t *s,
   L.q = take(L.q_bytes); L.k = take(L.kv_bytes); L.v = take(L.kv_bytes); L.bt = take(L.bt_bytes);
   L.sl = take(B * 4); L.qi = take((B + 1) * 4); L.out = take(L.out_bytes); L.lse = take(L.lse_bytes);
   L.tl = take(L.tl_bytes); L.dl = take(L.dl_bytes); L.ids = take(TD * 4); L.ua = take(TD * 4); L.us = take(B * 4);
-  L.tau = take(s->temperature ? B * 4 : 0);
+  L.tau = take(s->temperature ? B * 4 : 0); L.topk = take(s->top_k ? B * 4 : 0); L.topp = take(s->top_p ? B * 4 : 0);
   L.acc = take(B * 4); L.tok = take(TQ * 4); L.status = take(4); L.ws = take(L.ws_bytes);
   L.total = off;
   return L;
@@ -553,7 +578,7 @@ spx_status_t spx_verify_step_host(const spx_attn_args_t *attn, const spx_sample_
   h2d(L.bt, attn->block_table, L.bt_bytes); h2d(L.sl, attn->seq_lens, B * 4); h2d(L.qi, attn->q_indptr, (B + 1) * 4);
   h2d(L.tl, sample->target_logits, L.tl_bytes); h2d(L.dl, sample->draft_logits, L.dl_bytes);
   h2d(L.ids, sample->draft_token_ids, TD * 4); h2d(L.ua, sample->u_accept, TD * 4); h2d(L.us, sample->u_sample, B * 4);
-  h2d(L.tau, sample->temperature, B * 4);
+  h2d(L.tau, sample->temperature, B * 4); h2d(L.topk, sample->top_k, B * 4); h2d(L.topp, sample->top_p, B * 4);
   ok = ok && cudaMemsetAsync(d + L.status, 0, 4, stream) == cudaSuccess;
   if (!ok) return SPX_ERR_CUDA;
   spx_attn_args_t a = *attn;
@@ -567,6 +592,8 @@ spx_status_t spx_verify_step_host(const spx_attn_args_t *attn, const spx_sample_
   s.accepted_len = reinterpret_cast<int32_t *>(d + L.acc); s.out_tokens = reinterpret_cast<int32_t *>(d + L.tok);
   s.diag_ratio = nullptr;
   s.temperature = sample->temperature ? reinterpret_cast<float *>(d + L.tau) : nullptr;
+  s.top_k = sample->top_k ? reinterpret_cast<int32_t *>(d + L.topk) : nullptr;
+  s.top_p = sample->top_p ? reinterpret_cast<float *>(d + L.topp) : nullptr;
   const spx_status_t st = spx_verify_step(&a, &s, d + L.ws, L.ws_bytes, reinterpret_cast<int32_t *>(d + L.status), cuda_stream);
   if (st != SPX_OK) return st;
   d2h(attn->out, L.out, L.out_bytes); d2h(attn->lse, L.lse, L.lse_bytes);

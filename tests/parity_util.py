@@ -15,6 +15,10 @@ Tolerances (stated where they are used as well):
     then meaningless for an fp32 kernel; the class is stated in absolute probability mass instead:
     the GPU's token is tolerated iff s*R lies within 2^-22 (four fp32 ulps of unit mass, the
     resolution of p and q near 1) of the oracle's cumulative interval of that token.
+  * top-p filtering: the kept set is decided by comparing a running mass with top_p; the kernel
+    sums fp32 exponentials (exactly, in fixed point), the oracle float64 ones.  A request in which
+    some consulted row's crossing came within 1e-6 (in units of the survivors' mass) of tipping to
+    the neighbouring value is exempt as a whole, and counted.  top-k is exact (stored values).
 """
 from __future__ import annotations
 
@@ -33,6 +37,7 @@ ATTN_TOL = {
 ACCEPT_BAND = 1e-6
 CDF_BAND = 1e-6
 CDF_ABS_BAND = 2.0 ** -22       # variants only: absolute probability mass
+TOPP_BAND = 1e-6                # top-p only: margin of the crossing, in units of the survivors' mass
 
 
 def gpu_attention(b, ws=None, **kw):
@@ -83,17 +88,19 @@ class SampleReport:
     accept_near_tie: int = 0
     cdf_near_tie: int = 0
     cdf_abs_near_tie: int = 0           # requests at a temperature other than 1 only
+    topp_near_tie: int = 0              # requests whose top-p crossing was within TOPP_BAND of tipping
     hard_mismatch: List[int] = field(default_factory=list)
     accept_band_eligible: int = 0       # consulted drafts inside the accept band (oracle side)
 
 
 def check_sampling(b_cpu, acc_gpu, tok_gpu, ref: Optional[oracle.SampleResult] = None,
-                   temperature: Optional[torch.Tensor] = None) -> SampleReport:
+                   temperature: Optional[torch.Tensor] = None, top_k: Optional[torch.Tensor] = None,
+                   top_p: Optional[torch.Tensor] = None) -> SampleReport:
     """Bit-exactness of (accepted_len, out_tokens) outside the two counted near-tie classes.
     Greedy requests (temperature 0) have no near-tie class: they must match exactly."""
     if ref is None:
         ref = oracle.rejection_sample(b_cpu.target_logits, b_cpu.draft_logits, b_cpu.draft_ids, b_cpu.q_indptr,
-                                      b_cpu.u_accept, b_cpu.u_sample, temperature=temperature)
+                                      b_cpu.u_accept, b_cpu.u_sample, temperature=temperature, top_k=top_k, top_p=top_p)
     acc_gpu = acc_gpu.detach().cpu()
     tok_gpu = tok_gpu.detach().cpu()
     qi = b_cpu.q_indptr.tolist()
@@ -113,6 +120,11 @@ def check_sampling(b_cpu, acc_gpu, tok_gpu, ref: Optional[oracle.SampleResult] =
         if not tau > 0.0:
             rep.hard_mismatch.append(r)
             continue
+        if ref.margin is not None and float(ref.margin[r]) < TOPP_BAND:
+            rep.topp_near_tie += 1
+            continue
+        tk = 0 if top_k is None else int(top_k[r])
+        tp = 1.0 if top_p is None else float(top_p[r])
         upto = min(max(n_o, n_g), k - 1)
         if k > 0 and bool(near[d0:d0 + upto + 1].any()):
             rep.accept_near_tie += 1
@@ -121,14 +133,15 @@ def check_sampling(b_cpu, acc_gpu, tok_gpu, ref: Optional[oracle.SampleResult] =
                 bool((tok_gpu[t0 + n_o + 1:t1] == -1).all()):
             y_g = int(tok_gpu[t0 + n_o])
             if 0 <= y_g < b_cpu.spec.vocab:
-                cdf, R = oracle.emit_cdf(r, n_o, b_cpu.target_logits, b_cpu.draft_logits, b_cpu.q_indptr, tau=tau)
+                cdf, R = oracle.emit_cdf(r, n_o, b_cpu.target_logits, b_cpu.draft_logits, b_cpu.q_indptr, tau=tau,
+                                         top_k=tk, top_p=tp)
                 target = float(b_cpu.u_sample[r]) * R
                 lo = float(cdf[y_g - 1]) if y_g > 0 else 0.0
                 hi = float(cdf[y_g])
                 if hi > lo and lo - CDF_BAND * R <= target <= hi + CDF_BAND * R:
                     rep.cdf_near_tie += 1
                     continue
-                if tau != 1.0 and lo - CDF_ABS_BAND <= target <= hi + CDF_ABS_BAND:
+                if (tau != 1.0 or tk > 0 or tp < 1.0) and lo - CDF_ABS_BAND <= target <= hi + CDF_ABS_BAND:
                     rep.cdf_abs_near_tie += 1
                     continue
         rep.hard_mismatch.append(r)

@@ -1,0 +1,185 @@
+"""GPU parity of top-k / top-p filtered verification against the oracle.
+
+Bit-exact (accepted_len, out_tokens) outside the counted near-tie classes of parity_util (accept
+band, CDF bands, and the top-p crossing band).  top-k alone involves no floating-point decision.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import spx_workloads as W
+import paper_2609_34370_b200 as spx
+from parity_util import check_sampling
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+TOP_K = [0, 50, 1, 0, 1000, 5, 0, 20]
+TOP_P = [1.0, 1.0, 1.0, 0.9, 0.95, 0.5, 0.3, 1.0]
+TAUS = [1.0, 0.7, 1.0, 1.0, 1.3, 0.8, 0.0, 1.0]
+
+
+def _params(batch, vocab):
+    tk = torch.tensor([TOP_K[r % 8] for r in range(batch)], dtype=torch.int32)
+    tp = torch.tensor([TOP_P[r % 8] for r in range(batch)], dtype=torch.float32)
+    tau = torch.tensor([TAUS[r % 8] for r in range(batch)], dtype=torch.float32)
+    return tau, tk, tp
+
+
+def _redraft(b_cpu, tau, tk, tp, seed):
+    """Harness side: redraw the draft ids from the FILTERED draft distribution (the oracle's own
+    filtered rows serve as the generator's law; the expectation still comes from the full oracle
+    run), so that acceptance chains occur under filtering.  A few ids are left as they were, which
+    exercises drafts outside the kept sets."""
+    g = torch.Generator().manual_seed(seed)
+    ids = b_cpu.draft_ids.clone()
+    qi = b_cpu.q_indptr.tolist()
+    V = b_cpu.spec.vocab
+    for r in range(b_cpu.batch):
+        if float(tau[r]) == 0.0:
+            continue
+        d0, k = qi[r] - r, qi[r + 1] - qi[r] - 1
+        for i in range(k):
+            if torch.rand((), generator=g) < 0.85:
+                q, _, _ = oracle.filtered_row(b_cpu.draft_logits[d0 + i, :V], float(tau[r]), int(tk[r]), float(tp[r]))
+                ids[d0 + i] = int(torch.multinomial(q, 1, generator=g))
+    return dataclasses.replace(b_cpu, draft_ids=ids)
+
+
+def _run(b_cpu, tau, tk, tp, **kw):
+    b = b_cpu.to(DEV)
+    acc, tok, ratio, ws = spx.rejection_sample(b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample,
+                                               temperature=None if tau is None else tau.to(DEV),
+                                               top_k=None if tk is None else tk.to(DEV),
+                                               top_p=None if tp is None else tp.to(DEV), **kw)
+    torch.cuda.synchronize()
+    return acc, tok, ratio, ws
+
+
+def _report(name, rep):
+    print(f"\n[{name}] exact {rep.exact}/{rep.requests}, accept-near-tie {rep.accept_near_tie}, cdf-near-tie {rep.cdf_near_tie}, "
+          f"cdf-abs-near-tie {rep.cdf_abs_near_tie}, top-p-near-tie {rep.topp_near_tie}")
+
+
+@pytest.mark.parametrize("idx,vocab", [(0, None), (1, 5000), (1, 128256), (4, 40000)])
+def test_filtered_verification_matches_oracle(idx, vocab):
+    spec = W.CONFIGS[idx] if idx == 0 else W.scaled(W.CONFIGS[idx], batch=16, ctx_div=64, vocab=vocab)
+    b_cpu = W.generate(spec)
+    tau, tk, tp = _params(b_cpu.batch, spec.vocab)
+    b_cpu = _redraft(b_cpu, tau, tk, tp, seed=idx)
+    acc, tok, _, ws = _run(b_cpu, tau, tk, tp)
+    # top_k = 1 on rows whose target and draft agree on the maximum leaves a zero residual: reported, not an error
+    assert int(ws.status.item()) & ~spx.DEV_DEGENERATE == 0
+    rep = check_sampling(b_cpu, acc, tok, temperature=tau, top_k=tk, top_p=tp)
+    _report(f"{spec.name} V={spec.vocab}", rep)
+    assert not rep.hard_mismatch, rep
+    assert rep.exact + rep.topp_near_tie >= rep.requests - 2
+
+
+def test_filters_alone_and_off_switches():
+    spec = W.scaled(W.CONFIGS[1], batch=12, ctx_div=64, vocab=20000)
+    b_cpu = W.generate(spec)
+    B = b_cpu.batch
+    ones = torch.ones(B)
+    # only top_k given, only top_p given, temperature absent
+    for tk, tp in ((torch.full((B,), 40, dtype=torch.int32), None), (None, torch.full((B,), 0.8))):
+        bb = _redraft(b_cpu, ones, tk if tk is not None else torch.zeros(B, dtype=torch.int32),
+                      tp if tp is not None else ones, seed=3)
+        acc, tok, _, ws = _run(bb, None, tk, tp)
+        assert int(ws.status.item()) == 0
+        rep = check_sampling(bb, acc, tok, top_k=tk, top_p=tp)
+        assert not rep.hard_mismatch, rep
+    # values that switch the filters off give the base rule's outputs
+    b = b_cpu.to(DEV)
+    acc0, tok0, _, _ = spx.rejection_sample(b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample)
+    acc1, tok1, _, ws = _run(b_cpu, None, torch.tensor([0, -1, spec.vocab, 10 ** 6] * 3, dtype=torch.int32), ones)
+    assert int(ws.status.item()) == 0
+    rep = check_sampling(b_cpu, acc1, tok1)
+    assert not rep.hard_mismatch
+    assert torch.equal(acc0, acc1) and torch.equal(tok0, tok1)
+
+
+def test_top_k_one_equals_greedy_and_bad_top_p_is_reported():
+    spec = W.scaled(W.CONFIGS[1], batch=8, ctx_div=64, vocab=30000)
+    b_cpu = W.generate(spec)
+    B = b_cpu.batch
+    qi = b_cpu.q_indptr.tolist()
+    # drafts = the target's argmax for most positions (harness side, torch.argmax)
+    ids = b_cpu.draft_ids.clone()
+    for r in range(B):
+        for i in range(qi[r + 1] - qi[r] - 1):
+            if (r + i) % 4:
+                ids[qi[r] - r + i] = int(torch.argmax(b_cpu.target_logits[qi[r] + i, :spec.vocab].float()))
+    b_cpu = dataclasses.replace(b_cpu, draft_ids=ids)
+    tk1 = torch.ones(B, dtype=torch.int32)
+    acc, tok, _, ws = _run(b_cpu, None, tk1, None)
+    assert int(ws.status.item()) in (0, spx.DEV_DEGENERATE)
+    ref = oracle.rejection_sample(b_cpu.target_logits, b_cpu.draft_logits, b_cpu.draft_ids, b_cpu.q_indptr, b_cpu.u_accept,
+                                  b_cpu.u_sample, top_k=tk1)
+    assert torch.equal(acc.cpu(), ref.accepted_len) and torch.equal(tok.cpu(), ref.out_tokens)
+    # ... and, rows without ties for the maximum, equals greedy verification of the same drafts when the draft agrees
+    tp = torch.full((B,), 0.9)
+    tp[1], tp[4], tp[6] = 0.0, float("nan"), 1.5
+    acc2, tok2, _, ws = _run(b_cpu, None, None, tp)
+    assert int(ws.status.item()) & spx.DEV_BAD_PARAM
+    for r in (1, 4, 6):
+        assert int(acc2[r]) == 0 and bool((tok2[qi[r]:qi[r + 1]] == -1).all())
+    good = torch.full((B,), 0.9)
+    acc3, tok3, _, _ = _run(b_cpu, None, None, good)
+    for r in (0, 2, 3, 5, 7):
+        assert int(acc2[r]) == int(acc3[r]) and torch.equal(tok2[qi[r]:qi[r + 1]], tok3[qi[r]:qi[r + 1]])
+
+
+def test_ties_at_the_thresholds():
+    # coarse logits: many equal values, so the k-th value and the nucleus edge fall inside ties
+    V, VS, B, k = 3000, 3000, 6, 2
+    g = torch.Generator().manual_seed(5)
+    T = torch.randint(-6, 7, (B * (k + 1), VS), generator=g).float().mul(0.5).to(torch.bfloat16)
+    Dr = torch.randint(-6, 7, (B * k, VS), generator=g).float().mul(0.5).to(torch.bfloat16)
+    qi = torch.arange(0, (B + 1) * (k + 1), k + 1, dtype=torch.int32)
+    tk = torch.tensor([10, 300, 0, 0, 1, 2999], dtype=torch.int32)
+    tp = torch.tensor([1.0, 1.0, 0.37, 0.9, 1.0, 0.5])
+    ids = torch.zeros(B * k, dtype=torch.int32)
+    for r in range(B):
+        for i in range(k):
+            q, _, _ = oracle.filtered_row(Dr[r * k + i], 1.0, int(tk[r]), float(tp[r]))
+            ids[r * k + i] = int(torch.multinomial(q, 1, generator=g))
+    ua, us = torch.rand(B * k, generator=g), torch.rand(B, generator=g)
+    ref = oracle.rejection_sample(T, Dr, ids, qi, ua, us, top_k=tk, top_p=tp)
+    acc, tok, _, ws = spx.rejection_sample(T.to(DEV), Dr.to(DEV), ids.to(DEV), qi.to(DEV), ua.to(DEV), us.to(DEV),
+                                           top_k=tk.to(DEV), top_p=tp.to(DEV))
+    torch.cuda.synchronize()
+
+    class _B:
+        pass
+    bb = _B()
+    bb.batch, bb.q_indptr, bb.u_accept, bb.u_sample = B, qi, ua, us
+    bb.target_logits, bb.draft_logits, bb.draft_ids = T, Dr, ids
+    bb.spec = type("S", (), {"vocab": V})
+    rep = check_sampling(bb, acc, tok, ref, top_k=tk, top_p=tp)
+    _report("ties", rep)
+    assert not rep.hard_mismatch, (rep, acc.cpu().tolist(), ref.accepted_len.tolist())
+    # every emitted token lies inside the oracle's kept set of its row
+    for r in range(B):
+        n = int(acc[r])
+        y = int(tok[r * (k + 1) + n])
+        p, _, _ = oracle.filtered_row(T[r * (k + 1) + n], 1.0, int(tk[r]), float(tp[r]))
+        assert float(p[y]) > 0.0 or float(ref.margin[r]) < 1e-6
+
+
+def test_full_size_filtered():
+    spec = W.CONFIGS[1]
+    b_cpu = W.generate(spec)
+    tau, tk, tp = _params(b_cpu.batch, spec.vocab)
+    b_cpu = _redraft(b_cpu, tau, tk, tp, seed=11)
+    acc, tok, _, ws = _run(b_cpu, tau, tk, tp)
+    assert int(ws.status.item()) & ~spx.DEV_DEGENERATE == 0
+    rep = check_sampling(b_cpu, acc, tok, temperature=tau, top_k=tk, top_p=tp)
+    _report("llama3-8b, mixed filters", rep)
+    assert not rep.hard_mismatch, rep
+    # repeated launches agree bit for bit (integer atomics: no dependence on the order of arrival)
+    for _ in range(2):
+        acc2, tok2, _, _ = _run(b_cpu, tau, tk, tp)
+        assert torch.equal(acc, acc2) and torch.equal(tok, tok2)
