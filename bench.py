@@ -226,6 +226,16 @@ def time_extras(spx, binding, spec, b, attn_args, dev, iters: int = 200):
         ws.ensure(spx.workspace_size(attn_args, sv))
         out[f"sample_tau_{name}_us"] = timed(sample_call(sv))
         out[f"step_tau_{name}_us"] = timed(lambda: spx.verify_step(attn_args, sv, ws, dev))
+    # top-k / top-p filtered verification (every request filtered)
+    for name, tk_v, tp_v in (("topk50", 50, 1.0), ("topp0.9", 0, 0.9), ("topk50_topp0.9", 50, 0.9)):
+        tk_d = torch.full((b.batch,), tk_v, dtype=torch.int32, device=dev)
+        tp_d = torch.full((b.batch,), tp_v, dtype=torch.float32, device=dev)
+        sv = binding.make_sample_args(b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample,
+                                      acc, tok, None, None, None, tk_d, tp_d)
+        ws.ensure(spx.workspace_size(attn_args, sv))
+        out[f"sample_{name}_us"] = timed(sample_call(sv))
+        out[f"step_{name}_us"] = timed(lambda: spx.verify_step(attn_args, sv, ws, dev))
+    ws.status.bitwise_and_(~spx.DEV_DEGENERATE)
     # selective-speculation support and Algorithm 1
     cws = spx.Workspace.allocate(1 << 20, dev)
     out["draft_confidence_us"] = timed(lambda: spx.draft_confidence(b.draft_logits, b.draft_ids, b.q_indptr, ws=cws))

@@ -370,32 +370,79 @@ __device__ __forceinline__ uint32_t order_key32(float f) {
 
 // top-k / top-p thresholds of one logits row per block (kFilterThreads threads).
 //
-// The kept set is {v : key(x_v) >= T}.  T is found by a byte-wise radix descent from the top of
-// the key space: each level builds a 256-bin histogram (count, mass) of the elements that match
-// the prefix chosen so far and warp 0 picks the bin where the running count reaches top_k, or the
-// running mass reaches top_p times the survivors' mass.  Masses are sums of 2^(x*scale - M) in
-// 2^-44 fixed point: integer atomics make every sum exact and independent of the order of
-// arrival, so the result is reproducible and the cumulative mass at the top-k threshold equals
-// the survivors' mass bit for bit.  Histograms are private to each warp (shared-memory atomics
-// only collide inside a warp) and summed per level.  bf16 keys have 16 significant bits (2
-// levels), fp32 keys 32 (4 levels).  After the first pass the row is re-read out of L2.
+// The kept set is {v : key(x_v) >= T}.  T is found by a descent from the top, level by level; each
+// level is a 256-bin histogram (count, mass) of the elements still in play, and warp 0 picks the
+// bin where the running count reaches top_k, or the running mass reaches top_p times the survivors'
+// mass.
+//   Level 0 sweeps the whole row and bins every element by its distance below the row maximum in
+//   logit units, 1/8 unit per bin (bin = 255 - min(255, floor(8 (max - x))), monotone in x).  The
+//   leading byte of a float is the same for almost every logit of a row, so a histogram on key
+//   bytes would serialise the shared-memory atomics on a handful of addresses; the distance spreads
+//   a row over dozens of bins, and every lane of a warp owns its own copy of the histogram
+//   (hist[bin][lane]: one bank per lane, no replays inside a warp).  A mass is added as three
+//   15-bit pieces with 32-bit atomics (a copy sees at most vocab/32 elements, no piece overflows;
+//   64-bit shared-memory atomics are far slower).  Counts are kept only for a top-k descent,
+//   masses only for a top-p descent.
+//   One more sweep collects the elements of the chosen level-0 bin (a few hundred, typically) into
+//   shared memory, and the remaining levels walk their exact key bytes (2 for bf16, 4 for fp32)
+//   over that list.  A bin too crowded for the list (a row of equal values, a mass of masked
+//   tokens in the last bin) is walked with sweeps over the row instead: slower, same result.
+// Masses are sums of 2^(x*scale - M) in 2^-44 fixed point: integer arithmetic makes every sum exact
+// and independent of the order of arrival, so the result is reproducible and the cumulative mass
+// at the top-k threshold equals the survivors' mass bit for bit.  After the first sweep the row
+// comes out of L2.
 constexpr int kFilterThreads = 1024;
+constexpr int kFilterUnroll = 4;   // 16-byte loads in flight per thread: one block per SM has to cover the latency alone
 constexpr int kFilterWarps = kFilterThreads / 32;
+constexpr int kFilterListCap = 12288;
 constexpr float kMassScale = 17592186044416.f;  // 2^44
-constexpr int kFilterSmemBytes = kFilterWarps * 256 * (8 + 4) + 256 * (8 + 4) * 2 + 64;
+constexpr int kFilterSmemBytes = 4 * 256 * 32 * 4 + 256 * (8 + 4) * 2 + kFilterListCap * 4 + 64;
+
+// Calls f(x) for every element of a row; the block's threads stride over 16-byte vectors and keep
+// kFilterUnroll of them in flight.
+template <typename T, typename F>
+__device__ __forceinline__ void sweep_row(const T *base, int vocab, int tid, F f) {
+  constexpr int N = Vec<T>::N;
+  constexpr int stride = kFilterThreads * N;
+  int v = tid * N;
+  for (; v + (kFilterUnroll - 1) * stride + N <= vocab; v += kFilterUnroll * stride) {
+    uint4 raw[kFilterUnroll];
+#pragma unroll
+    for (int u = 0; u < kFilterUnroll; ++u) raw[u] = __ldg(reinterpret_cast<const uint4 *>(base + v + u * stride));
+#pragma unroll
+    for (int u = 0; u < kFilterUnroll; ++u) {
+      union { uint4 q; T e[N]; } tmp;
+      tmp.q = raw[u];
+#pragma unroll
+      for (int i = 0; i < N; ++i) f(ld_as_float(tmp.e, i));
+    }
+  }
+  for (; v < vocab; v += stride) {
+    if (v + N <= vocab) {
+      union { uint4 q; T e[N]; } tmp;
+      tmp.q = __ldg(reinterpret_cast<const uint4 *>(base + v));
+#pragma unroll
+      for (int i = 0; i < N; ++i) f(ld_as_float(tmp.e, i));
+    } else {
+      for (int i = 0; i < N && v + i < vocab; ++i) f(ld_as_float(base, v + i));
+    }
+  }
+}
 
 template <typename T>
 __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SampleParams p) {
   extern __shared__ __align__(16) unsigned char fsm[];
-  unsigned long long *w_mass = reinterpret_cast<unsigned long long *>(fsm);                    // [warps][256]
-  unsigned long long *s_mass = w_mass + kFilterWarps * 256;                                    // [256] level sums
-  unsigned long long *s_mass1 = s_mass + 256;                                                  // [256] level-1 copy
-  uint32_t *w_cnt = reinterpret_cast<uint32_t *>(s_mass1 + 256);                               // [warps][256]
-  uint32_t *s_cnt = w_cnt + kFilterWarps * 256;
+  unsigned long long *s_mass = reinterpret_cast<unsigned long long *>(fsm);                    // [256] level sums
+  unsigned long long *s_mass1 = s_mass + 256;                                                  // [256] level-0 copy
+  uint32_t *h_cnt = reinterpret_cast<uint32_t *>(s_mass1 + 256);                               // [256][lane]
+  uint32_t *h_m0 = h_cnt + 256 * 32;                                                           // mass bits 0..14
+  uint32_t *h_m1 = h_m0 + 256 * 32;                                                            // mass bits 15..29
+  uint32_t *h_m2 = h_m1 + 256 * 32;                                                            // mass bits 30..44
+  uint32_t *s_cnt = h_m2 + 256 * 32;
   uint32_t *s_cnt1 = s_cnt + 256;
-  __shared__ uint32_t s_bin;
+  float *s_list = reinterpret_cast<float *>(s_cnt1 + 256);                                     // [kFilterListCap]
+  __shared__ uint32_t s_bin, s_above_cnt, s_list_n;
   __shared__ unsigned long long s_above_mass, s_bin_mass;
-  __shared__ uint32_t s_above_cnt;
   const int row = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int r = p.row_req[row];
@@ -403,14 +450,14 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
     if (tid == 0) { p.row_thresh[row] = 0; p.row_z[row] = -1.0; }
     return;
   }
-  constexpr int kLevels = sizeof(T) == 2 ? 2 : 4;
-  constexpr int kKeyShift = sizeof(T) == 2 ? 16 : 0;  // bf16: the low 16 bits of the fp32 key are zero
-  constexpr int N = Vec<T>::N;
+  constexpr int kLevels = sizeof(T) == 2 ? 2 : 4;      // exact key bytes after level 0
+  constexpr int kKeyShift = sizeof(T) == 2 ? 16 : 0;   // bf16: the low 16 bits of the fp32 key carry nothing
   const int tk_raw = p.top_k ? p.top_k[r] : 0;
   const bool use_k = tk_raw >= 1 && tk_raw < p.vocab;
   const float tp = p.top_p ? p.top_p[r] : 1.f;
   const bool use_p = tp < 1.f;
   const float scale = p.row_scale[row];
+  const float inv_w = 8.f / scale;   // distance in log2 units -> eighths of a logit unit
   const T *base = row < p.total_q ? reinterpret_cast<const T *>(p.target) + (int64_t)row * p.row_stride
                                   : reinterpret_cast<const T *>(p.draft) + (int64_t)(row - p.total_q) * p.row_stride;
   float M = -INFINITY;
@@ -418,42 +465,40 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
     const float2 *st = p.seg_stats + (int64_t)row * p.nsub;
     for (int j = 0; j < p.nsub; ++j) M = fmaxf(M, st[j].x);
   }
-
-  // one histogram pass: elements whose key matches `prefix` in the bits above `shift + 8`
-  auto hist_pass = [&](uint32_t prefix, int level) {
-    const int shift = kKeyShift + 8 * (kLevels - 1 - level);
-    for (int i = tid; i < kFilterWarps * 256; i += kFilterThreads) { w_cnt[i] = 0; w_mass[i] = 0ull; }
-    __syncthreads();
-    uint32_t *my_cnt = w_cnt + warp * 256;
-    unsigned long long *my_mass = w_mass + warp * 256;
-    auto add = [&](float x) {
-      const uint32_t key = order_key32(x);
-      if (level > 0 && (key >> (shift + 8)) != (prefix >> (shift + 8))) return;
-      const uint32_t bin = (key >> shift) & 255u;
-      atomicAdd(&my_cnt[bin], 1u);
-      const float e = fast_exp2(fmaf(x, scale, -M));
-      atomicAdd(&my_mass[bin], __float2ull_rn(e * kMassScale));
-    };
-    for (int v = tid * N; v < p.vocab; v += kFilterThreads * N) {
-      if (v + N <= p.vocab) {
-        union { uint4 u; T e[N]; } tmp;
-        tmp.u = __ldg(reinterpret_cast<const uint4 *>(base + v));
-#pragma unroll
-        for (int i = 0; i < N; ++i) add(ld_as_float(tmp.e, i));
-      } else {
-        for (int i = 0; i < N && v + i < p.vocab; ++i) add(ld_as_float(base, v + i));
-      }
-    }
-    __syncthreads();
-    if (tid < 256) {
-      uint32_t c = 0;
-      unsigned long long m = 0ull;
-      for (int w = 0; w < kFilterWarps; ++w) { c += w_cnt[w * 256 + tid]; m += w_mass[w * 256 + tid]; }
-      s_cnt[tid] = c;
-      s_mass[tid] = m;
-    }
-    __syncthreads();
+  auto bin0_of = [&](float x) -> uint32_t {
+    const float d = fmaxf(fmaf(x, -scale, M), 0.f) * inv_w;
+    return 255u - (uint32_t)fminf(d, 255.f);
   };
+  auto mass_of = [&](float x) -> unsigned long long { return __float2ull_rn(fast_exp2(fmaf(x, scale, -M)) * kMassScale); };
+
+  // level 0: the whole row into the per-lane copies, then their sums into s_cnt / s_mass
+  for (int i = tid; i < 4 * 256 * 32; i += kFilterThreads) h_cnt[i] = 0;   // the four arrays are contiguous
+  __syncthreads();
+  sweep_row<T>(base, p.vocab, tid, [&](float x) {
+    const uint32_t slot = bin0_of(x) * 32 + lane;
+    if (use_k) atomicAdd(&h_cnt[slot], 1u);
+    if (use_p) {
+      const unsigned long long m = mass_of(x);
+      atomicAdd(&h_m0[slot], (uint32_t)(m & 0x7fffull));
+      atomicAdd(&h_m1[slot], (uint32_t)((m >> 15) & 0x7fffull));
+      atomicAdd(&h_m2[slot], (uint32_t)(m >> 30));
+    }
+  });
+  __syncthreads();
+  if (tid < 256) {
+    uint32_t c = 0;
+    unsigned long long m = 0ull;
+    for (int j = 0; j < 32; ++j) {
+      const int slot = tid * 32 + ((j + tid) & 31);
+      c += h_cnt[slot];
+      m += (unsigned long long)h_m0[slot] + ((unsigned long long)h_m1[slot] << 15) + ((unsigned long long)h_m2[slot] << 30);
+    }
+    s_cnt[tid] = s_cnt1[tid] = c;
+    s_mass[tid] = s_mass1[tid] = m;
+  }
+  __syncthreads();
+  unsigned long long total = 0ull;
+  for (int b = 0; b < 256; ++b) total += s_mass1[b];   // every thread: 256 broadcast reads
 
   // warp 0: the highest bin b such that (count or mass of bins >= b, plus what lies above the
   // prefix) reaches the target; leaves the bin, and count / mass of the bins above it, in shared memory
@@ -488,7 +533,7 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
         }
         if (chosen < 0) {  // only without a crossing: lowest occupied bin of the whole level
           cc = 0; mm = 0ull; chosen = 0;
-          for (int bb = 255; bb >= 0; --bb) if (s_cnt[bb]) chosen = bb;
+          for (int bb = 255; bb >= 0; --bb) if (s_cnt[bb] || s_mass[bb]) chosen = bb;
           for (int bb = 255; bb > chosen; --bb) { cc += s_cnt[bb]; mm += s_mass[bb]; }
         }
         s_bin = (uint32_t)chosen;
@@ -500,54 +545,76 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
     __syncthreads();
   };
 
-  // level 0 serves both descents
-  hist_pass(0u, 0);
-  if (tid < 256) { s_cnt1[tid] = s_cnt[tid]; s_mass1[tid] = s_mass[tid]; }
-  __syncthreads();
-  unsigned long long total = 0ull;
-  for (int b = 0; b < 256; ++b) total += s_mass1[b];   // every thread: 256 broadcast reads
-
-  uint32_t Tk = 0;
-  unsigned long long Zk = total;
-  if (use_k) {
-    uint32_t prefix = 0, need = (uint32_t)tk_raw;
-    unsigned long long above = 0ull;
-    for (int level = 0; level < kLevels; ++level) {
-      if (level > 0) hist_pass(prefix, level);
-      pick(true, need, 0.0, 0ull);
-      const int shift = kKeyShift + 8 * (kLevels - 1 - level);
+  // One descent.  On entry s_cnt / s_mass hold level 0.  Returns the threshold key; *Z receives the
+  // mass at or above it (meaningful only when masses were kept at level 0, i.e. use_p).
+  auto descend = [&](bool by_count, uint32_t need, double need_mass, unsigned long long *Z) -> uint32_t {
+    pick(by_count, need, need_mass, 0ull);
+    const uint32_t b0 = s_bin;
+    need -= s_above_cnt;
+    unsigned long long above = s_above_mass;
+    __syncthreads();
+    // the elements of bin b0, into shared memory if they fit
+    if (tid == 0) s_list_n = 0;
+    __syncthreads();
+    sweep_row<T>(base, p.vocab, tid, [&](float x) {
+      if (bin0_of(x) != b0) return;
+      const uint32_t i = atomicAdd(&s_list_n, 1u);
+      if (i < (uint32_t)kFilterListCap) s_list[i] = x;
+    });
+    __syncthreads();
+    const uint32_t n_list = s_list_n;
+    const bool listed = n_list <= (uint32_t)kFilterListCap;
+    uint32_t prefix = 0;
+    for (int level = 1; level <= kLevels; ++level) {
+      const int shift = kKeyShift + 8 * (kLevels - level);
+      if (tid < 256) { s_cnt[tid] = 0; s_mass[tid] = 0ull; }
+      __syncthreads();
+      auto add = [&](float x) {
+        const uint32_t key = order_key32(x);
+        if (level > 1 && (key >> (shift + 8)) != (prefix >> (shift + 8))) return;
+        const uint32_t bin = (key >> shift) & 255u;
+        atomicAdd(&s_cnt[bin], 1u);
+        atomicAdd(&s_mass[bin], mass_of(x));
+      };
+      if (listed) {
+        for (uint32_t i = tid; i < n_list; i += kFilterThreads) add(s_list[i]);
+      } else {
+        sweep_row<T>(base, p.vocab, tid, [&](float x) { if (bin0_of(x) == b0) add(x); });
+      }
+      __syncthreads();
+      pick(by_count, need, need_mass, above);
       prefix |= s_bin << shift;
       need -= s_above_cnt;
       above += s_above_mass;
-      if (level == kLevels - 1) Zk = above + s_bin_mass;
+      if (level == kLevels) *Z = above + s_bin_mass;
       __syncthreads();
     }
-    Tk = prefix;
-  }
+    return prefix;
+  };
+
+  uint32_t Tk = 0;
+  unsigned long long Zk = total;
+  if (use_k) Tk = descend(true, (uint32_t)tk_raw, 0.0, &Zk);
   uint32_t Tf = Tk;
   unsigned long long Zf = Zk;
   if (use_p) {
-    const double need_mass = (double)tp * (double)Zk;
-    uint32_t prefix = 0;
-    unsigned long long above = 0ull;
-    for (int level = 0; level < kLevels; ++level) {
-      if (level == 0) {
-        if (use_k) {  // the level-0 histogram was overwritten by the top-k descent: restore it
-          if (tid < 256) { s_cnt[tid] = s_cnt1[tid]; s_mass[tid] = s_mass1[tid]; }
-          __syncthreads();
-        }
-      } else {
-        hist_pass(prefix, level);
-      }
-      pick(false, 0u, need_mass, above);
-      const int shift = kKeyShift + 8 * (kLevels - 1 - level);
-      prefix |= s_bin << shift;
-      above += s_above_mass;
-      if (level == kLevels - 1) Zf = above + s_bin_mass;
+    if (use_k) {  // level 0 again (the top-k descent reused the arrays)
+      if (tid < 256) { s_cnt[tid] = s_cnt1[tid]; s_mass[tid] = s_mass1[tid]; }
       __syncthreads();
     }
-    Tf = prefix;
+    Tf = descend(false, 0u, (double)tp * (double)Zk, &Zf);
     if (Tf < Tk) { Tf = Tk; Zf = Zk; }  // cannot happen with exact sums; keeps the sets nested regardless
+  } else {
+    // top-k alone kept only counts at level 0: one more sweep adds up the kept mass in registers
+    unsigned long long acc = 0ull;
+    sweep_row<T>(base, p.vocab, tid, [&](float x) { if (order_key32(x) >= Tf) acc += mass_of(x); });
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    __syncthreads();
+    if (lane == 0) s_mass[warp] = acc;
+    __syncthreads();
+    Zf = 0ull;
+    for (int w = 0; w < kFilterWarps; ++w) Zf += s_mass[w];
   }
   if (tid == 0) {
     p.row_thresh[row] = Tf;

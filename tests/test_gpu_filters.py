@@ -169,6 +169,42 @@ def test_ties_at_the_thresholds():
         assert float(p[y]) > 0.0 or float(ref.margin[r]) < 1e-6
 
 
+def test_crowded_threshold_bin():
+    # tens of thousands of tokens share the value at which top-k / top-p cut (a block of equal logits, and a mass
+    # of "masked" tokens far below the maximum): more than the kernel can park on chip, so it walks the row instead
+    V, B, k = 60000, 4, 1
+    g = torch.Generator().manual_seed(9)
+    T = (torch.randn(B * (k + 1), V, generator=g) * 2).to(torch.bfloat16)
+    Dr = (torch.randn(B * k, V, generator=g) * 2).to(torch.bfloat16)
+    for rows in (T, Dr):
+        rows[:, 5000:35000] = 1.0            # 30000 equal logits
+        rows[:, 40000:] = -200.0             # 20000 masked tokens, all in the last distance bin
+    qi = torch.arange(0, (B + 1) * (k + 1), k + 1, dtype=torch.int32)
+    tk = torch.tensor([20000, 0, 45000, 50000], dtype=torch.int32)
+    tp = torch.tensor([1.0, 0.6, 0.97, 1.0])
+    ids = torch.zeros(B * k, dtype=torch.int32)
+    for r in range(B):
+        q, kept, _ = oracle.filtered_row(Dr[r], 1.0, int(tk[r]), float(tp[r]))
+        ids[r] = int(torch.multinomial(q, 1, generator=g))
+    assert oracle.filtered_row(T[0], 1.0, 20000, 1.0)[1] > 30000      # the whole tie is kept
+    assert oracle.filtered_row(T[3 * 2], 1.0, 50000, 1.0)[1] == V     # cut inside the masked block: all of it kept
+    ua, us = torch.rand(B * k, generator=g), torch.rand(B, generator=g)
+    ref = oracle.rejection_sample(T, Dr, ids, qi, ua, us, top_k=tk, top_p=tp)
+    acc, tok, _, ws = spx.rejection_sample(T.to(DEV), Dr.to(DEV), ids.to(DEV), qi.to(DEV), ua.to(DEV), us.to(DEV),
+                                           top_k=tk.to(DEV), top_p=tp.to(DEV))
+    torch.cuda.synchronize()
+
+    class _B:
+        pass
+    bb = _B()
+    bb.batch, bb.q_indptr, bb.u_accept, bb.u_sample = B, qi, ua, us
+    bb.target_logits, bb.draft_logits, bb.draft_ids = T, Dr, ids
+    bb.spec = type("S", (), {"vocab": V})
+    rep = check_sampling(bb, acc, tok, ref, top_k=tk, top_p=tp)
+    _report("crowded bin", rep)
+    assert not rep.hard_mismatch, (rep, acc.cpu().tolist(), ref.accepted_len.tolist(), ref.margin.tolist())
+
+
 def test_full_size_filtered():
     spec = W.CONFIGS[1]
     b_cpu = W.generate(spec)
