@@ -271,6 +271,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--extras", action="store_true",
                     help="also time the pieces around the step: KV append / rollback, verification variants")
+    ap.add_argument("--extras-iters", type=int, default=200, help="timed calls per extras entry (profiling runs: a few)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling captures of a smaller case)")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -362,7 +363,7 @@ def main():
 
     extras = None
     if args.extras and rank == 0:
-        extras = time_extras(spx, binding, spec, b, a, dev)
+        extras = time_extras(spx, binding, spec, b, a, dev, iters=args.extras_iters)
 
     # ---- end to end through the host-buffer entry point (every rank, max time) ----
     b_host = None
