@@ -437,3 +437,21 @@ def filtered_row(logits_row: torch.Tensor, tau: float = 1.0, top_k: int = 0, top
     kept = lib.oracle_filtered_row(_ptr(row), _dtype_code(row), 0, V, float(tau), int(top_k), float(top_p), _ptr(p),
                                    _ptr(scratch), c.byref(m))
     return p, int(kept), float(m.value)
+
+
+def lm_head(hidden: torch.Tensor, weight: torch.Tensor, v_begin: int = 0, v_end: Optional[int] = None) -> torch.Tensor:
+    """logits[:, v_begin:v_end] = hidden @ weight[v_begin:v_end].T in float64 (plain loops)."""
+    lib = _load()
+    h = _cpu(hidden).contiguous()
+    w = _cpu(weight).contiguous()
+    assert h.dim() == 2 and w.dim() == 2 and h.shape[1] == w.shape[1] and _dtype_code(h) == _dtype_code(w)
+    V = w.shape[0]
+    v_end = V if v_end is None else int(v_end)
+    out = torch.empty((h.shape[0], v_end - int(v_begin)), dtype=torch.float64)
+    lib.oracle_lm_head.restype = c.c_int
+    lib.oracle_lm_head.argtypes = [c.c_int32, c.c_int32, c.c_int64, c.c_int32, c.c_void_p, c.c_void_p, c.c_int64, c.c_int64,
+                                   c.c_void_p]
+    st = lib.oracle_lm_head(h.shape[0], h.shape[1], V, _dtype_code(h), _ptr(h), _ptr(w), int(v_begin), v_end, _ptr(out))
+    if st != OK:
+        raise OracleError(st)
+    return out

@@ -49,7 +49,8 @@
  * Appendix A.1-A.3) conservation s^a + s^r + n = B, the recurrences' limits against the closed
  * forms, G against throughput ratios built from the token counts and times of Appendix A.3, and
  * Algorithm 1 against scipy's binomial pmf, its closed forms at pp = 1 and theta = 1, and a
- * Python brute force.
+ * Python brute force; for the LM head (tests/test_oracle_lm_head.py) torch's float64 matmul,
+ * identity / one-hot weights, linearity, and integer inputs whose products are exact.
  */
 #include <math.h>
 #include <stdint.h>
@@ -823,6 +824,34 @@ int oracle_lookahead_memory(int32_t nreq, const int32_t *ell, const int32_t *tau
     }
     M[i - 1] = L_total + ((double)nreq - E_nfin) * E_gen - E_lfin;
   }
+  return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* (G) LM head: the logits the sampling half consumes                                    */
+/* ------------------------------------------------------------------------------------ */
+
+/*
+ * logits[m][v] = sum_k H[m][k] W[v][k] for the M new positions' final hidden states H [M, K] and
+ * the vocabulary projection W [V, K], both stored row-major in `dtype`; float64 products and a
+ * plain left-to-right sum over k.  (Section 6 places the LM head on the stage that verifies; the
+ * paper gives no formula beyond that: this is the definition of a linear layer without bias.)
+ * Only the columns [v_begin, v_end) are computed (a full-size check samples column blocks);
+ * out is [M][v_end - v_begin] doubles.
+ */
+int oracle_lm_head(int32_t M, int32_t K, int64_t V, int32_t dtype, const void *H, const void *W,
+                   int64_t v_begin, int64_t v_end, double *out) {
+  if (M < 0 || K <= 0 || V <= 0 || v_begin < 0 || v_end > V || v_begin > v_end) return ORACLE_ERR_ARG;
+  if (dtype != ORACLE_BF16 && dtype != ORACLE_F32) return ORACLE_ERR_ARG;
+  const int64_t nv = v_end - v_begin;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int m = 0; m < M; ++m)
+    for (int64_t v = 0; v < nv; ++v) {
+      double acc = 0.0;
+      for (int k = 0; k < K; ++k)
+        acc += widen(H, dtype, (int64_t)m * K + k) * widen(W, dtype, (v_begin + v) * K + k);
+      out[(int64_t)m * nv + v] = acc;
+    }
   return ORACLE_OK;
 }
 
