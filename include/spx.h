@@ -156,6 +156,7 @@ typedef struct {
   const float *temperature;    /* optional [B]: see "Verification variants"; NULL = all 1     */
   const int32_t *top_k;        /* optional [B]                                                */
   const float *top_p;          /* optional [B]                                                */
+  const float *target_tile_stats; /* optional: spx_lm_head's tile_stats of the target rows    */
 } spx_sample_args_t;
 
 /*
@@ -285,6 +286,32 @@ double spx_selective_batch(double batch, int32_t stages, double alpha);
 double spx_selective_effective_batch(double batch, int32_t stages, double alpha, double theta_alpha);
 double spx_delay_gain(double iterations, int32_t n_evictions, double pdr, double running, double i_delay,
                       const double *i_wait /* host, [n_evictions] */);
+
+/*
+ * LM head with the sampling half's statistics fused into its epilogue (the paper's Section 6
+ * keeps an LM head on the stage that verifies; the step's target logits are its output):
+ *   logits[m][v] = sum_k hidden[m][k] * weight[v][k],  m < rows, v < vocab,
+ * bf16 operands, fp32 accumulation on the tensor cores, result rounded to bf16 (nearest even) and
+ * stored at logits[m * logits_row_stride + v].  hidden is [rows, hidden_dim] and weight is
+ * [vocab, hidden_dim], both row-major and dense; all device pointers, 16-byte aligned;
+ * hidden_dim and logits_row_stride multiples of 8.  tile_stats (optional) receives, for every row
+ * and every block of 256 vocabulary columns, (max * log2 e, sum_v 2^((x_v - max) log2 e)) of the
+ * values AS STORED: [rows][ceil(vocab / 256)] pairs of floats.  Passed as
+ * spx_sample_args_t.target_tile_stats they replace the sampling half's own read of the target
+ * logits for its statistics (temperature 1, no filters; ignored otherwise).
+ * Errors: SPX_ERR_INVALID_ARG / SPX_ERR_UNSUPPORTED for bad shapes or alignment; a bounded wait
+ * that expires inside the kernel sets SPX_DEV_TIMEOUT.
+ */
+typedef struct {
+  int32_t rows, hidden_dim, vocab;
+  const void *hidden;          /* [rows, hidden_dim] bf16                                      */
+  const void *weight;          /* [vocab, hidden_dim] bf16                                     */
+  void *logits;                /* [rows, logits_row_stride] bf16, written                      */
+  int64_t logits_row_stride;   /* elements                                                     */
+  float *tile_stats;           /* optional [rows][ceil(vocab/256)][2], written                 */
+} spx_lm_head_args_t;
+
+spx_status_t spx_lm_head(const spx_lm_head_args_t *args, int32_t *dev_status, void *cuda_stream);
 
 /*
  * Convenience for callers whose data lives on the HOST: every pointer in the two structs is a

@@ -19,7 +19,7 @@ EXPORTS = ("spx_workspace_size", "spx_verify_attention", "spx_rejection_sample",
            "spx_set_timing_events", "spx_rejection_sample_static", "spx_kv_append", "spx_kv_rollback",
            "spx_draft_confidence_workspace", "spx_draft_confidence", "spx_select_speculation",
            "spx_lookahead_memory", "spx_sp_effective_batch", "spx_selective_batch", "spx_selective_effective_batch",
-           "spx_delay_gain")
+           "spx_delay_gain", "spx_lm_head")
 
 
 class AttnArgs(C.Structure):
@@ -42,7 +42,7 @@ class SampleArgs(C.Structure):
         ("target_logits", C.c_void_p), ("draft_logits", C.c_void_p), ("draft_token_ids", C.c_void_p),
         ("q_indptr", C.c_void_p), ("u_accept", C.c_void_p), ("u_sample", C.c_void_p),
         ("accepted_len", C.c_void_p), ("out_tokens", C.c_void_p), ("diag_ratio", C.c_void_p),
-        ("temperature", C.c_void_p), ("top_k", C.c_void_p), ("top_p", C.c_void_p),
+        ("temperature", C.c_void_p), ("top_k", C.c_void_p), ("top_p", C.c_void_p), ("target_tile_stats", C.c_void_p),
     ]
 
 
@@ -63,6 +63,14 @@ class ConfArgs(C.Structure):
         ("logits_dtype", C.c_int),
         ("draft_logits", C.c_void_p), ("draft_token_ids", C.c_void_p), ("q_indptr", C.c_void_p),
         ("conf_max", C.c_void_p), ("conf_tok", C.c_void_p), ("req_conf", C.c_void_p),
+    ]
+
+
+class LmHeadArgs(C.Structure):
+    _fields_ = [
+        ("rows", C.c_int32), ("hidden_dim", C.c_int32), ("vocab", C.c_int32),
+        ("hidden", C.c_void_p), ("weight", C.c_void_p), ("logits", C.c_void_p), ("logits_row_stride", C.c_int64),
+        ("tile_stats", C.c_void_p),
     ]
 
 
@@ -126,6 +134,8 @@ def load_library():
             fn.argtypes = [C.c_double, C.c_int32, C.c_double] + [C.c_double] * nargs
         lib.spx_delay_gain.restype = C.c_double
         lib.spx_delay_gain.argtypes = [C.c_double, C.c_int32, C.c_double, C.c_double, C.c_double, C.POINTER(C.c_double)]
+        lib.spx_lm_head.restype = C.c_int
+        lib.spx_lm_head.argtypes = [C.POINTER(LmHeadArgs), C.c_void_p, C.c_void_p]
         lib.spx_set_timing_events.restype = None
         lib.spx_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
         _lib = lib
@@ -439,3 +449,30 @@ def selective_effective_batch(batch: float, stages: int, alpha: float, theta_alp
 def delay_gain(iterations: float, pdr: float, running: float, i_delay: float, i_wait) -> float:
     w = (C.c_double * len(i_wait))(*[float(x) for x in i_wait])
     return float(load_library().spx_delay_gain(float(iterations), len(i_wait), float(pdr), float(running), float(i_delay), w))
+
+
+LM_TILE_COLS = 256
+
+
+def lm_head(hidden, weight, logits: Optional[torch.Tensor] = None, want_stats: bool = True,
+            tile_stats: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None):
+    """spx_lm_head on the current stream.  Returns (logits [rows, stride] bf16, tile_stats or None, status)."""
+    _require_cuda(hidden, weight)
+    lib = load_library()
+    dev = hidden.device
+    rows, K = hidden.shape
+    V = weight.shape[0]
+    if logits is None:
+        stride = V + (-V) % 8
+        logits = torch.empty((rows, stride), dtype=torch.bfloat16, device=dev)
+    if want_stats and tile_stats is None:
+        tile_stats = torch.empty((rows, (V + LM_TILE_COLS - 1) // LM_TILE_COLS, 2), dtype=torch.float32, device=dev)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    a = LmHeadArgs()
+    a.rows, a.hidden_dim, a.vocab = rows, K, V
+    a.hidden, a.weight, a.logits = _ptr(hidden), _ptr(weight), _ptr(logits)
+    a.logits_row_stride = logits.stride(0)
+    a.tile_stats = _ptr(tile_stats) if want_stats else None
+    _check(lib.spx_lm_head(C.byref(a), status.data_ptr(), _stream(dev)))
+    return logits, (tile_stats if want_stats else None), status

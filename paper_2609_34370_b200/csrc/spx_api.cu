@@ -14,6 +14,7 @@
 #include "kv_cache.cuh"
 #include "select.cuh"
 #include "lookahead.cuh"
+#include "lm_head.cuh"
 #include "plan.cuh"
 #include "sampler.cuh"
 #include "spx.h"
@@ -743,6 +744,48 @@ double spx_delay_gain(double iterations, int32_t n_evictions, double pdr, double
   const double recompute = (iterations + (double)(n_evictions + 1) * (pdr - 1.0)) / (iterations + pdr - 1.0);
   const double idle = (running + 1.0 - i_delay / iterations) / (running + 1.0 - waited / iterations);
   return recompute * idle;
+}
+
+// ---- LM head ------------------------------------------------------------------------------------
+static bool make_matrix_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) return false;
+  cuuint64_t dims[2] = {cols, rows}, strides[1] = {cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kLmBK, box_rows}, estr[2] = {1, 1};
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+spx_status_t spx_lm_head(const spx_lm_head_args_t *a, int32_t *dev_status, void *cuda_stream) {
+  t_launches = 0;
+  if (!a || !dev_status) return SPX_ERR_INVALID_ARG;
+  if (a->rows < 0 || a->hidden_dim <= 0 || a->vocab <= 0 || a->logits_row_stride < a->vocab) return SPX_ERR_INVALID_ARG;
+  if (a->hidden_dim % 8 != 0 || a->logits_row_stride % 8 != 0) return SPX_ERR_UNSUPPORTED;
+  if (a->rows == 0) return SPX_OK;
+  if (!a->hidden || !a->weight || !a->logits) return SPX_ERR_INVALID_ARG;
+  if (((uintptr_t)a->hidden | (uintptr_t)a->weight | (uintptr_t)a->logits) & 15) return SPX_ERR_INVALID_ARG;
+  DeviceInfo info;
+  if (!get_device_info(&info)) return SPX_ERR_CUDA;
+  CUtensorMap hmap, wmap;
+  if (!make_matrix_map(&hmap, a->hidden, a->rows, a->hidden_dim, kLmBM) ||
+      !make_matrix_map(&wmap, a->weight, a->vocab, a->hidden_dim, kLmBN))
+    return SPX_ERR_CUDA;
+  LmParams p{};
+  p.M = a->rows; p.K = a->hidden_dim; p.V = a->vocab;
+  p.m_tiles = (a->rows + kLmBM - 1) / kLmBM;
+  p.n_tiles = (a->vocab + kLmBN - 1) / kLmBN;
+  p.k_blocks = (a->hidden_dim + kLmBK - 1) / kLmBK;
+  p.logits = static_cast<__nv_bfloat16 *>(a->logits);
+  p.row_stride = a->logits_row_stride;
+  p.tile_stats = reinterpret_cast<float2 *>(a->tile_stats);
+  p.dev_status = dev_status;
+  if (cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLmSmemBytes) != cudaSuccess) return SPX_ERR_CUDA;
+  const long long tiles = (long long)p.m_tiles * p.n_tiles;
+  const int grid = tiles < info.num_sms ? (int)tiles : info.num_sms;
+  lm_head_kernel<<<grid, kLmThreads, kLmSmemBytes, static_cast<cudaStream_t>(cuda_stream)>>>(hmap, wmap, p);
+  ++t_launches;
+  return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
 }
 
 // ---- sampling without caller-provided scratch ------------------------------------------------
