@@ -182,6 +182,7 @@ def time_extras(spx, binding, spec, b, attn_args, dev, iters: int = 200):
     """Device time (CUDA events, mean of `iters` calls after 5 warm-up calls, L2 not flushed for the
     small ones: they are launch-bound) of the calls around the step and of the verification variants."""
     def timed(fn):
+        nonlocal iters
         for _ in range(5):
             fn()
         torch.cuda.synchronize()
@@ -254,6 +255,26 @@ def time_extras(spx, binding, spec, b, attn_args, dev, iters: int = 200):
     tau = torch.full((b.batch,), 32, dtype=torch.int32, device=dev)
     prec = torch.full((b.batch,), 0.83, dtype=torch.float64, device=dev)
     out["lookahead_memory_us"] = timed(lambda: spx.lookahead_memory(ell, tau, prec, 2, 0.7))
+    # LM head (hidden 4096, the workload's vocabulary, one row per target position), fused statistics on;
+    # torch's bf16 matmul (cuBLAS) beside it as the library reference
+    hid = 4096
+    gh = torch.Generator(device=dev).manual_seed(spec.seed + 9)
+    H = torch.randn((b.total_q, hid), generator=gh, device=dev).to(torch.bfloat16)
+    Wt = (torch.randn((spec.vocab, hid), generator=gh, device=dev) * (3.0 / hid ** 0.5)).to(torch.bfloat16)
+    lg = torch.empty((b.total_q, spec.vocab + (-spec.vocab) % 8), dtype=torch.bfloat16, device=dev)
+    ts = torch.empty((b.total_q, (spec.vocab + 255) // 256, 2), dtype=torch.float32, device=dev)
+    lm_iters = max(3, min(iters, 20))
+    saved, iters = iters, lm_iters
+    out["lm_head_us"] = timed(lambda: spx.lm_head(H, Wt, logits=lg, tile_stats=ts, status=status))
+    out["lm_head_nostats_us"] = timed(lambda: spx.lm_head(H, Wt, logits=lg, want_stats=False, status=status))
+    ref_out = torch.empty((b.total_q, spec.vocab), dtype=torch.bfloat16, device=dev)
+    out["cublas_matmul_us"] = timed(lambda: torch.matmul(H, Wt.t(), out=ref_out))
+    iters = saved
+    flops = 2.0 * b.total_q * hid * spec.vocab
+    out["lm_head_tflops"] = flops / (out["lm_head_us"] * 1e-6) / 1e12
+    out["cublas_matmul_tflops"] = flops / (out["cublas_matmul_us"] * 1e-6) / 1e12
+    out["lm_head_weight_gbs"] = Wt.numel() * 2 / (out["lm_head_us"] * 1e-6) / 1e9
+    del H, Wt, lg, ts, ref_out
     if int(ws.status.item()) != 0 or int(status.item()) != 0 or int(cws.status.item()) != 0:
         out["status"] = [int(ws.status.item()), int(status.item()), int(cws.status.item())]
     return out

@@ -193,7 +193,8 @@ def make_attn_args(q, k_cache, v_cache, kv_strides, block_table, seq_lens, q_ind
 
 
 def make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, accepted_len,
-                     out_tokens, diag_ratio=None, vocab=None, temperature=None, top_k=None, top_p=None) -> SampleArgs:
+                     out_tokens, diag_ratio=None, vocab=None, temperature=None, top_k=None, top_p=None,
+                     target_tile_stats=None) -> SampleArgs:
     s = SampleArgs()
     s.batch = q_indptr.numel() - 1
     s.total_q = target_logits.shape[0]
@@ -205,6 +206,7 @@ def make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept,
     s.u_accept, s.u_sample = _ptr(u_accept), _ptr(u_sample)
     s.accepted_len, s.out_tokens, s.diag_ratio = _ptr(accepted_len), _ptr(out_tokens), _ptr(diag_ratio)
     s.temperature, s.top_k, s.top_p = _ptr(temperature), _ptr(top_k), _ptr(top_p)
+    s.target_tile_stats = _ptr(target_tile_stats)
     return s
 
 
@@ -255,7 +257,8 @@ def verify_attention(q, k_cache, v_cache, kv_strides, block_table, seq_lens, q_i
 
 
 def rejection_sample(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, vocab=None,
-                     want_ratio=False, ws: Optional[Workspace] = None, temperature=None, top_k=None, top_p=None):
+                     want_ratio=False, ws: Optional[Workspace] = None, temperature=None, top_k=None, top_p=None,
+                     target_tile_stats=None):
     """spx_rejection_sample on the current stream.  Returns (accepted_len, out_tokens, ratio, ws).
     ``temperature`` ([B] float32 on the device, optional) selects the verification variant per request."""
     _require_cuda(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample)
@@ -270,7 +273,7 @@ def rejection_sample(target_logits, draft_logits, draft_ids, q_indptr, u_accept,
     tokens = torch.empty(TQ, dtype=torch.int32, device=dev)
     ratio = torch.empty(TQ - B, dtype=torch.float32, device=dev) if want_ratio else None
     s = make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, accepted, tokens,
-                         ratio, vocab, temperature, top_k, top_p)
+                         ratio, vocab, temperature, top_k, top_p, target_tile_stats)
     need = workspace_size(None, s)
     if ws is None:
         ws = Workspace.allocate(need, dev)

@@ -50,6 +50,7 @@ struct SampleParams {
   int32_t *row_req;          // [(TQ+TD)] request whose filter applies to the row, -1 = none
   uint32_t *row_thresh;      // [(TQ+TD)] order key of the lowest kept logit (0 = everything kept)
   double *row_z;             // [(TQ+TD)] kept mass sum 2^(x*scale - M); < 0 = unfiltered, use the statistics
+  int32_t first_row;         // statistics pass: rows below this one already have their statistics (LM-head epilogue)
   uint2 *req_thresh;         // [B]  thresholds of rows n (target, draft)
   float *seg_pmass;          // [B][nseg] kept target mass of each segment of row n
 };
@@ -280,7 +281,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleP
   const __nv_bfloat16 *target = reinterpret_cast<const __nv_bfloat16 *>(p.target);
   const __nv_bfloat16 *draft = reinterpret_cast<const __nv_bfloat16 *>(p.draft);
   auto chunk_src = [&](int g, int &row, int &e0) -> const __nv_bfloat16 * {
-    row = g / chunks_per_row;
+    row = p.first_row + g / chunks_per_row;
     e0 = (g % chunks_per_row) * kRingStageElems;
     const __nv_bfloat16 *base = row < p.total_q ? target + (int64_t)row * p.row_stride
                                                 : draft + (int64_t)(row - p.total_q) * p.row_stride;
@@ -291,10 +292,10 @@ __global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleP
     if (lane == 0) {
       int i = 0;
       // the scale of the next chunk's row is fetched one iteration ahead, off the issue path
-      float sc_next = (kScaled && (int)blockIdx.x < n_chunks) ? p.row_scale[blockIdx.x / chunks_per_row] : 1.f;
+      float sc_next = (kScaled && (int)blockIdx.x < n_chunks) ? p.row_scale[p.first_row + blockIdx.x / chunks_per_row] : 1.f;
       for (int g = blockIdx.x; g < n_chunks; g += gridDim.x, ++i) {
         const float sc = sc_next;
-        if (kScaled && g + (int)gridDim.x < n_chunks) sc_next = p.row_scale[(g + gridDim.x) / chunks_per_row];
+        if (kScaled && g + (int)gridDim.x < n_chunks) sc_next = p.row_scale[p.first_row + (g + gridDim.x) / chunks_per_row];
         const int s = i % kRingStages;
         if (i >= kRingStages && !ring_wait(&empty[s], ((i / kRingStages) - 1) & 1, abort, p.dev_status)) break;
         int row, e0;

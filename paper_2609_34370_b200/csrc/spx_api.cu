@@ -351,7 +351,8 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
 }
 
 template <typename T, bool kScaled, bool kFiltered = false>
-static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream, int num_sms, int phases) {
+static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream, int num_sms, int phases,
+                                     const float2 *tile_stats = nullptr) {
   const int rows = p.total_q + p.total_d;
   const int n_units = rows * p.nsub;
   int per_sm = 0;
@@ -373,9 +374,18 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
           cudaSuccess)
         return SPX_ERR_CUDA;
       const int chunks_per_row = (p.vocab + kRingStageElems - 1) / kRingStageElems;
-      const int n_chunks = rows * chunks_per_row;
-      row_stats_ring_kernel<kScaled><<<num_sms < n_chunks ? num_sms : n_chunks, kRingThreads, kRingSmemBytes, stream>>>(
-          p, chunks_per_row, n_chunks);
+      const int n_chunks = (rows - p.first_row) * chunks_per_row;
+      if (p.first_row > 0) {
+        // the target rows' statistics came out of the LM-head epilogue, per 256-column tile: fold them
+        // into sub-segments; only the draft rows are read here
+        const int n = p.first_row * p.nsub;
+        lm_stats_merge_kernel<<<(n + 255) / 256, 256, 0, stream>>>(tile_stats, p.first_row, (p.vocab + kLmBN - 1) / kLmBN, p.nsub,
+                                                                  kSubElems / kLmBN, p.seg_stats);
+        ++t_launches;
+      }
+      if (n_chunks > 0)
+        row_stats_ring_kernel<kScaled><<<num_sms < n_chunks ? num_sms : n_chunks, kRingThreads, kRingSmemBytes, stream>>>(
+            p, chunks_per_row, n_chunks);
     } else {
       row_stats_kernel<T, kScaled><<<grid, kSampThreads, 0, stream>>>(p, n_units);
     }
@@ -429,6 +439,10 @@ static spx_status_t launch_sampler(const spx_sample_args_t *s, unsigned char *ws
     p.row_scale = reinterpret_cast<float *>(ws + w.row_scale);
     return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16, true>(p, stream, num_sms, phases)
                                        : launch_sampler_t<float, true>(p, stream, num_sms, phases);
+  }
+  if (s->logits_dtype == SPX_BF16 && s->target_tile_stats) {
+    p.first_row = p.total_q;   // base rule on bf16 logits: the LM head's statistics stand in for the target rows
+    return launch_sampler_t<__nv_bfloat16, false>(p, stream, num_sms, phases, reinterpret_cast<const float2 *>(s->target_tile_stats));
   }
   return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16, false>(p, stream, num_sms, phases)
                                      : launch_sampler_t<float, false>(p, stream, num_sms, phases);
@@ -592,6 +606,7 @@ spx_status_t spx_verify_step_host(const spx_attn_args_t *attn, const spx_sample_
   s.q_indptr = a.q_indptr; s.u_accept = reinterpret_cast<float *>(d + L.ua); s.u_sample = reinterpret_cast<float *>(d + L.us);
   s.accepted_len = reinterpret_cast<int32_t *>(d + L.acc); s.out_tokens = reinterpret_cast<int32_t *>(d + L.tok);
   s.diag_ratio = nullptr;
+  s.target_tile_stats = nullptr;  // a host pointer here: the statistics pass reads the target rows itself
   s.temperature = sample->temperature ? reinterpret_cast<float *>(d + L.tau) : nullptr;
   s.top_k = sample->top_k ? reinterpret_cast<int32_t *>(d + L.topk) : nullptr;
   s.top_p = sample->top_p ? reinterpret_cast<float *>(d + L.topp) : nullptr;

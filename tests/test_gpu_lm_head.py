@@ -66,6 +66,46 @@ def test_integer_data_is_bit_exact_and_repeatable():
         assert torch.equal(again[:, :V], logits[:, :V])
 
 
+def test_fused_statistics_feed_the_sampling_half():
+    """Integer data: the GPU's logits equal the oracle's bit for bit, so the sampling half run on them with
+    the epilogue's statistics can be held against the oracle run on the oracle's own logits."""
+    from parity_util import check_sampling
+    rng = np.random.default_rng(11)
+    B, k, K, V = 24, 3, 64, 5000
+    TQ, TD = B * (k + 1), B * k
+    H = torch.from_numpy(rng.integers(-2, 3, size=(TQ, K)).astype(np.float32)).to(torch.bfloat16)
+    W = torch.from_numpy((rng.integers(-1, 2, size=(V, K)) * (rng.random((V, K)) < 0.3)).astype(np.float32)).to(torch.bfloat16)
+    ref_logits = oracle.lm_head(H, W)
+    assert float(ref_logits.abs().max()) < 256
+    T = ref_logits.to(torch.bfloat16)                               # exact
+    qi = torch.arange(0, (B + 1) * (k + 1), k + 1, dtype=torch.int32)
+    t_rows = torch.tensor([r * (k + 1) + i for r in range(B) for i in range(k)])
+    Dr = (T[t_rows].float() + torch.from_numpy(rng.integers(-1, 2, size=(TD, V)).astype(np.float32))).to(torch.bfloat16)
+    g = torch.Generator().manual_seed(3)
+    ids = torch.multinomial(torch.softmax(Dr.float(), dim=1), 1, generator=g).view(-1).to(torch.int32)
+    ua, us = torch.rand(TD, generator=g), torch.rand(B, generator=g)
+    logits, stats, status = spx.lm_head(H.to(DEV), W.to(DEV))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(logits[:, :V].cpu(), T)
+    acc, tok, _, ws = spx.rejection_sample(logits, Dr.to(DEV).contiguous(), ids.to(DEV), qi.to(DEV), ua.to(DEV), us.to(DEV),
+                                           vocab=V, target_tile_stats=stats)
+    acc0, tok0, _, _ = spx.rejection_sample(logits, Dr.to(DEV).contiguous(), ids.to(DEV), qi.to(DEV), ua.to(DEV), us.to(DEV), vocab=V)
+    torch.cuda.synchronize()
+    assert int(ws.status.item()) == 0
+
+    class _B:
+        pass
+    bb = _B()
+    bb.batch, bb.q_indptr, bb.u_accept, bb.u_sample = B, qi, ua, us
+    bb.target_logits, bb.draft_logits, bb.draft_ids = T, Dr, ids
+    bb.spec = type("S", (), {"vocab": V})
+    rep = check_sampling(bb, acc, tok)
+    assert not rep.hard_mismatch, rep
+    assert int(acc.sum()) > 0
+    print(f"\n[fused statistics] exact {rep.exact}/{rep.requests}, near ties {rep.accept_near_tie + rep.cdf_near_tie}; "
+          f"same as the unfused pass on {int((acc == acc0).sum())}/{B} requests")
+
+
 def test_llama_shape_on_sampled_column_blocks():
     g = torch.Generator().manual_seed(8)
     M, K, V = 384, 4096, 128256
