@@ -269,6 +269,15 @@ def time_extras(spx, binding, spec, b, attn_args, dev, iters: int = 200):
     out["lm_head_nostats_us"] = timed(lambda: spx.lm_head(H, Wt, logits=lg, want_stats=False, status=status))
     ref_out = torch.empty((b.total_q, spec.vocab), dtype=torch.bfloat16, device=dev)
     out["cublas_matmul_us"] = timed(lambda: torch.matmul(H, Wt.t(), out=ref_out))
+    # sampling half on the LM head's logits: own statistics pass over all rows vs the epilogue's statistics
+    if b.draft_logits.stride(0) == lg.stride(0):
+        s_plain = binding.make_sample_args(lg, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample, acc, tok,
+                                           None, spec.vocab)
+        s_fused = binding.make_sample_args(lg, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample, acc, tok,
+                                           None, spec.vocab, None, None, None, ts)
+        ws.ensure(spx.workspace_size(attn_args, s_plain))
+        out["sample_on_lm_logits_us"] = timed(sample_call(s_plain))
+        out["sample_with_lm_stats_us"] = timed(sample_call(s_fused))
     iters = saved
     flops = 2.0 * b.total_q * hid * spec.vocab
     out["lm_head_tflops"] = flops / (out["lm_head_us"] * 1e-6) / 1e12
