@@ -104,3 +104,44 @@ def test_binding_refuses_host_tensors():
     with pytest.raises(spx.SpxError):
         spx.rejection_sample(t, t[:0], torch.zeros(0, dtype=torch.int32), torch.tensor([0, 1, 2], dtype=torch.int32),
                              torch.zeros(0), torch.zeros(2))
+
+
+def test_calls_around_the_step_refuse_bad_arguments_before_any_launch(lib):
+    status = C.c_int32(0)
+    fake = C.c_void_p(0x1000)                                       # never dereferenced: every call below fails validation first
+    # KV append / rollback
+    ka = binding.KvAppendArgs()
+    assert lib.spx_kv_append(None, C.byref(status), None) == binding.ERR_INVALID_ARG
+    ka.batch, ka.total_q, ka.num_kv_heads, ka.head_dim, ka.page_size, ka.num_pages, ka.max_pages_per_req = 2, 6, 8, 128, 12, 10, 4
+    ka.kv_dtype, ka.kv_stride_page, ka.kv_stride_head, ka.kv_stride_token = 0, 8 * 12 * 128, 12 * 128, 128
+    assert lib.spx_kv_append(C.byref(ka), C.byref(status), None) == binding.ERR_UNSUPPORTED      # page size not a power of two
+    ka.page_size = 16
+    assert lib.spx_kv_append(C.byref(ka), C.byref(status), None) == binding.ERR_INVALID_ARG      # null pointers
+    assert lib.spx_kv_append(C.byref(ka), None, None) == binding.ERR_INVALID_ARG
+    assert lib.spx_kv_rollback(-1, fake, fake, fake, fake, C.byref(status), None) == binding.ERR_INVALID_ARG
+    assert lib.spx_kv_rollback(3, None, fake, fake, fake, C.byref(status), None) == binding.ERR_INVALID_ARG
+    assert lib.spx_kv_rollback(0, None, None, None, None, C.byref(status), None) == binding.OK   # empty batch: nothing to do
+    # selection
+    for alpha in (-0.1, 1.5, float("nan")):
+        assert lib.spx_select_speculation(4, fake, fake, alpha, fake, None, C.byref(status), None) == binding.ERR_INVALID_ARG
+    assert lib.spx_select_speculation(4, None, fake, 0.3, fake, None, C.byref(status), None) == binding.ERR_INVALID_ARG
+    # confidence
+    ca = binding.ConfArgs()
+    ca.batch, ca.total_q, ca.vocab, ca.logits_row_stride, ca.logits_dtype = 4, 12, 1000, 1001, 0
+    assert lib.spx_draft_confidence_workspace(C.byref(ca)) == 0                                  # stride not a multiple of 8
+    ca.logits_row_stride = 1000
+    assert lib.spx_draft_confidence_workspace(C.byref(ca)) > 0
+    assert lib.spx_draft_confidence(C.byref(ca), None, 0, C.byref(status), None) == binding.ERR_INVALID_ARG
+    # look-ahead memory
+    for pp, theta, horizon in ((0, 0.5, 64), (2, -0.1, 64), (2, 0.5, 0), (2, 0.5, 257)):
+        assert lib.spx_lookahead_memory(4, fake, fake, fake, pp, theta, horizon, fake, None) == binding.ERR_INVALID_ARG
+    assert lib.spx_lookahead_memory(4, None, fake, fake, 2, 0.5, 64, fake, None) == binding.ERR_INVALID_ARG
+    # LM head
+    la = binding.LmHeadArgs()
+    la.rows, la.hidden_dim, la.vocab, la.logits_row_stride = 4, 60, 100, 104
+    assert lib.spx_lm_head(C.byref(la), C.byref(status), None) == binding.ERR_UNSUPPORTED        # hidden size not a multiple of 8
+    la.hidden_dim = 64
+    assert lib.spx_lm_head(C.byref(la), C.byref(status), None) == binding.ERR_INVALID_ARG        # null pointers
+    la.logits_row_stride = 96
+    assert lib.spx_lm_head(C.byref(la), C.byref(status), None) == binding.ERR_INVALID_ARG        # stride below the vocabulary
+    assert status.value == 0
