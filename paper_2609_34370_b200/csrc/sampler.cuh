@@ -548,6 +548,9 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
 
   // One descent.  On entry s_cnt / s_mass hold level 0.  Returns the threshold key; *Z receives the
   // mass at or above it (meaningful only when masses were kept at level 0, i.e. use_p).
+  unsigned long long mass_above_bin = 0ull;  // top-k alone: this thread's share of the mass in the bins above the chosen one
+  bool list_ok = false;
+  uint32_t list_len = 0;
   auto descend = [&](bool by_count, uint32_t need, double need_mass, unsigned long long *Z) -> uint32_t {
     pick(by_count, need, need_mass, 0ull);
     const uint32_t b0 = s_bin;
@@ -557,14 +560,19 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
     // the elements of bin b0, into shared memory if they fit
     if (tid == 0) s_list_n = 0;
     __syncthreads();
+    const bool sum_above = by_count && !use_p;  // no masses were kept at level 0: add up what lies above the bin here
     sweep_row<T>(base, p.vocab, tid, [&](float x) {
-      if (bin0_of(x) != b0) return;
+      const uint32_t bx = bin0_of(x);
+      if (sum_above && bx > b0) mass_above_bin += mass_of(x);
+      if (bx != b0) return;
       const uint32_t i = atomicAdd(&s_list_n, 1u);
       if (i < (uint32_t)kFilterListCap) s_list[i] = x;
     });
     __syncthreads();
     const uint32_t n_list = s_list_n;
     const bool listed = n_list <= (uint32_t)kFilterListCap;
+    list_ok = listed;
+    list_len = n_list;
     uint32_t prefix = 0;
     for (int level = 1; level <= kLevels; ++level) {
       const int shift = kKeyShift + 8 * (kLevels - level);
@@ -606,9 +614,17 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
     Tf = descend(false, 0u, (double)tp * (double)Zk, &Zf);
     if (Tf < Tk) { Tf = Tk; Zf = Zk; }  // cannot happen with exact sums; keeps the sets nested regardless
   } else {
-    // top-k alone kept only counts at level 0: one more sweep adds up the kept mass in registers
+    // top-k alone kept only counts at level 0.  The kept mass is what lay above the chosen bin (added up
+    // during the collecting sweep) plus the listed elements at or above the threshold; a bin too
+    // crowded for the list costs one more sweep instead.
     unsigned long long acc = 0ull;
-    sweep_row<T>(base, p.vocab, tid, [&](float x) { if (order_key32(x) >= Tf) acc += mass_of(x); });
+    if (list_ok) {
+      acc = mass_above_bin;
+      for (uint32_t i = tid; i < list_len; i += kFilterThreads)
+        if (order_key32(s_list[i]) >= Tf) acc += mass_of(s_list[i]);
+    } else {
+      sweep_row<T>(base, p.vocab, tid, [&](float x) { if (order_key32(x) >= Tf) acc += mass_of(x); });
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     __syncthreads();
