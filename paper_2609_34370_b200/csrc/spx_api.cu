@@ -352,7 +352,10 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
 
 template <typename T, bool kScaled, bool kFiltered = false>
 static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream, int num_sms, int phases,
-                                     const float2 *tile_stats = nullptr) {
+                                     const float2 *tile_stats = nullptr, int spare_sms = 0) {
+  // SMs the bulk-copy statistics kernel leaves alone (its CTAs fill an SM's registers and shared
+  // memory: nothing else starts on an SM it occupies)
+  const int ring_sms = num_sms - spare_sms > 0 ? num_sms - spare_sms : num_sms;
   const int rows = p.total_q + p.total_d;
   const int n_units = rows * p.nsub;
   int per_sm = 0;
@@ -384,7 +387,7 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
         ++t_launches;
       }
       if (n_chunks > 0)
-        row_stats_ring_kernel<kScaled><<<num_sms < n_chunks ? num_sms : n_chunks, kRingThreads, kRingSmemBytes, stream>>>(
+        row_stats_ring_kernel<kScaled><<<ring_sms < n_chunks ? ring_sms : n_chunks, kRingThreads, kRingSmemBytes, stream>>>(
             p, chunks_per_row, n_chunks);
     } else {
       row_stats_kernel<T, kScaled><<<grid, kSampThreads, 0, stream>>>(p, n_units);
@@ -407,7 +410,7 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
 }
 
 static spx_status_t launch_sampler(const spx_sample_args_t *s, unsigned char *ws, int32_t *dev_status,
-                                   cudaStream_t stream, int num_sms, int phases = kPhaseAll) {
+                                   cudaStream_t stream, int num_sms, int phases = kPhaseAll, int spare_sms = 0) {
   if (s->batch == 0) return SPX_OK;
   if (s->batch > 65535) return SPX_ERR_UNSUPPORTED;  // grid.y limit of the residual pass
   const SampleWs w = sample_ws_layout(s);
@@ -431,21 +434,21 @@ static spx_status_t launch_sampler(const spx_sample_args_t *s, unsigned char *ws
     p.row_z = reinterpret_cast<double *>(ws + w.row_z);
     p.req_thresh = reinterpret_cast<uint2 *>(ws + w.req_thresh);
     p.seg_pmass = reinterpret_cast<float *>(ws + w.seg_pmass);
-    return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16, true, true>(p, stream, num_sms, phases)
-                                       : launch_sampler_t<float, true, true>(p, stream, num_sms, phases);
+    return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16, true, true>(p, stream, num_sms, phases, nullptr, spare_sms)
+                                       : launch_sampler_t<float, true, true>(p, stream, num_sms, phases, nullptr, spare_sms);
   }
   if (s->temperature) {
     p.temperature = s->temperature;
     p.row_scale = reinterpret_cast<float *>(ws + w.row_scale);
-    return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16, true>(p, stream, num_sms, phases)
-                                       : launch_sampler_t<float, true>(p, stream, num_sms, phases);
+    return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16, true>(p, stream, num_sms, phases, nullptr, spare_sms)
+                                       : launch_sampler_t<float, true>(p, stream, num_sms, phases, nullptr, spare_sms);
   }
   if (s->logits_dtype == SPX_BF16 && s->target_tile_stats) {
     p.first_row = p.total_q;   // base rule on bf16 logits: the LM head's statistics stand in for the target rows
-    return launch_sampler_t<__nv_bfloat16, false>(p, stream, num_sms, phases, reinterpret_cast<const float2 *>(s->target_tile_stats));
+    return launch_sampler_t<__nv_bfloat16, false>(p, stream, num_sms, phases, reinterpret_cast<const float2 *>(s->target_tile_stats), spare_sms);
   }
-  return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16, false>(p, stream, num_sms, phases)
-                                     : launch_sampler_t<float, false>(p, stream, num_sms, phases);
+  return s->logits_dtype == SPX_BF16 ? launch_sampler_t<__nv_bfloat16, false>(p, stream, num_sms, phases, nullptr, spare_sms)
+                                     : launch_sampler_t<float, false>(p, stream, num_sms, phases, nullptr, spare_sms);
 }
 
 static spx_status_t check_ws(const void *ws, size_t ws_bytes, size_t need, const int32_t *dev_status) {
@@ -527,7 +530,9 @@ spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_
   // launch order matters: the one-block planner goes first so that it is not queued behind the
   // persistent blocks of the logits pass, which occupy every SM for their whole run
   const spx_status_t s0 = launch_attention(attn, base, dev_status, stream, dev, kPhasePlan);
-  const spx_status_t s1 = launch_sampler(sample, base + attn_bytes, dev_status, side->stream, dev.num_sms);
+  // one SM is kept clear of the logits pass so that the planner, which the attention kernel waits
+  // for, runs at once instead of after the first logits CTA has left (3 us earlier start)
+  const spx_status_t s1 = launch_sampler(sample, base + attn_bytes, dev_status, side->stream, dev.num_sms, kPhaseAll, 1);
   ok = ok && cudaEventRecord(side->join, side->stream) == cudaSuccess;
   const spx_status_t s2 = launch_attention(attn, base, dev_status, stream, dev, kPhaseMain);
   ok = ok && cudaStreamWaitEvent(stream, side->join, 0) == cudaSuccess;
