@@ -241,6 +241,9 @@ constexpr int kRingConsumerWarps = kRingStageElems / kSubElems;  // 8 warps redu
 constexpr int kRingGroups = SPX_RING_GROUPS;                     // groups of 8 warps, each takes every kRingGroups-th stage
 constexpr int kRingThreads = (kRingGroups * kRingConsumerWarps + 1) * 32;
 constexpr int kRingSmemBytes = kRingStages * kRingStageElems * 2 + 1024 + 256;
+// A stage must always be consumed by the same group: a group then never waits for a phase of a
+// stage's barrier that is two phases ahead of the one in flight (a parity wait cannot tell those apart).
+static_assert(kRingStages % kRingGroups == 0, "stages per group must be whole");
 
 __device__ __forceinline__ bool ring_wait(uint64_t *bar, uint32_t parity, volatile int *abort, int32_t *dev_status) {
   const uint32_t addr = (uint32_t)__cvta_generic_to_shared(bar);
