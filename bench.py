@@ -278,6 +278,8 @@ def time_extras(spx, binding, spec, b, attn_args, dev, iters: int = 200):
         ws.ensure(spx.workspace_size(attn_args, s_plain))
         out["sample_on_lm_logits_us"] = timed(sample_call(s_plain))
         out["sample_with_lm_stats_us"] = timed(sample_call(s_fused))
+        out["step_on_lm_logits_us"] = timed(lambda: spx.verify_step(attn_args, s_plain, ws, dev))
+        out["step_with_lm_stats_us"] = timed(lambda: spx.verify_step(attn_args, s_fused, ws, dev))
     iters = saved
     flops = 2.0 * b.total_q * hid * spec.vocab
     out["lm_head_tflops"] = flops / (out["lm_head_us"] * 1e-6) / 1e12
