@@ -21,7 +21,8 @@ constexpr int kSegElems = 8192;       // tokens per segment (residual pass, fina
 constexpr int kSubElems = SPX_SUB_ELEMS;  // tokens per sub-segment (statistics pass)
 constexpr int kSubPerSeg = kSegElems / kSubElems;
 constexpr int kSampThreads = 256;
-constexpr int kElemsPerThread = kSegElems / kSampThreads;  // 32
+constexpr int kResidThreads = 256;   // residual kernel: at most 64 registers a thread for bf16 logits, four blocks an SM
+constexpr int kElemsPerThread = kSegElems / kResidThreads;  // 32
 
 struct SampleParams {
   int32_t batch, total_q, total_d, vocab, nseg, nsub;
@@ -77,25 +78,39 @@ template <> struct Vec<float> {
   }
 };
 
-// Load the kElemsPerThread consecutive tokens [v0, v0+32) of a row that this thread owns into
-// x[] (log2 domain: logit * scale, scale = log2(e) / temperature); tokens >= vocab become -inf.
+// The kElemsPerThread consecutive tokens [v0, v0+32) of a row that a thread owns, kept as raw
+// 16-byte vectors and converted token by token (for bf16 logits half the registers of the converted
+// values).  get(i, scale) is token v0+i in the log2 domain (logit * scale, scale = log2(e) /
+// temperature, or the stored logit with scale 1); tokens >= vocab read as -inf.
 template <typename T>
-__device__ __forceinline__ void load_thread_span(const T *row, int v0, int vocab, float (&x)[kElemsPerThread], float scale) {
-  constexpr int N = Vec<T>::N;
+struct RawSpan {
+  static constexpr int N = Vec<T>::N, NV = kElemsPerThread / N;
+  uint4 raw[NV];
+  __device__ __forceinline__ void issue(const T *row, int v0, int vocab) {
 #pragma unroll
-  for (int c = 0; c < kElemsPerThread / N; ++c) {
-    const int v = v0 + c * N;
-    if (v + N <= vocab) {
-      float f[N];
-      Vec<T>::load(row + v, f, scale);
+    for (int c = 0; c < NV; ++c) {
+      const int v = v0 + c * N;
+      if (v + N <= vocab) {
+        raw[c] = __ldg(reinterpret_cast<const uint4 *>(row + v));
+      } else {
+        union { uint4 u; T e[N]; } tmp;
 #pragma unroll
-      for (int i = 0; i < N; ++i) x[c * N + i] = f[i];
-    } else {
-#pragma unroll
-      for (int i = 0; i < N; ++i) x[c * N + i] = (v + i < vocab) ? ld_as_float(row, v + i) * scale : -INFINITY;
+        for (int i = 0; i < N; ++i) {
+          if (v + i < vocab) tmp.e[i] = row[v + i];
+          else st_from_float(tmp.e, i, -INFINITY);
+        }
+        raw[c] = tmp.u;
+      }
     }
   }
-}
+  __device__ __forceinline__ float get(int i, float scale) const {
+    const uint4 &u = raw[i / N];
+    const int j = sizeof(T) == 2 ? (i % N) >> 1 : i % N;
+    const uint32_t w = j == 0 ? u.x : j == 1 ? u.y : j == 2 ? u.z : u.w;
+    if (sizeof(T) == 2) return __uint_as_float((i & 1) ? (w & 0xffff0000u) : (w << 16)) * scale;
+    return __uint_as_float(w) * scale;
+  }
+};
 
 // Merge two (max, sum) pairs.
 __device__ __forceinline__ void merge_ms(float &m, float &s, float m2, float s2) {
@@ -873,7 +888,7 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_
 // Segment choice in float64 over the segment masses, token choice by an fp32 scan of the chosen
 // segment (thread t owns tokens [32t, 32t+32) of it).
 template <typename T, bool kScaled, bool kFiltered>
-__global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams p) {
+__global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_select_kernel(SampleParams p) {
   const int seg_mine = blockIdx.x, r = blockIdx.y;
   const float4 nm = p.req_norm[r];
   if (nm.w < 0.f) return;  // invalid request, or a greedy one (decided beside the accept test)
@@ -905,23 +920,25 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
   const T *trow = reinterpret_cast<const T *>(p.target) + (int64_t)(t0 + n) * p.row_stride;
   const T *drow = reinterpret_cast<const T *>(p.draft) + (int64_t)(t0 - r + n) * p.row_stride;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  __shared__ float s_w[kSampThreads / 32];
+  __shared__ float s_w[kResidThreads / 32];
   __shared__ int s_last;
-  __shared__ float s_wp[kSampThreads / 32];
+  __shared__ float s_wp[kResidThreads / 32];
   if (!bonus || masked) {
     const int v0 = seg_mine * kSegElems + threadIdx.x * kElemsPerThread;
-    float xt[kElemsPerThread], xd[kElemsPerThread];
-    load_thread_span(trow, v0, p.vocab, xt, load_scale);
-    if (!bonus) load_thread_span(drow, v0, p.vocab, xd, load_scale);
+    RawSpan<T> st, sd;
+    st.issue(trow, v0, p.vocab);
+    if (!bonus) sd.issue(drow, v0, p.vocab);
+    else sd = st;  // never read as a draft row: qd_of() is zero for a bonus request
     float acc = 0.f, accp = 0.f;
 #pragma unroll
     for (int i = 0; i < kElemsPerThread; ++i) {
+      const float xt = st.get(i, load_scale), xd = sd.get(i, load_scale);
       if (kFiltered) {
-        const float pt = pt_of(xt[i]);
-        acc += fmaxf(0.f, pt - (bonus ? 0.f : qd_of(xd[i])));
+        const float pt = pt_of(xt);
+        acc += fmaxf(0.f, pt - (bonus ? 0.f : qd_of(xd)));
         accp += pt;
       } else {
-        acc += fmaxf(0.f, ex(xt[i], nm.x) * nm.y - ex(xd[i], nm.z) * nm.w);
+        acc += fmaxf(0.f, ex(xt, nm.x) * nm.y - ex(xd, nm.z) * nm.w);
       }
     }
     acc = warp_sum(acc);
@@ -930,11 +947,11 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
     __syncthreads();
     if (threadIdx.x == 0) {
       float tot = 0.f;
-      for (int w = 0; w < kSampThreads / 32; ++w) tot += s_w[w];
+      for (int w = 0; w < kResidThreads / 32; ++w) tot += s_w[w];
       p.seg_resid[(int64_t)r * p.nseg + seg_mine] = tot;
       if (kFiltered) {
         float totp = 0.f;
-        for (int w = 0; w < kSampThreads / 32; ++w) totp += s_wp[w];
+        for (int w = 0; w < kResidThreads / 32; ++w) totp += s_wp[w];
         p.seg_pmass[(int64_t)r * p.nseg + seg_mine] = totp;
       }
       __threadfence();
@@ -954,31 +971,47 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
       acc += (double)(tstats[j].y * fast_exp2(tstats[j].x - nm.x));
     return acc * (double)nm.y;
   };
+  // The segment masses are fetched by one thread each before the scan (one memory round trip for
+  // the lot; a scan that loads as it goes pays one round trip per segment, 10 us on a 128k
+  // vocabulary).  Segments beyond the staging array, if any, are read in place.
+  constexpr int kStageSegs = 128;
+  __shared__ double s_mass[kStageSegs];
   __shared__ int s_seg;
   __shared__ float s_target;
   __shared__ int s_degenerate;
-  __shared__ float s_scan[kSampThreads / 32];
+  __shared__ float s_scan[kResidThreads / 32];
   __shared__ int s_tok;
+  const volatile float *resid = p.seg_resid + (int64_t)r * p.nseg;
+  auto stage = [&](bool from_target) {
+    for (int i = threadIdx.x; i < min(p.nseg, kStageSegs); i += kResidThreads)
+      s_mass[i] = from_target ? target_mass(i) : (double)resid[i];
+    __syncthreads();
+  };
+  auto mass_at = [&](int i, bool from_target) -> double {
+    return i < kStageSegs ? s_mass[i] : from_target ? target_mass(i) : (double)resid[i];
+  };
+  bool use_target = bonus && !masked;
+  stage(use_target);
+  if (threadIdx.x == 0) {
+    double R = 0.0;
+    for (int i = 0; i < p.nseg; ++i) R += mass_at(i, use_target);
+    s_degenerate = !use_target && !(R > 0.0);
+  }
+  __syncthreads();
+  if (s_degenerate) {  // the residual is identically zero: draw from the target row instead
+    use_target = true;
+    stage(true);
+  }
   if (threadIdx.x == 0) {
     // segment masses (float64), total R, target s*R, first segment whose inclusive sum exceeds it
-    const volatile float *resid = p.seg_resid + (int64_t)r * p.nseg;
     double R = 0.0;
-    int degenerate = 0;
-    if (!bonus || masked) {
-      for (int i = 0; i < p.nseg; ++i) R += (double)resid[i];
-      if (!(R > 0.0)) degenerate = 1;
-    }
-    const bool use_target = (bonus && !masked) || degenerate;
-    if (use_target) {
-      R = 0.0;
-      for (int i = 0; i < p.nseg; ++i) R += target_mass(i);
-    }
+    for (int i = 0; i < p.nseg; ++i) R += mass_at(i, use_target);
     const double target = (double)p.u_sample[r] * R;
     double cum = 0.0;
     int seg = -1, last_pos = -1;
     double before = 0.0, last_before = 0.0;
     for (int i = 0; i < p.nseg; ++i) {
-      const double mass = use_target ? target_mass(i) : (double)resid[i];
+      const double mass = mass_at(i, use_target);
       if (mass > 0.0) { last_pos = i; last_before = cum; }
       if (cum + mass > target) { seg = i; before = cum; break; }
       cum += mass;
@@ -986,9 +1019,8 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
     if (seg < 0) { seg = last_pos; before = last_before; }
     s_seg = seg;
     s_target = (float)(target - before);
-    s_degenerate = degenerate;
     s_tok = 0x7fffffff;
-    if (degenerate) atomicOr(p.dev_status, SPX_DEV_DEGENERATE);
+    if (s_degenerate) atomicOr(p.dev_status, SPX_DEV_DEGENERATE);
   }
   __syncthreads();
   const int seg = s_seg;
@@ -996,22 +1028,26 @@ __global__ void __launch_bounds__(kSampThreads) resid_select_kernel(SampleParams
     if (threadIdx.x == 0) p.out_tokens[t0 + n] = -1;
     return;
   }
-  const bool use_target = (bonus && !masked) || s_degenerate;
   const float target = s_target;
   const int v0 = seg * kSegElems + threadIdx.x * kElemsPerThread;
   float w[kElemsPerThread];
   {
-    float xt[kElemsPerThread];
-    load_thread_span(trow, v0, p.vocab, xt, load_scale);
+    RawSpan<T> st;
+    st.issue(trow, v0, p.vocab);
     if (use_target || (kFiltered && bonus)) {
 #pragma unroll
-      for (int i = 0; i < kElemsPerThread; ++i) w[i] = kFiltered ? pt_of(xt[i]) : ex(xt[i], nm.x) * nm.y;
+      for (int i = 0; i < kElemsPerThread; ++i) {
+        const float xt = st.get(i, load_scale);
+        w[i] = kFiltered ? pt_of(xt) : ex(xt, nm.x) * nm.y;
+      }
     } else {
-      float xd[kElemsPerThread];
-      load_thread_span(drow, v0, p.vocab, xd, load_scale);
+      RawSpan<T> sd;
+      sd.issue(drow, v0, p.vocab);
 #pragma unroll
-      for (int i = 0; i < kElemsPerThread; ++i)
-        w[i] = kFiltered ? fmaxf(0.f, pt_of(xt[i]) - qd_of(xd[i])) : fmaxf(0.f, ex(xt[i], nm.x) * nm.y - ex(xd[i], nm.z) * nm.w);
+      for (int i = 0; i < kElemsPerThread; ++i) {
+        const float xt = st.get(i, load_scale), xd = sd.get(i, load_scale);
+        w[i] = kFiltered ? fmaxf(0.f, pt_of(xt) - qd_of(xd)) : fmaxf(0.f, ex(xt, nm.x) * nm.y - ex(xd, nm.z) * nm.w);
+      }
     }
   }
   float tsum = 0.f;

@@ -407,7 +407,7 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
     }
     const int accept_blocks = (p.batch * 32 + 127) / 128;
     accept_kernel<T, kScaled, kFiltered><<<accept_blocks + (kScaled ? p.batch : 0), 128, 0, stream>>>(p, accept_blocks);
-    resid_select_kernel<T, kScaled, kFiltered><<<dim3(p.nseg, p.batch), kSampThreads, 0, stream>>>(p);
+    resid_select_kernel<T, kScaled, kFiltered><<<dim3(p.nseg, p.batch), kResidThreads, 0, stream>>>(p);
     t_launches += 2;
   }
   return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
@@ -521,11 +521,14 @@ spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   unsigned char *base = static_cast<unsigned char *>(ws);
   // The halves are independent given their inputs: the sampling half is forked onto the internal
-  // stream and joined back before the call hands the caller's stream back.  Its blocks share the
-  // SMs with the persistent attention CTAs (which leave registers and 8 KB of shared memory
-  // free for them), so the logits pass fills the bandwidth the attention kernel leaves unused and
-  // the short accept/resample kernels disappear behind it.  (Measured on the Llama-3-8B shape:
-  // 176 us per step this way, 183 us with the two bandwidth-bound kernels back to back.)
+  // stream and joined back before the call hands the caller's stream back.  On the Llama-3-8B
+  // shape the step then runs as: logits statistics (about 31 us, every SM but one), attention
+  // (about 111 us; its CTAs take the SMs as the statistics CTAs leave them, with the accept
+  // kernel's few warps beside them), and a tail of about 17 us in which the residual kernel and
+  // the combine kernel share the SMs the attention CTAs free.  The residual kernel cannot run beside
+  // the attention CTAs: their six warps leave about 3000 registers free on two of an SM's four
+  // sub-partitions, less than two of its warps need; a four-warp variant that did fit slowed the
+  // attention kernel by 27 us a step.
   SideStream *side = get_side_stream(dev.device);
   if (!side) return SPX_ERR_CUDA;
   bool ok = cudaEventRecord(side->fork, stream) == cudaSuccess;
