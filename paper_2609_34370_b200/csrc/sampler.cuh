@@ -6,9 +6,9 @@
 // the loads of its next sub-segment in flight while it reduces the current one, no block-level
 // synchronisation) reduces each sub-segment to (max, sum exp(x - max)).  accept_kernel (one warp per
 // request, one lane per row) merges the segment pairs per row, evaluates p(x)/q(x) for the
-// drafts in float64 and fixes n.  resid_select_kernel re-reads rows n of the rejecting requests,
-// reduces max(0, p - q) per segment, and the block that finishes a request last picks the
-// segment by a float64 scan of the segment masses and the token by an fp32 scan inside it.
+// drafts in float64 and fixes n.  resid_mass_kernel re-reads rows n of the rejecting requests and
+// reduces max(0, p - q) per segment; resid_pick_kernel (one block per request) picks the segment
+// by a float64 scan of the segment masses and the token by an fp32 scan inside it.
 #pragma once
 #include "common.cuh"
 
@@ -40,7 +40,6 @@ struct SampleParams {
   float2 *seg_stats;   // [(TQ+TD)][nsub]  per sub-segment (max in log2 domain, sum)
   float *seg_resid;    // [B][nseg]        residual mass of each segment of row n (units of 1)
   float4 *req_norm;    // [B]  (Mt, 1/St, Md, 1/Sd) of row n, log2 domain maxima; Md = NaN => bonus
-  int32_t *req_done;   // [B]  segments of row n finished (zeroed by accept_kernel)
   int32_t *dev_status;
   // verification variants (both NULL: temperature 1 everywhere)
   const float *temperature;  // [B]  > 0: sample at that temperature; 0: greedy (NULL with filters: 1)
@@ -760,7 +759,7 @@ __device__ __forceinline__ void greedy_request(const SampleParams &p, int r) {
 // One warp per request, lane = row (lanes 0..k: target rows, lanes k+1..2k: draft rows).  Each lane
 // merges its row's segment pairs (fp32 exponentials, float64 sum); the accept ratios of all
 // drafts are evaluated in parallel in float64 and the first failure fixes n.  Writes
-// accepted_len, the accepted ids and the -1 padding; slot n is left for resid_select_kernel.
+// accepted_len, the accepted ids and the -1 padding; slot n is left for resid_pick_kernel.
 template <typename T, bool kScaled, bool kFiltered>
 __global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_blocks) {
   if (kScaled && (int)blockIdx.x >= accept_blocks) {  // variants: one extra block per request for the greedy ones
@@ -776,7 +775,6 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_
   const T *target = reinterpret_cast<const T *>(p.target);
   const T *draft = reinterpret_cast<const T *>(p.draft);
   const float nanf_ = __int_as_float(0x7fc00000);
-  if (lane == 0) p.req_done[r] = 0;
   if (k < 0 || k > SPX_MAX_K || t0 < 0 || t0 + k + 1 > p.total_q) {
     if (lane == 0) {
       atomicOr(p.dev_status, SPX_DEV_BAD_LEN);
@@ -883,93 +881,122 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_
   }
 }
 
-// Residual mass per segment of row n, then the final draw by the block that finishes the request
-// last (bonus requests need no residual pass: their block 0 draws at once).  grid = (nseg, B).
-// Segment choice in float64 over the segment masses, token choice by an fp32 scan of the chosen
-// segment (thread t owns tokens [32t, 32t+32) of it).
+// What the two residual kernels need to know about request r: the normalisers of rows n, the
+// filter thresholds, the row pointers and the probability terms of one token.
 template <typename T, bool kScaled, bool kFiltered>
-__global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_select_kernel(SampleParams p) {
-  const int seg_mine = blockIdx.x, r = blockIdx.y;
-  const float4 nm = p.req_norm[r];
-  if (nm.w < 0.f) return;  // invalid request, or a greedy one (decided beside the accept test)
-  const bool bonus = (nm.z != nm.z);
-  // filtering: tokens below the row's threshold carry no mass.  A masked request always takes the
-  // full pass (the statistics of the unfiltered row are of no use to it), a bonus draw as a residual
-  // against a draft term of zero.
-  uint2 thr = make_uint2(0u, 0u);
-  if (kFiltered) thr = p.req_thresh[r];
-  const bool masked = kFiltered && (thr.x != 0u || thr.y != 0u);
-  if (bonus && !masked && seg_mine != 0) return;
-  const int t0 = p.q_indptr[r];
-  // the variants keep the stored logit and scale it inside one fused multiply-add with the
-  // maximum (a separately rounded product would cost |x * scale| * 2^-24 of relative accuracy,
-  // which matters at low temperature); the base rule scales at load time
-  const float scale = kScaled ? p.row_scale[t0] : kLog2e;
-  const float load_scale = kScaled ? 1.f : kLog2e;
-  auto ex = [&](float x, float M) -> float { return kScaled ? fast_exp2(fmaf(x, scale, -M)) : fast_exp2(x - M); };
+struct ResidCtx {
+  float4 nm;        // (Mt, 1/St, Md, 1/Sd) of rows n; Md = NaN: bonus draw
+  uint2 thr;        // order keys of the lowest kept logit of rows n (target, draft); 0 = unfiltered
+  bool bonus, masked;
+  int t0, n;
+  float scale;      // log2(e)/tau of the request (variants), log2(e) otherwise
+  const T *trow, *drow;
+  static constexpr float kLoadScale = kScaled ? 1.f : kLog2e;
+
+  // false: nothing to draw (an invalid request, or a greedy one decided beside the accept test)
+  __device__ __forceinline__ bool init(const SampleParams &p, int r) {
+    nm = p.req_norm[r];
+    if (nm.w < 0.f) return false;
+    bonus = (nm.z != nm.z);
+    // filtering: tokens below the row's threshold carry no mass.  A masked request always takes
+    // the full pass (the statistics of the unfiltered row are of no use to it), a bonus draw as a
+    // residual against a draft term of zero.
+    thr = make_uint2(0u, 0u);
+    if (kFiltered) thr = p.req_thresh[r];
+    masked = kFiltered && (thr.x != 0u || thr.y != 0u);
+    t0 = p.q_indptr[r];
+    n = p.accepted_len[r];
+    // the variants keep the stored logit and scale it inside one fused multiply-add with the
+    // maximum (a separately rounded product would cost |x * scale| * 2^-24 of relative accuracy,
+    // which matters at low temperature); the base rule scales at load time
+    scale = kScaled ? p.row_scale[t0] : kLog2e;
+    trow = reinterpret_cast<const T *>(p.target) + (int64_t)(t0 + n) * p.row_stride;
+    drow = reinterpret_cast<const T *>(p.draft) + (int64_t)(t0 - r + n) * p.row_stride;
+    return true;
+  }
+  __device__ __forceinline__ bool full_pass() const { return !bonus || masked; }
+  __device__ __forceinline__ float ex(float x, float M) const {
+    return kScaled ? fast_exp2(fmaf(x, scale, -M)) : fast_exp2(x - M);
+  }
   // probability terms of one token (xt, xd are stored logits whenever kFiltered)
-  auto pt_of = [&](float xt) -> float {
+  __device__ __forceinline__ float pt_of(float xt) const {
     const float v = ex(xt, nm.x) * nm.y;
     return (kFiltered && order_key32(xt) < thr.x) ? 0.f : v;
-  };
-  auto qd_of = [&](float xd) -> float {
+  }
+  __device__ __forceinline__ float qd_of(float xd) const {
     if (kFiltered && (bonus || order_key32(xd) < thr.y)) return 0.f;
     return ex(xd, nm.z) * nm.w;
-  };
-  const int n = p.accepted_len[r];
-  const T *trow = reinterpret_cast<const T *>(p.target) + (int64_t)(t0 + n) * p.row_stride;
-  const T *drow = reinterpret_cast<const T *>(p.draft) + (int64_t)(t0 - r + n) * p.row_stride;
+  }
+  // residual weight max(0, p - q) of one token
+  __device__ __forceinline__ float resid_of(float xt, float xd) const {
+    if (kFiltered) return fmaxf(0.f, pt_of(xt) - qd_of(xd));
+    return fmaxf(0.f, ex(xt, nm.x) * nm.y - ex(xd, nm.z) * nm.w);
+  }
+};
+
+// Residual mass max(0, p - q) of each segment of rows n (and the kept target mass under
+// filters).  grid = (nseg, B); bonus requests without a mask need no pass.  The masses are plain
+// stores: the draw runs as the next kernel of the stream, so no fence or counter sits between a
+// block's loads and its exit (with a last-block-done counter every block paid two more memory
+// round trips, and the step's tail is made of these).
+template <typename T, bool kScaled, bool kFiltered>
+__global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_mass_kernel(SampleParams p) {
+  const int seg_mine = blockIdx.x, r = blockIdx.y;
+  ResidCtx<T, kScaled, kFiltered> c;
+  if (!c.init(p, r) || !c.full_pass()) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   __shared__ float s_w[kResidThreads / 32];
-  __shared__ int s_last;
   __shared__ float s_wp[kResidThreads / 32];
-  if (!bonus || masked) {
-    const int v0 = seg_mine * kSegElems + threadIdx.x * kElemsPerThread;
-    RawSpan<T> st, sd;
-    st.issue(trow, v0, p.vocab);
-    if (!bonus) sd.issue(drow, v0, p.vocab);
-    else sd = st;  // never read as a draft row: qd_of() is zero for a bonus request
-    float acc = 0.f, accp = 0.f;
+  const int v0 = seg_mine * kSegElems + threadIdx.x * kElemsPerThread;
+  RawSpan<T> st, sd;
+  st.issue(c.trow, v0, p.vocab);
+  if (!c.bonus) sd.issue(c.drow, v0, p.vocab);
+  else sd = st;  // never read as a draft row: qd_of() is zero for a bonus request
+  float acc = 0.f, accp = 0.f;
 #pragma unroll
-    for (int i = 0; i < kElemsPerThread; ++i) {
-      const float xt = st.get(i, load_scale), xd = sd.get(i, load_scale);
-      if (kFiltered) {
-        const float pt = pt_of(xt);
-        acc += fmaxf(0.f, pt - (bonus ? 0.f : qd_of(xd)));
-        accp += pt;
-      } else {
-        acc += fmaxf(0.f, ex(xt, nm.x) * nm.y - ex(xd, nm.z) * nm.w);
-      }
-    }
-    acc = warp_sum(acc);
-    if (kFiltered) accp = warp_sum(accp);
-    if (lane == 0) { s_w[warp] = acc; if (kFiltered) s_wp[warp] = accp; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      float tot = 0.f;
-      for (int w = 0; w < kResidThreads / 32; ++w) tot += s_w[w];
-      p.seg_resid[(int64_t)r * p.nseg + seg_mine] = tot;
-      if (kFiltered) {
-        float totp = 0.f;
-        for (int w = 0; w < kResidThreads / 32; ++w) totp += s_wp[w];
-        p.seg_pmass[(int64_t)r * p.nseg + seg_mine] = totp;
-      }
-      __threadfence();
-      s_last = (atomicAdd(&p.req_done[r], 1) == p.nseg - 1);
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();  // the other blocks' segment masses are visible from here on
+  for (int i = 0; i < kElemsPerThread; ++i) {
+    const float xt = st.get(i, c.kLoadScale), xd = sd.get(i, c.kLoadScale);
+    acc += c.resid_of(xt, xd);
+    if (kFiltered) accp += c.pt_of(xt);
   }
+  acc = warp_sum(acc);
+  if (kFiltered) accp = warp_sum(accp);
+  if (lane == 0) { s_w[warp] = acc; if (kFiltered) s_wp[warp] = accp; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tot = 0.f;
+    for (int w = 0; w < kResidThreads / 32; ++w) tot += s_w[w];
+    p.seg_resid[(int64_t)r * p.nseg + seg_mine] = tot;
+    if (kFiltered) {
+      float totp = 0.f;
+      for (int w = 0; w < kResidThreads / 32; ++w) totp += s_wp[w];
+      p.seg_pmass[(int64_t)r * p.nseg + seg_mine] = totp;
+    }
+  }
+}
 
-  const float2 *tstats = p.seg_stats + (int64_t)(t0 + n) * p.nsub;
+// The final draw of request r = blockIdx.x: segment choice in float64 over the segment masses,
+// token choice by an fp32 scan of the chosen segment (thread t owns tokens [32t, 32t+32) of it).
+// Launched with programmatic stream serialization: what the accept kernel left is read before the
+// wait, the masses of resid_mass_kernel after it.
+template <typename T, bool kScaled, bool kFiltered>
+__global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_pick_kernel(SampleParams p) {
+  const int r = blockIdx.x;
+  ResidCtx<T, kScaled, kFiltered> c;
+  const bool live = c.init(p, r);
+  const float u = p.u_sample[r];
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // a no-op under a plain launch
+  if (!live) return;
+  const bool bonus = c.bonus, masked = c.masked;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float2 *tstats = p.seg_stats + (int64_t)(c.t0 + c.n) * p.nsub;
   // probability mass of segment i of the target row, from its sub-segment statistics
   auto target_mass = [&](int i) -> double {
-    if (masked) return (double)reinterpret_cast<const volatile float *>(p.seg_pmass)[(int64_t)r * p.nseg + i];
+    if (masked) return (double)p.seg_pmass[(int64_t)r * p.nseg + i];
     double acc = 0.0;
     for (int j = i * kSubPerSeg; j < min((i + 1) * kSubPerSeg, p.nsub); ++j)
-      acc += (double)(tstats[j].y * fast_exp2(tstats[j].x - nm.x));
-    return acc * (double)nm.y;
+      acc += (double)(tstats[j].y * fast_exp2(tstats[j].x - c.nm.x));
+    return acc * (double)c.nm.y;
   };
   // The segment masses are fetched by one thread each before the scan (one memory round trip for
   // the lot; a scan that loads as it goes pays one round trip per segment, 10 us on a 128k
@@ -981,7 +1008,7 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_s
   __shared__ int s_degenerate;
   __shared__ float s_scan[kResidThreads / 32];
   __shared__ int s_tok;
-  const volatile float *resid = p.seg_resid + (int64_t)r * p.nseg;
+  const float *resid = p.seg_resid + (int64_t)r * p.nseg;
   auto stage = [&](bool from_target) {
     for (int i = threadIdx.x; i < min(p.nseg, kStageSegs); i += kResidThreads)
       s_mass[i] = from_target ? target_mass(i) : (double)resid[i];
@@ -1006,7 +1033,7 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_s
     // segment masses (float64), total R, target s*R, first segment whose inclusive sum exceeds it
     double R = 0.0;
     for (int i = 0; i < p.nseg; ++i) R += mass_at(i, use_target);
-    const double target = (double)p.u_sample[r] * R;
+    const double target = (double)u * R;
     double cum = 0.0;
     int seg = -1, last_pos = -1;
     double before = 0.0, last_before = 0.0;
@@ -1025,7 +1052,7 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_s
   __syncthreads();
   const int seg = s_seg;
   if (seg < 0) {  // no mass anywhere (cannot happen for finite logits)
-    if (threadIdx.x == 0) p.out_tokens[t0 + n] = -1;
+    if (threadIdx.x == 0) p.out_tokens[c.t0 + c.n] = -1;
     return;
   }
   const float target = s_target;
@@ -1033,21 +1060,18 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_s
   float w[kElemsPerThread];
   {
     RawSpan<T> st;
-    st.issue(trow, v0, p.vocab);
+    st.issue(c.trow, v0, p.vocab);
     if (use_target || (kFiltered && bonus)) {
 #pragma unroll
       for (int i = 0; i < kElemsPerThread; ++i) {
-        const float xt = st.get(i, load_scale);
-        w[i] = kFiltered ? pt_of(xt) : ex(xt, nm.x) * nm.y;
+        const float xt = st.get(i, c.kLoadScale);
+        w[i] = kFiltered ? c.pt_of(xt) : c.ex(xt, c.nm.x) * c.nm.y;
       }
     } else {
       RawSpan<T> sd;
-      sd.issue(drow, v0, p.vocab);
+      sd.issue(c.drow, v0, p.vocab);
 #pragma unroll
-      for (int i = 0; i < kElemsPerThread; ++i) {
-        const float xt = st.get(i, load_scale), xd = sd.get(i, load_scale);
-        w[i] = kFiltered ? fmaxf(0.f, pt_of(xt) - qd_of(xd)) : fmaxf(0.f, ex(xt, nm.x) * nm.y - ex(xd, nm.z) * nm.w);
-      }
+      for (int i = 0; i < kElemsPerThread; ++i) w[i] = c.resid_of(st.get(i, c.kLoadScale), sd.get(i, c.kLoadScale));
     }
   }
   float tsum = 0.f;
@@ -1092,7 +1116,7 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_s
     if (last >= 0) atomicMax(&s_tok, last);
     __syncthreads();
   }
-  if (threadIdx.x == 0) p.out_tokens[t0 + n] = s_tok;
+  if (threadIdx.x == 0) p.out_tokens[c.t0 + c.n] = s_tok;
 }
 
 }  // namespace spx
