@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(kSimtThreads) attn_simt_kernel(AttnParams p) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = p.G;
   if (p.hdr->overflow) return;
-  const int n_items = p.hdr->n_work * p.Hkv;
+  const int n_items = p.hdr->n_work;
 
   for (;;) {
     __syncthreads();
@@ -61,8 +61,8 @@ __global__ void __launch_bounds__(kSimtThreads) attn_simt_kernel(AttnParams p) {
     __syncthreads();
     const int item = s_item;
     if (item >= n_items) break;
-    const WorkEntry we = p.work[item / p.Hkv];
-    const int g = item % p.Hkv;
+    const WorkEntry we = p.work[item];
+    const int g = we.g;
     const int r = we.req;
     const int q0 = p.q_indptr[r];
     const int m = p.q_indptr[r + 1] - q0;
@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(kSimtThreads) attn_simt_kernel(AttnParams p) {
         for (int row = tid; row < R; row += kSimtThreads)
           p.lse[(int64_t)(q0 + row / G) * p.Hq + g * G + row % G] = (sM[row] + log2f(sL[row])) * kLn2;
     } else {
-      const int64_t slot = ((int64_t)we.part_slot * p.Hkv + g) * p.rows_cap;
+      const int64_t slot = (int64_t)we.part_slot * p.rows_cap;
       for (int i = tid; i < R * D; i += kSimtThreads) p.part_o[slot * D + i] = sO[i];
       for (int row = tid; row < R; row += kSimtThreads) p.part_ml[slot + row] = make_float2(sM[row], sL[row]);
     }

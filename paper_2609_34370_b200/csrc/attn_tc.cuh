@@ -186,18 +186,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
   // the plan is read from here on: under programmatic dependent launch, wait for the planner
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
-  const int n_items = p.hdr->overflow ? 0 : p.hdr->n_work * p.Hkv;
-  const int n_cta = gridDim.x;
-  // Item sequence of this CTA: row `it` of the size-sorted list, walked boustrophedon so that the
-  // big and small ends of each row alternate between CTAs.
-  auto item_index = [&](int it) -> int {
-    const int col = (it & 1) ? (n_cta - 1 - (int)blockIdx.x) : (int)blockIdx.x;
-    const long long idx = (long long)it * n_cta + col;
-    return idx < n_items ? (int)idx : -1;
-  };
+  // this CTA's range of the plan: entries cta_off[c] .. cta_off[c+1] of the work list, in order
+  const bool planned = !p.hdr->overflow && (int)blockIdx.x < p.hdr->n_cta;
+  const int item_begin = planned ? p.cta_off[blockIdx.x] : 0;
+  const int item_end = planned ? p.cta_off[blockIdx.x + 1] : 0;
+  auto item_index = [&](int it) -> int { return item_begin + it < item_end ? item_begin + it : -1; };
   auto load_item = [&](int idx, ItemInfo &I) {
-    const WorkEntry we = p.work[idx / p.Hkv];
-    I.req = we.req; I.g = idx % p.Hkv; I.tile_begin = we.tile_begin; I.tile_end = we.tile_end; I.part_slot = we.part_slot;
+    const WorkEntry we = p.work[idx];
+    I.req = we.req; I.g = we.g; I.tile_begin = we.tile_begin; I.tile_end = we.tile_end; I.part_slot = we.part_slot;
     I.q0 = p.q_indptr[we.req];
     I.m = p.q_indptr[we.req + 1] - I.q0;
     I.L = p.seq_lens[we.req];
@@ -283,7 +279,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
       for (int it = 0; ok; ++it, ++qc) {
         const int idx = item_index(it);
         if (idx < 0 || bars->abort) break;
-        const WorkEntry we = p.work[idx / p.Hkv];
+        const WorkEntry we = p.work[idx];
         const int n_tiles = we.tile_end - we.tile_begin;
         const uint32_t qb = qc & 1;
         ok = mbar_wait(&bars->q_full[qb], (qc >> 1) & 1, bars, p.dev_status);
@@ -484,7 +480,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
           }
           if (valid_row && p.lse) p.lse[(int64_t)(I.q0 + j) * p.Hq + I.g * p.G + hg] = (m_ref + log2f(l_sum)) * kLn2;
         } else {
-          const int64_t slot = ((int64_t)I.part_slot * p.Hkv + I.g) * p.rows_cap + row;
+          const int64_t slot = (int64_t)I.part_slot * p.rows_cap + row;
           float *dst = p.part_o + slot * D;
 #pragma unroll 1
           for (int c = 0; c < D / 32; ++c) {

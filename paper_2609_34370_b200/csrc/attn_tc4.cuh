@@ -135,18 +135,16 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   // programmatic dependent launch this is where the kernel waits for the planner to finish.
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
-  const int n_items = p.hdr->overflow ? 0 : p.hdr->n_work * p.Hkv;
-  const int n_cta = gridDim.x;
-  auto item_index = [&](int it) -> int {
-    const int col = (it & 1) ? (n_cta - 1 - (int)blockIdx.x) : (int)blockIdx.x;
-    const long long idx = (long long)it * n_cta + col;
-    return idx < n_items ? (int)idx : -1;
-  };
+  // this CTA's range of the plan: entries cta_off[c] .. cta_off[c+1] of the work list, in order
+  const bool planned = !p.hdr->overflow && (int)blockIdx.x < p.hdr->n_cta;
+  const int item_begin = planned ? p.cta_off[blockIdx.x] : 0;
+  const int item_end = planned ? p.cta_off[blockIdx.x + 1] : 0;
+  auto item_index = [&](int it) -> int { return item_begin + it < item_end ? item_begin + it : -1; };
   // Work entries carry everything a role needs about the request (one 32-byte load).
-  auto entry_of = [&](int idx) -> WorkEntry { return p.work[idx / p.Hkv]; };
+  auto entry_of = [&](int idx) -> WorkEntry { return p.work[idx]; };
   auto make_item = [&](const WorkEntry &we, int idx) -> ItemInfo {
     ItemInfo I;
-    I.req = we.req; I.g = idx % p.Hkv; I.tile_begin = we.tile_begin; I.tile_end = we.tile_end; I.part_slot = we.part_slot;
+    I.req = we.req; I.g = we.g; I.tile_begin = we.tile_begin; I.tile_end = we.tile_end; I.part_slot = we.part_slot;
     I.q0 = we.q0; I.m = we.m; I.L = we.L;
     I.R = I.m * p.G;
     I.t_end = min(we.tile_end * kTileTokens, I.L);
@@ -219,7 +217,7 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
       const int page = page_la;
       advance(la);
       page_la = load_page(la);
-      const int g = cur.idx % p.Hkv;
+      const int g = cur.e.g;
       const int t_end = min(cur.e.tile_end * kTileTokens, cur.e.L);
       for (int ti = 0; ti < tiles_per_group && cur.tile0 + ti < cur.e.tile_end; ++ti, ++tc_) {
         const int tile = cur.tile0 + ti;
@@ -260,7 +258,7 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
       auto tiles_of = [&](int it) -> int {
         const int idx = item_index(it);
         if (idx < 0) return 0;
-        const WorkEntry *we = p.work + idx / p.Hkv;
+        const WorkEntry *we = p.work + idx;
         return we->tile_end - we->tile_begin;
       };
       // the tile count of the following item is loaded when an item opens, long before it is needed
@@ -413,7 +411,7 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
           }
           if (tblk == 0 && p.lse) p.lse[(int64_t)(J.q0 + j) * p.Hq + J.g * p.G + hg] = (pend.m_ref + log2f(l_row)) * kLn2;
         } else {
-          const int64_t slot = ((int64_t)J.part_slot * p.Hkv + J.g) * p.rows_cap + row;
+          const int64_t slot = (int64_t)J.part_slot * p.rows_cap + row;
           float *dst = p.part_o + slot * D + tblk * CB;
 #pragma unroll
           for (int v = 0; v < CB / 4; ++v)

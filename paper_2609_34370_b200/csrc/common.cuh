@@ -43,17 +43,21 @@ __device__ __forceinline__ float warp_sum(float v) {
 // Work plan shared by the attention kernels.  Built on the device by plan_kernel so that no
 // host copy of seq_lens is needed.
 //
-// Each request's KV range is cut into tiles of kTileTokens tokens and the tiles into
-// n_chunks[r] balanced chunks of at most chunk_tiles tiles; one work entry is one
-// (request, chunk) and is executed once per kv-head.  Entries are ordered by decreasing size
-// so that the dynamic scheduler (an atomic counter) approximates longest-processing-time-first.
+// A pair is one (request, kv head); its KV range is tiles_r tiles of kTileTokens tokens.  The
+// pairs of the valid requests, in (request, head) order, form one tile axis of length T, which is
+// cut into n_cta contiguous ranges of equal length; CTA c of a persistent kernel executes range c
+// (entries cta_off[c] .. cta_off[c+1] of the work list, in axis order).  A cut within kSnapTiles
+// of a pair boundary moves onto it, so most pairs stay whole; a pair that k cuts cross has k+1
+// chunks, whose partial results the combine kernel merges.  Every CTA gets the same number of
+// tiles to within one, and at most n_cta - 1 pairs are split, whatever the length mix.
 // ------------------------------------------------------------------------------------------
+constexpr int kSnapTiles = 2;   // a cut this close to a pair boundary is moved onto the boundary
 struct PlanHeader {
-  int32_t n_work;        // number of (request, chunk) entries
-  int32_t chunk_tiles;   // largest chunk, in tiles
-  int32_t n_part_slots;  // partial-result slots in use (chunks of split requests)
+  int32_t n_work;        // number of work entries
+  int32_t n_cta;         // ranges the tile axis was cut into
+  int32_t n_part_slots;  // partial-result slots in use (chunks of split pairs)
   int32_t total_tiles;   // sum over requests of tiles (one kv-head)
-  int32_t work_counter;  // dynamic scheduler cursor, zeroed by the planner
+  int32_t work_counter;  // dynamic scheduler cursor (SIMT kernel), zeroed by the planner
   int32_t overflow;      // 1 if the plan did not fit the workspace (nothing is executed then)
   int32_t pad[2];
 };
@@ -62,11 +66,11 @@ struct __align__(16) WorkEntry {
   int32_t req;         // request index
   int32_t tile_begin;  // first tile of the chunk
   int32_t tile_end;    // one past the last tile
-  int32_t part_slot;   // partial slot, or -1 when the request is not split (direct output)
+  int32_t part_slot;   // partial slot, or -1 when the pair is not split (direct output)
   int32_t q0;          // q_indptr[req]: first query row of the request
   int32_t m;           // k+1 query positions
   int32_t L;           // seq_lens[req]
-  int32_t pad;
+  int32_t g;           // kv head
 };
 
 struct AttnParams {
@@ -83,15 +87,18 @@ struct AttnParams {
   float *lse;
   // plan + partials (workspace)
   PlanHeader *hdr;
-  int32_t *req_nchunks;    // [B]  0 = invalid request
-  int32_t *req_part_base;  // [B]
+  int32_t *pair_nchunks;   // [B*Hkv]  chunks of the pair, 0 = invalid request
+  int32_t *pair_part_base; // [B*Hkv]  first partial slot of a split pair
+  int32_t *tile_prefix;    // [B+1]  tiles of the requests before r (one kv head)
+  int32_t *valid_prefix;   // [B+1]  valid requests before r
+  int32_t *cta_off;        // [n_cta+1]  work entries of the CTAs before c
   int32_t *req_bad;        // [B]  set when a needed page id was out of range
   int32_t head_inner;      // tensor-map dimension order: 1 = (d, head, token, page), 0 = (d, token, head, page)
   WorkEntry *work;         // [max_work]
-  WorkEntry *work_tmp;     // [max_work]
   int32_t max_work;
-  float *part_o;           // [slot][Hkv][rows_cap][D]
-  float2 *part_ml;         // [slot][Hkv][rows_cap]  (m in log2 domain, l)
+  int32_t max_part_slots;
+  float *part_o;           // [slot][rows_cap][D]
+  float2 *part_ml;         // [slot][rows_cap]  (m in log2 domain, l)
   int32_t rows_cap;        // G * max_q_len
   int32_t *dev_status;
   long long *prof;         // optional per-CTA cycle counters (profiling builds only), else NULL

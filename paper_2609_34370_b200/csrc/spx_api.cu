@@ -75,8 +75,8 @@ constexpr int kPlanSmCount = 148;  // workspace sizing must not depend on a devi
 // workspace layout
 // ---------------------------------------------------------------------------------------------
 struct AttnWs {
-  size_t hdr, nchunks, part_base, req_bad, work, work_tmp, part_ml, part_o, total;
-  int32_t max_work, rows_cap;
+  size_t hdr, nchunks, part_base, tile_prefix, valid_prefix, cta_off, req_bad, work, part_ml, part_o, total;
+  int32_t max_work, max_part_slots, rows_cap;
 };
 
 static spx_status_t check_attn(const spx_attn_args_t *a, bool need_ptrs) {
@@ -108,18 +108,23 @@ static AttnWs attn_ws_layout(const spx_attn_args_t *a) {
   const int max_q = a->max_q_len == 0 ? SPX_MAX_K + 1 : a->max_q_len;
   const int G = a->num_q_heads / a->num_kv_heads;
   w.rows_cap = G * max_q;
-  // sum_r ceil(tiles_r / c) <= sum_r tiles_r / c + B with c >= total*Hkv / (sms*waves)
-  w.max_work = a->batch + kPlanSmCount * kPlanWaves + 1;
+  // one entry per (request, kv head) pair plus one per cut of the tile axis; a cut adds at most
+  // one chunk to a pair, so the split pairs have at most two chunks per cut between them
+  const size_t pairs = (size_t)a->batch * a->num_kv_heads;
+  w.max_work = (int)(pairs + kPlanSmCount + 1);
+  w.max_part_slots = 2 * kPlanSmCount;
   size_t off = 0;
   w.hdr = off; off = align_up(off + sizeof(PlanHeader), 256);
-  w.nchunks = off; off = align_up(off + sizeof(int32_t) * (size_t)a->batch, 256);
-  w.part_base = off; off = align_up(off + sizeof(int32_t) * (size_t)a->batch, 256);
+  w.nchunks = off; off = align_up(off + sizeof(int32_t) * pairs, 256);
+  w.part_base = off; off = align_up(off + sizeof(int32_t) * pairs, 256);
+  w.tile_prefix = off; off = align_up(off + sizeof(int32_t) * ((size_t)a->batch + 1), 256);
+  w.valid_prefix = off; off = align_up(off + sizeof(int32_t) * ((size_t)a->batch + 1), 256);
+  w.cta_off = off; off = align_up(off + sizeof(int32_t) * (kPlanSmCount + 1), 256);
   w.req_bad = off; off = align_up(off + sizeof(int32_t) * (size_t)a->batch, 256);
   w.work = off; off = align_up(off + sizeof(WorkEntry) * (size_t)w.max_work, 256);
-  w.work_tmp = off; off = align_up(off + sizeof(WorkEntry) * (size_t)w.max_work, 256);
-  const size_t slots = (size_t)w.max_work;
-  w.part_ml = off; off = align_up(off + sizeof(float2) * slots * a->num_kv_heads * w.rows_cap, 256);
-  w.part_o = off; off = align_up(off + sizeof(float) * slots * a->num_kv_heads * w.rows_cap * a->head_dim, 256);
+  const size_t slots = (size_t)w.max_part_slots;
+  w.part_ml = off; off = align_up(off + sizeof(float2) * slots * w.rows_cap, 256);
+  w.part_o = off; off = align_up(off + sizeof(float) * slots * w.rows_cap * a->head_dim, 256);
   w.total = off;
   return w;
 }
@@ -287,22 +292,25 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
   p.block_table = a->block_table; p.seq_lens = a->seq_lens; p.q_indptr = a->q_indptr;
   p.out = a->out; p.lse = a->lse;
   p.hdr = reinterpret_cast<PlanHeader *>(ws + w.hdr);
-  p.req_nchunks = reinterpret_cast<int32_t *>(ws + w.nchunks);
-  p.req_part_base = reinterpret_cast<int32_t *>(ws + w.part_base);
+  p.pair_nchunks = reinterpret_cast<int32_t *>(ws + w.nchunks);
+  p.pair_part_base = reinterpret_cast<int32_t *>(ws + w.part_base);
+  p.tile_prefix = reinterpret_cast<int32_t *>(ws + w.tile_prefix);
+  p.valid_prefix = reinterpret_cast<int32_t *>(ws + w.valid_prefix);
+  p.cta_off = reinterpret_cast<int32_t *>(ws + w.cta_off);
   p.req_bad = reinterpret_cast<int32_t *>(ws + w.req_bad);
   p.work = reinterpret_cast<WorkEntry *>(ws + w.work);
-  p.work_tmp = reinterpret_cast<WorkEntry *>(ws + w.work_tmp);
   p.max_work = w.max_work;
+  p.max_part_slots = w.max_part_slots;
   p.part_ml = reinterpret_cast<float2 *>(ws + w.part_ml);
   p.part_o = reinterpret_cast<float *>(ws + w.part_o);
   p.rows_cap = w.rows_cap;
   p.dev_status = dev_status;
   p.prof = t_prof;
 
-  // the plan never targets more chunks than the workspace was sized for
+  // one range of the plan per CTA of the persistent kernels, never more than the workspace was sized for
   const int sms = dev.num_sms < kPlanSmCount ? dev.num_sms : kPlanSmCount;
   if (phases & kPhasePlan) {
-    plan_kernel<<<1, 1024, 0, stream>>>(p, sms * kPlanWaves);
+    plan_kernel<<<1, 1024, 0, stream>>>(p, sms);
     ++t_launches;
     if (cudaGetLastError() != cudaSuccess) return SPX_ERR_CUDA;
   }
@@ -315,15 +323,15 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
     if (!make_pool_map(&kmap, a->k_cache, a, p.head_inner) || !make_pool_map(&vmap, a->v_cache, a, p.head_inner))
       return SPX_ERR_CUDA;
     if (p.rows_cap <= 32)
-      e = p.D == 128 ? launch_tc4<128, 32>(kmap, vmap, p, dev.num_sms, stream) : launch_tc4<64, 32>(kmap, vmap, p, dev.num_sms, stream);
+      e = p.D == 128 ? launch_tc4<128, 32>(kmap, vmap, p, sms, stream) : launch_tc4<64, 32>(kmap, vmap, p, sms, stream);
     else if (p.rows_cap <= 64)
-      e = p.D == 128 ? launch_tc4<128, 64>(kmap, vmap, p, dev.num_sms, stream) : launch_tc4<64, 64>(kmap, vmap, p, dev.num_sms, stream);
+      e = p.D == 128 ? launch_tc4<128, 64>(kmap, vmap, p, sms, stream) : launch_tc4<64, 64>(kmap, vmap, p, sms, stream);
     else if (p.D == 128)
-      e = p.rows_cap <= 64 ? launch_tc<128, 64>(kmap, vmap, p, dev.num_sms, stream)
-                           : launch_tc<128, 128>(kmap, vmap, p, dev.num_sms, stream);
+      e = p.rows_cap <= 64 ? launch_tc<128, 64>(kmap, vmap, p, sms, stream)
+                           : launch_tc<128, 128>(kmap, vmap, p, sms, stream);
     else
-      e = p.rows_cap <= 64 ? launch_tc<64, 64>(kmap, vmap, p, dev.num_sms, stream)
-                           : launch_tc<64, 128>(kmap, vmap, p, dev.num_sms, stream);
+      e = p.rows_cap <= 64 ? launch_tc<64, 64>(kmap, vmap, p, sms, stream)
+                           : launch_tc<64, 128>(kmap, vmap, p, sms, stream);
   } else {
     const SimtSmem lay(p.rows_cap, p.D);
     if (lay.total > dev.max_smem_optin) return SPX_ERR_UNSUPPORTED;

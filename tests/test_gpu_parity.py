@@ -4,6 +4,8 @@ Small cases are compared element by element on every request; full-size workload
 sampler on every request and attention on a sample of requests the oracle can afford, plus
 properties that hold at any size.  Tolerances are in tests/parity_util.py.
 """
+import dataclasses
+
 import pytest
 import torch
 
@@ -52,6 +54,26 @@ def test_small_workloads_match_oracle(idx, layout):
     assert torch.equal(torch.isnan(got), ~consulted) or rep.accept_near_tie > 0
     both = consulted & ~torch.isnan(got)
     assert torch.allclose(got[both], ref.rho[both], rtol=2e-5)
+
+
+def test_attention_plan_large_batch_and_long_requests():
+    """The work plan cuts the concatenated tile axis of all (request, kv head) pairs into one range
+    per CTA.  A batch above 1024 requests takes the planner's multi-pass path (prefix sums in
+    global memory, many whole pairs per range); a batch of few long requests makes every pair
+    span several ranges (several partial chunks per pair)."""
+    many = dataclasses.replace(W.CONFIGS[1], batch=1100, vocab=64, ctx=("uniform", 20, 400),
+                               k=("choice", (0, 1, 2, 4)), name="many-short")
+    few = dataclasses.replace(W.CONFIGS[1], batch=3, vocab=64, ctx=("uniform", 9000, 14000),
+                              k=("const", 4), name="few-long")
+    for spec, sample in ((many, 40), (few, None)):
+        b_cpu = W.generate(spec)
+        b = b_cpu.to(DEV)
+        out, lse, ws = gpu_attention(b)
+        assert int(ws.status.item()) == 0
+        reqs = list(range(b_cpu.batch)) if sample is None else list(range(0, b_cpu.batch, b_cpu.batch // sample))
+        ref_o, ref_l = oracle_attention(b_cpu, reqs)
+        check_attention(b_cpu, out, lse, ref_o, ref_l, reqs)
+        assert not torch.isnan(out.float()).any()
 
 
 def test_bf16_variant_of_tiny_workload():
