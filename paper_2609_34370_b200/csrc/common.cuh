@@ -45,11 +45,12 @@ __device__ __forceinline__ float warp_sum(float v) {
 //
 // A pair is one (request, kv head); its KV range is tiles_r tiles of kTileTokens tokens.  The
 // pairs of the valid requests, in (request, head) order, form one tile axis of length T, which is
-// cut into n_cta contiguous ranges of equal length; CTA c of a persistent kernel executes range c
-// (entries cta_off[c] .. cta_off[c+1] of the work list, in axis order).  A cut within kSnapTiles
+// cut into n_cta contiguous ranges of equal cost (tiles plus a fixed cost per entry); CTA c of a
+// persistent kernel executes range c (entries cta_off[c] .. cta_off[c+1] of the work list, in
+// axis order).  A cut within kSnapTiles
 // of a pair boundary moves onto it, so most pairs stay whole; a pair that k cuts cross has k+1
-// chunks, whose partial results the combine kernel merges.  Every CTA gets the same number of
-// tiles to within one, and at most n_cta - 1 pairs are split, whatever the length mix.
+// chunks, whose partial results the combine kernel merges.  At most n_cta - 1 pairs are split,
+// whatever the length mix.
 // ------------------------------------------------------------------------------------------
 constexpr int kSnapTiles = 2;   // a cut this close to a pair boundary is moved onto the boundary
 struct PlanHeader {
