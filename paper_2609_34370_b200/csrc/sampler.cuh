@@ -21,7 +21,7 @@ constexpr int kSegElems = 8192;       // tokens per segment (residual pass, fina
 constexpr int kSubElems = SPX_SUB_ELEMS;  // tokens per sub-segment (statistics pass)
 constexpr int kSubPerSeg = kSegElems / kSubElems;
 constexpr int kSampThreads = 256;
-constexpr int kResidThreads = 256;   // residual kernel: at most 64 registers a thread for bf16 logits, four blocks an SM
+constexpr int kResidThreads = 256;   // residual kernels
 constexpr int kElemsPerThread = kSegElems / kResidThreads;  // 32
 
 struct SampleParams {
@@ -77,6 +77,21 @@ template <> struct Vec<float> {
   }
 };
 
+// Element j of a raw 16-byte vector of logits, times scale.
+template <typename T>
+__device__ __forceinline__ float raw_elem(const uint4 &u, int j, float scale) {
+  const int k = sizeof(T) == 2 ? j >> 1 : j;
+  const uint32_t w = k == 0 ? u.x : k == 1 ? u.y : k == 2 ? u.z : u.w;
+  if (sizeof(T) == 2) return __uint_as_float((j & 1) ? (w & 0xffff0000u) : (w << 16)) * scale;
+  return __uint_as_float(w) * scale;
+}
+
+// 16-byte asynchronous copy global -> shared.  Used for data only the copying thread reads back:
+// cp.async.wait_all orders it, no barrier is needed.
+__device__ __forceinline__ void cp_async16(void *smem, const void *gmem) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+
 // The kElemsPerThread consecutive tokens [v0, v0+32) of a row that a thread owns, kept as raw
 // 16-byte vectors and converted token by token (for bf16 logits half the registers of the converted
 // values).  get(i, scale) is token v0+i in the log2 domain (logit * scale, scale = log2(e) /
@@ -102,13 +117,7 @@ struct RawSpan {
       }
     }
   }
-  __device__ __forceinline__ float get(int i, float scale) const {
-    const uint4 &u = raw[i / N];
-    const int j = sizeof(T) == 2 ? (i % N) >> 1 : i % N;
-    const uint32_t w = j == 0 ? u.x : j == 1 ? u.y : j == 2 ? u.z : u.w;
-    if (sizeof(T) == 2) return __uint_as_float((i & 1) ? (w & 0xffff0000u) : (w << 16)) * scale;
-    return __uint_as_float(w) * scale;
-  }
+  __device__ __forceinline__ float get(int i, float scale) const { return raw_elem<T>(raw[i / N], i % N, scale); }
 };
 
 // Merge two (max, sum) pairs.
@@ -939,25 +948,70 @@ struct ResidCtx {
 // stores: the draw runs as the next kernel of the stream, so no fence or counter sits between a
 // block's loads and its exit (with a last-block-done counter every block paid two more memory
 // round trips, and the step's tail is made of these).
+constexpr int kResidStageBytes = 2 * kSegElems * 2;  // bf16 logits: the block's segment of both rows
 template <typename T, bool kScaled, bool kFiltered>
-__global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_mass_kernel(SampleParams p) {
+__global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 6 : 1) resid_mass_kernel(SampleParams p) {
   const int seg_mine = blockIdx.x, r = blockIdx.y;
   ResidCtx<T, kScaled, kFiltered> c;
   if (!c.init(p, r) || !c.full_pass()) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   __shared__ float s_w[kResidThreads / 32];
   __shared__ float s_wp[kResidThreads / 32];
-  const int v0 = seg_mine * kSegElems + threadIdx.x * kElemsPerThread;
-  RawSpan<T> st, sd;
-  st.issue(c.trow, v0, p.vocab);
-  if (!c.bonus) sd.issue(c.drow, v0, p.vocab);
-  else sd = st;  // never read as a draft row: qd_of() is zero for a bonus request
   float acc = 0.f, accp = 0.f;
+  if constexpr (sizeof(T) == 2) {
+    // bf16 logits: each thread parks its vectors in shared memory with asynchronous copies and
+    // reads them back itself (vector (c, thread) of a row holds tokens (c*256 + thread)*8 ..+8 of
+    // the segment: every copy instruction of a warp covers 512 contiguous bytes).  Nothing of the
+    // segment sits in registers while it is in flight, so six blocks share an SM and the pass
+    // needs about one wave of blocks instead of two.
+    extern __shared__ __align__(16) unsigned char resid_stage[];
+    constexpr int N = 8, NV = kSegElems / N / kResidThreads;
+    uint4 *stg = reinterpret_cast<uint4 *>(resid_stage);  // [row][vector][thread]
+    auto park = [&](const T *row, int which) {
 #pragma unroll
-  for (int i = 0; i < kElemsPerThread; ++i) {
-    const float xt = st.get(i, c.kLoadScale), xd = sd.get(i, c.kLoadScale);
-    acc += c.resid_of(xt, xd);
-    if (kFiltered) accp += c.pt_of(xt);
+      for (int v = 0; v < NV; ++v) {
+        const int e0 = seg_mine * kSegElems + (v * kResidThreads + (int)threadIdx.x) * N;
+        uint4 *dst = stg + (which * NV + v) * kResidThreads + threadIdx.x;
+        if (e0 + N <= p.vocab) {
+          cp_async16(dst, row + e0);
+        } else {
+          union { uint4 u; T e[N]; } tmp;
+#pragma unroll
+          for (int i = 0; i < N; ++i) {
+            if (e0 + i < p.vocab) tmp.e[i] = row[e0 + i];
+            else st_from_float(tmp.e, i, -INFINITY);
+          }
+          *dst = tmp.u;
+        }
+      }
+    };
+    park(c.trow, 0);
+    if (!c.bonus) park(c.drow, 1);
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const uint4 ut = stg[v * kResidThreads + threadIdx.x];
+      // a bonus request has no draft row: qd_of() is zero for it whatever is passed
+      const uint4 ud = c.bonus ? ut : stg[(NV + v) * kResidThreads + threadIdx.x];
+#pragma unroll
+      for (int i = 0; i < N; ++i) {
+        const float xt = raw_elem<T>(ut, i, c.kLoadScale), xd = raw_elem<T>(ud, i, c.kLoadScale);
+        acc += c.resid_of(xt, xd);
+        if (kFiltered) accp += c.pt_of(xt);
+      }
+    }
+  } else {
+    const int v0 = seg_mine * kSegElems + threadIdx.x * kElemsPerThread;
+    RawSpan<T> st, sd;
+    st.issue(c.trow, v0, p.vocab);
+    if (!c.bonus) sd.issue(c.drow, v0, p.vocab);
+    else sd = st;  // never read as a draft row: qd_of() is zero for a bonus request
+#pragma unroll
+    for (int i = 0; i < kElemsPerThread; ++i) {
+      const float xt = st.get(i, c.kLoadScale), xd = sd.get(i, c.kLoadScale);
+      acc += c.resid_of(xt, xd);
+      if (kFiltered) accp += c.pt_of(xt);
+    }
   }
   acc = warp_sum(acc);
   if (kFiltered) accp = warp_sum(accp);

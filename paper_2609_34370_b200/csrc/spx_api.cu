@@ -414,7 +414,7 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
     }
     const int accept_blocks = (p.batch * 32 + 127) / 128;
     accept_kernel<T, kScaled, kFiltered><<<accept_blocks + (kScaled ? p.batch : 0), 128, 0, stream>>>(p, accept_blocks);
-    resid_mass_kernel<T, kScaled, kFiltered><<<dim3(p.nseg, p.batch), kResidThreads, 0, stream>>>(p);
+    resid_mass_kernel<T, kScaled, kFiltered><<<dim3(p.nseg, p.batch), kResidThreads, sizeof(T) == 2 ? kResidStageBytes : 0, stream>>>(p);
     if (launch_pdl(resid_pick_kernel<T, kScaled, kFiltered>, dim3(p.batch), dim3(kResidThreads), 0, stream, p) != cudaSuccess)
       return SPX_ERR_CUDA;
     t_launches += 3;
