@@ -35,7 +35,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one verify-attention launch, from the ncu
 # captures summarised under profiles/ (None until captured for that workload).
-NCU_TRAFFIC_BYTES = {"llama3-8b": 633.7e6}  # profiles/launch_list_llama3-8b.txt: 622.1 MB read + 11.6 MB written
+NCU_TRAFFIC_BYTES = {"llama3-8b": 625.2e6}  # profiles/launch_list_llama3-8b.txt: 621.7 MB read + 3.5 MB written
 
 
 def measured_peak():
