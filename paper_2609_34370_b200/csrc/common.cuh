@@ -45,7 +45,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 //
 // A pair is one (request, kv head); its KV range is tiles_r tiles of kTileTokens tokens.  The
 // pairs of the valid requests, in (request, head) order, form one tile axis of length T, which is
-// cut into n_cta contiguous ranges of equal cost (tiles plus a fixed cost per entry); CTA c of a
+// cut into n_cta contiguous ranges of equal cost (tiles plus a fixed cost per pair); CTA c of a
 // persistent kernel executes range c (entries cta_off[c] .. cta_off[c+1] of the work list, in
 // axis order).  A cut within kSnapTiles
 // of a pair boundary moves onto it, so most pairs stay whole; a pair that k cuts cross has k+1
@@ -92,6 +92,7 @@ struct AttnParams {
   int32_t *pair_part_base; // [B*Hkv]  first partial slot of a split pair
   int32_t *tile_prefix;    // [B+1]  tiles of the requests before r (one kv head)
   int32_t *valid_prefix;   // [B+1]  valid requests before r
+  int32_t *cost_prefix;    // [B+1]  planning cost (one kv head) of the requests before r
   int32_t *cta_off;        // [n_cta+1]  work entries of the CTAs before c
   int32_t *req_bad;        // [B]  set when a needed page id was out of range
   int32_t head_inner;      // tensor-map dimension order: 1 = (d, head, token, page), 0 = (d, token, head, page)

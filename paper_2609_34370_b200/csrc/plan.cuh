@@ -33,9 +33,12 @@ __device__ __forceinline__ int block_exclusive_scan_1024(int v, int *scratch, in
 }
 
 constexpr int kPlanMaxCta = 256;  // ranges the planner can cut the tile axis into
-// Cost of a work entry in quarter tiles: measured on the Llama-3-70B shape (many one- and two-tile
-// pairs), an entry costs about 1.3 tile times on top of its tiles.
-constexpr int kCostPerTile = 4, kCostPerItem = 5;
+// Cost of a pair on the axis the cuts are placed on, in quarter tiles: its tiles plus a fixed part
+// that is larger for short pairs, whose tiles do not overlap with anything.  Fitted to per-CTA run
+// times of the attention kernel on the Llama-3-8B, Llama-3-70B and mixed-length shapes: 0.3-0.4
+// tile times per entry, 0.65 for pairs of 3-6 tiles, 1.1-1.6 for pairs of one or two tiles.
+constexpr int kCostPerTile = 4;
+__device__ __forceinline__ int plan_entry_cost(int tiles) { return tiles <= 2 ? 6 : tiles <= 6 ? 3 : 1; }
 
 // One block.  Validates each request's (k+1, L, page count), cuts the tile axis of the valid
 // requests' (request, kv head) pairs into n_cta ranges of equal length, lays out partial-result
@@ -47,20 +50,21 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int n_cta) {
   __shared__ int s_cut_vq[kPlanMaxCta + 1];  // index, among the valid requests' pairs, of the first pair that ends after cut c
   __shared__ int s_cut_in[kPlanMaxCta + 1];  // 1: cut c lies strictly inside that pair
   __shared__ int s_off[kPlanMaxCta + 1];     // work entries of the ranges before c
-  __shared__ int s_carry_t, s_carry_v, s_carry_p, s_bad;
+  __shared__ int s_carry_t, s_carry_v, s_carry_c, s_carry_p, s_bad;
   // The prefix sums of a batch of up to kPlanSmemReqs requests stay in shared memory: the searches
   // below would otherwise be chains of global loads, each a memory round trip beside the
   // bandwidth-bound kernel that runs while the plan is made (29 us instead of 6 for 64 requests).
   constexpr int kPlanSmemReqs = 1024;
-  __shared__ int s_tp[kPlanSmemReqs + 1], s_vp[kPlanSmemReqs + 1];
+  __shared__ int s_tp[kPlanSmemReqs + 1], s_vp[kPlanSmemReqs + 1], s_cp[kPlanSmemReqs + 1];
   __shared__ int s_q0[kPlanSmemReqs], s_m[kPlanSmemReqs], s_L[kPlanSmemReqs];
   const bool in_smem = p.batch <= kPlanSmemReqs;
   auto tile_prefix = [&](int i) -> int { return in_smem ? s_tp[i] : p.tile_prefix[i]; };
   auto valid_prefix = [&](int i) -> int { return in_smem ? s_vp[i] : p.valid_prefix[i]; };
+  auto cost_prefix = [&](int i) -> int { return in_smem ? s_cp[i] : p.cost_prefix[i]; };  // per kv head
   const int tid = threadIdx.x;
   const int Hkv = p.Hkv;
   if (n_cta > kPlanMaxCta) n_cta = kPlanMaxCta;
-  if (tid == 0) { s_carry_t = 0; s_carry_v = 0; s_carry_p = 0; s_bad = 0; }
+  if (tid == 0) { s_carry_t = 0; s_carry_v = 0; s_carry_c = 0; s_carry_p = 0; s_bad = 0; }
   __syncthreads();
 
   // pass 1: validate; prefix sums of tiles and of valid requests
@@ -82,24 +86,28 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int n_cta) {
     const int tot_t = s_total;
     const int off_v = block_exclusive_scan_1024(tiles > 0 ? 1 : 0, s_scratch, &s_total) + s_carry_v;
     const int tot_v = s_total;
+    const int cost = tiles > 0 ? kCostPerTile * tiles + plan_entry_cost(tiles) : 0;
+    const int off_c = block_exclusive_scan_1024(cost, s_scratch, &s_total) + s_carry_c;
+    const int tot_c = s_total;
     if (r < p.batch) {
-      if (in_smem) { s_tp[r] = off_t; s_vp[r] = off_v; }
-      else { p.tile_prefix[r] = off_t; p.valid_prefix[r] = off_v; }
+      if (in_smem) { s_tp[r] = off_t; s_vp[r] = off_v; s_cp[r] = off_c; }
+      else { p.tile_prefix[r] = off_t; p.valid_prefix[r] = off_v; p.cost_prefix[r] = off_c; }
     }
     __syncthreads();
-    if (tid == 0) { s_carry_t += tot_t; s_carry_v += tot_v; }
+    if (tid == 0) { s_carry_t += tot_t; s_carry_v += tot_v; s_carry_c += tot_c; }
     __syncthreads();
   }
   if (tid == 0) {
-    if (in_smem) { s_tp[p.batch] = s_carry_t; s_vp[p.batch] = s_carry_v; }
-    else { p.tile_prefix[p.batch] = s_carry_t; p.valid_prefix[p.batch] = s_carry_v; }
+    if (in_smem) { s_tp[p.batch] = s_carry_t; s_vp[p.batch] = s_carry_v; s_cp[p.batch] = s_carry_c; }
+    else { p.tile_prefix[p.batch] = s_carry_t; p.valid_prefix[p.batch] = s_carry_v; p.cost_prefix[p.batch] = s_carry_c; }
     if (s_bad) atomicOr(p.dev_status, SPX_DEV_BAD_LEN);
   }
   __syncthreads();  // the prefix arrays are read back below (same block: visible after the barrier)
   const long long total_tiles = s_carry_t;
   const long long T = total_tiles * Hkv;
   const int n_valid_pairs = s_carry_v * Hkv;
-  const bool too_long = T >= (1ll << 30);
+  const long long Tw = (long long)s_carry_c * Hkv;  // length of the cost axis
+  const bool too_long = T >= (1ll << 30) || s_carry_c >= (1 << 30) || s_carry_c < 0;
   const bool may_split = T >= 2ll * kSnapTiles * n_cta;  // cuts inside pairs are then distinct
 
   // pass 2: the cuts.  Thread c places cut c at c*T/n_cta, finds the pair it falls in and moves it
@@ -111,26 +119,23 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int n_cta) {
     } else if (tid == n_cta) {
       cut = (int)T; vq = n_valid_pairs;
     } else {
-      // the cut is placed on the cost axis (a pair costs kCostPerItem + kCostPerTile per tile),
-      // so that a range of many short pairs gets fewer tiles than a range inside one long pair
-      const long long Tw = (long long)kCostPerTile * T + (long long)kCostPerItem * n_valid_pairs;
+      // the cut is placed on the cost axis, so that a range of many short pairs gets fewer tiles
+      // than a range inside one long pair
       const long long x = (long long)tid * Tw / n_cta;
-      auto wbase = [&](int i) -> long long {
-        return (long long)Hkv * ((long long)kCostPerTile * tile_prefix(i) + (long long)kCostPerItem * valid_prefix(i));
-      };
-      // largest r with wbase(r) <= x (a request with tiles, since x < Tw)
+      // largest r with Hkv * cost_prefix(r) <= x (a request with tiles, since x < Tw)
       int lo = 0, hi = p.batch - 1;
       while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
-        if (wbase(mid) <= x) lo = mid; else hi = mid - 1;
+        if ((long long)cost_prefix(mid) * Hkv <= x) lo = mid; else hi = mid - 1;
       }
       const int r = lo;
       const int tp = tile_prefix(r), tiles = tile_prefix(r + 1) - tp;
-      const int pair_cost = kCostPerTile * tiles + kCostPerItem;
-      const int rel = (int)(x - wbase(r));
+      const int pair_cost = cost_prefix(r + 1) - cost_prefix(r);
+      const int entry_cost = pair_cost - kCostPerTile * tiles;
+      const int rel = (int)(x - (long long)cost_prefix(r) * Hkv);
       int g = rel / pair_cost;
       const int offw = rel - g * pair_cost;
-      int off = offw < kCostPerItem ? 0 : (offw - kCostPerItem) / kCostPerTile;
+      int off = offw < entry_cost ? 0 : (offw - entry_cost) / kCostPerTile;
       if (!may_split || off < kSnapTiles) off = 0;
       else if (tiles - off < kSnapTiles) { off = 0; ++g; }  // onto the end of the pair = the start of the next
       inside = off > 0;

@@ -75,7 +75,7 @@ constexpr int kPlanSmCount = 148;  // workspace sizing must not depend on a devi
 // workspace layout
 // ---------------------------------------------------------------------------------------------
 struct AttnWs {
-  size_t hdr, nchunks, part_base, tile_prefix, valid_prefix, cta_off, req_bad, work, part_ml, part_o, total;
+  size_t hdr, nchunks, part_base, tile_prefix, valid_prefix, cost_prefix, cta_off, req_bad, work, part_ml, part_o, total;
   int32_t max_work, max_part_slots, rows_cap;
 };
 
@@ -119,6 +119,7 @@ static AttnWs attn_ws_layout(const spx_attn_args_t *a) {
   w.part_base = off; off = align_up(off + sizeof(int32_t) * pairs, 256);
   w.tile_prefix = off; off = align_up(off + sizeof(int32_t) * ((size_t)a->batch + 1), 256);
   w.valid_prefix = off; off = align_up(off + sizeof(int32_t) * ((size_t)a->batch + 1), 256);
+  w.cost_prefix = off; off = align_up(off + sizeof(int32_t) * ((size_t)a->batch + 1), 256);
   w.cta_off = off; off = align_up(off + sizeof(int32_t) * (kPlanSmCount + 1), 256);
   w.req_bad = off; off = align_up(off + sizeof(int32_t) * (size_t)a->batch, 256);
   w.work = off; off = align_up(off + sizeof(WorkEntry) * (size_t)w.max_work, 256);
@@ -296,6 +297,7 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
   p.pair_part_base = reinterpret_cast<int32_t *>(ws + w.part_base);
   p.tile_prefix = reinterpret_cast<int32_t *>(ws + w.tile_prefix);
   p.valid_prefix = reinterpret_cast<int32_t *>(ws + w.valid_prefix);
+  p.cost_prefix = reinterpret_cast<int32_t *>(ws + w.cost_prefix);
   p.cta_off = reinterpret_cast<int32_t *>(ws + w.cta_off);
   p.req_bad = reinterpret_cast<int32_t *>(ws + w.req_bad);
   p.work = reinterpret_cast<WorkEntry *>(ws + w.work);
