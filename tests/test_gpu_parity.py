@@ -210,6 +210,33 @@ def test_device_side_faults_are_reported_not_fatal():
     assert torch.equal(acc[1:].cpu(), ref.accepted_len[1:]) and torch.equal(tok[q1:].cpu(), ref.out_tokens[q1:])
 
 
+def test_vocabulary_beyond_the_staged_segment_masses():
+    """A vocabulary of more than 128 segments of 8192 tokens: the draw reads the segment masses
+    beyond its shared-memory staging array in place.  Three requests: one rejected early (the
+    residual draw lands in a late segment for u_sample near 1), one bonus draw, one k = 0."""
+    V = 8192 * 130 + 40
+    g = torch.Generator().manual_seed(11)
+    T = (torch.randn(5, V, generator=g) * 2).to(torch.bfloat16)
+    qi = torch.tensor([0, 2, 4, 5], dtype=torch.int32)                  # k = 1, 1, 0
+    Dr = torch.stack([T[0].roll(7), T[2]]).clone()                      # request 0: another law; request 1: q == p
+    ids = torch.tensor([int(torch.argmax(Dr[0].float())), 123], dtype=torch.int32)
+    ua = torch.tensor([0.999999, 0.5])
+    for us_val in (0.003, 0.5, 1 - 2.0 ** -20):
+        us = torch.full((3,), us_val)
+        ref = oracle.rejection_sample(T, Dr, ids, qi, ua, us)
+        acc, tok, _, ws = spx.rejection_sample(T.to(DEV), Dr.to(DEV), ids.to(DEV), qi.to(DEV), ua.to(DEV), us.to(DEV))
+        torch.cuda.synchronize()
+        assert int(ws.status.item()) == 0
+        assert ref.accepted_len.tolist() == [0, 1, 0]
+        assert torch.equal(acc.cpu(), ref.accepted_len)
+        b = type("B", (), {})()
+        b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample = T, Dr, ids, qi, ua, us
+        b.batch = 3
+        b.spec = type("S", (), {"vocab": V})
+        rep = check_sampling(b, acc, tok, ref)
+        assert not rep.hard_mismatch, rep
+
+
 def test_sampler_special_cases_on_gpu():
     # q == p accepts everything; disjoint supports reject at 0; k = 0 plain sampling; u_sample extremes
     V = 9000
