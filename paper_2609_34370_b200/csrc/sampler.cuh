@@ -498,35 +498,6 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
   };
   auto mass_of = [&](float x) -> unsigned long long { return __float2ull_rn(fast_exp2(fmaf(x, scale, -M)) * kMassScale); };
 
-  // level 0: the whole row into the per-lane copies, then their sums into s_cnt / s_mass
-  for (int i = tid; i < 4 * 256 * 32; i += kFilterThreads) h_cnt[i] = 0;   // the four arrays are contiguous
-  __syncthreads();
-  sweep_row<T>(base, p.vocab, tid, [&](float x) {
-    const uint32_t slot = bin0_of(x) * 32 + lane;
-    if (use_k) atomicAdd(&h_cnt[slot], 1u);
-    if (use_p) {
-      const unsigned long long m = mass_of(x);
-      atomicAdd(&h_m0[slot], (uint32_t)(m & 0x7fffull));
-      atomicAdd(&h_m1[slot], (uint32_t)((m >> 15) & 0x7fffull));
-      atomicAdd(&h_m2[slot], (uint32_t)(m >> 30));
-    }
-  });
-  __syncthreads();
-  if (tid < 256) {
-    uint32_t c = 0;
-    unsigned long long m = 0ull;
-    for (int j = 0; j < 32; ++j) {
-      const int slot = tid * 32 + ((j + tid) & 31);
-      c += h_cnt[slot];
-      m += (unsigned long long)h_m0[slot] + ((unsigned long long)h_m1[slot] << 15) + ((unsigned long long)h_m2[slot] << 30);
-    }
-    s_cnt[tid] = s_cnt1[tid] = c;
-    s_mass[tid] = s_mass1[tid] = m;
-  }
-  __syncthreads();
-  unsigned long long total = 0ull;
-  for (int b = 0; b < 256; ++b) total += s_mass1[b];   // every thread: 256 broadcast reads
-
   // warp 0: the highest bin b such that (count or mass of bins >= b, plus what lies above the
   // prefix) reaches the target; leaves the bin, and count / mass of the bins above it, in shared memory
   auto pick = [&](bool by_count, uint32_t need_cnt, double need_mass, unsigned long long mass_above_prefix) {
@@ -571,6 +542,109 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
     }
     __syncthreads();
   };
+
+  // Exact key-byte levels over the n_list logits in s_list (every level narrows the key by one
+  // byte; after the last the key is complete).  Returns the threshold key, *Z the mass at or above it.
+  auto levels_over_list = [&](bool by_count, uint32_t need, double need_mass, uint32_t n_list, unsigned long long *Z) -> uint32_t {
+    uint32_t prefix = 0;
+    unsigned long long above = 0ull;
+    for (int level = 1; level <= kLevels; ++level) {
+      const int shift = kKeyShift + 8 * (kLevels - level);
+      if (tid < 256) { s_cnt[tid] = 0; s_mass[tid] = 0ull; }
+      __syncthreads();
+      for (uint32_t i = tid; i < n_list; i += kFilterThreads) {
+        const float x = s_list[i];
+        const uint32_t key = order_key32(x);
+        if (level > 1 && (key >> (shift + 8)) != (prefix >> (shift + 8))) continue;
+        const uint32_t bin = (key >> shift) & 255u;
+        atomicAdd(&s_cnt[bin], 1u);
+        atomicAdd(&s_mass[bin], mass_of(x));
+      }
+      __syncthreads();
+      pick(by_count, need, need_mass, above);
+      prefix |= s_bin << shift;
+      need -= s_above_cnt;
+      above += s_above_mass;
+      if (level == kLevels) *Z = above + s_bin_mass;
+      __syncthreads();
+    }
+    return prefix;
+  };
+
+  // top-k with K no larger than the number of sub-segments of the row: the K-th largest of the
+  // sub-segment maxima (known from the statistics pass) is a lower bound of the K-th largest
+  // logit, so one compare-only sweep collects every candidate (a few hundred logits for K = 50
+  // on a 128k vocabulary) and the exact levels run over that list - no histogram of the whole row.
+  // A list that overflows (many equal logits) falls back to the general path below.
+  if (use_k && tk_raw <= p.nsub && p.nsub <= kFilterThreads) {
+    __shared__ float s_bound;
+    const float2 *st = p.seg_stats + (int64_t)row * p.nsub;
+    if (tid < p.nsub) {
+      const float mine = st[tid].x;
+      int rank = 0;
+      for (int j = 0; j < p.nsub; ++j) {
+        const float o = st[j].x;
+        rank += (o > mine || (o == mine && j < tid)) ? 1 : 0;
+      }
+      if (rank == tk_raw - 1) s_bound = mine;
+    }
+    if (tid == 0) s_list_n = 0;
+    __syncthreads();
+    const float bound = s_bound - (fabsf(s_bound) * 1e-6f + 1e-6f);  // in the scaled (log2) domain, like the statistics
+    sweep_row<T>(base, p.vocab, tid, [&](float x) {
+      if (x * scale >= bound) {
+        const uint32_t i = atomicAdd(&s_list_n, 1u);
+        if (i < (uint32_t)kFilterListCap) s_list[i] = x;
+      }
+    });
+    __syncthreads();
+    const uint32_t n_list = s_list_n;
+    if (n_list <= (uint32_t)kFilterListCap) {
+      unsigned long long Zk = 0ull, Zf = 0ull;
+      const uint32_t Tk = levels_over_list(true, (uint32_t)tk_raw, 0.0, n_list, &Zk);
+      uint32_t Tf = Tk;
+      Zf = Zk;
+      if (use_p) {
+        Tf = levels_over_list(false, 0u, (double)tp * (double)Zk, n_list, &Zf);
+        if (Tf < Tk) { Tf = Tk; Zf = Zk; }
+      }
+      if (tid == 0) {
+        p.row_thresh[row] = Tf;
+        p.row_z[row] = (double)Zf / (double)kMassScale;
+      }
+      return;
+    }
+    __syncthreads();
+  }
+
+  // level 0: the whole row into the per-lane copies, then their sums into s_cnt / s_mass
+  for (int i = tid; i < 4 * 256 * 32; i += kFilterThreads) h_cnt[i] = 0;   // the four arrays are contiguous
+  __syncthreads();
+  sweep_row<T>(base, p.vocab, tid, [&](float x) {
+    const uint32_t slot = bin0_of(x) * 32 + lane;
+    if (use_k) atomicAdd(&h_cnt[slot], 1u);
+    if (use_p) {
+      const unsigned long long m = mass_of(x);
+      atomicAdd(&h_m0[slot], (uint32_t)(m & 0x7fffull));
+      atomicAdd(&h_m1[slot], (uint32_t)((m >> 15) & 0x7fffull));
+      atomicAdd(&h_m2[slot], (uint32_t)(m >> 30));
+    }
+  });
+  __syncthreads();
+  if (tid < 256) {
+    uint32_t c = 0;
+    unsigned long long m = 0ull;
+    for (int j = 0; j < 32; ++j) {
+      const int slot = tid * 32 + ((j + tid) & 31);
+      c += h_cnt[slot];
+      m += (unsigned long long)h_m0[slot] + ((unsigned long long)h_m1[slot] << 15) + ((unsigned long long)h_m2[slot] << 30);
+    }
+    s_cnt[tid] = s_cnt1[tid] = c;
+    s_mass[tid] = s_mass1[tid] = m;
+  }
+  __syncthreads();
+  unsigned long long total = 0ull;
+  for (int b = 0; b < 256; ++b) total += s_mass1[b];   // every thread: 256 broadcast reads
 
   // One descent.  On entry s_cnt / s_mass hold level 0.  Returns the threshold key; *Z receives the
   // mass at or above it (meaningful only when masses were kept at level 0, i.e. use_p).
