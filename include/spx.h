@@ -368,6 +368,26 @@ void spx_set_timing_events(void *start_event, void *stop_event);
 /* Number of kernels the last call on this thread enqueued (for launch accounting). */
 int32_t spx_last_launch_count(void);
 
+/*
+ * Inspection aid: where, inside the workspace of spx_verify_attention / spx_verify_step, the
+ * attention work plan lies after a call with these arguments (the attention part comes first in
+ * the workspace of spx_verify_step).  The plan cuts the 128-token tiles of all (request, kv head)
+ * pairs, in (request, head) order, into one contiguous range per CTA of the persistent attention
+ * kernel.  Writes byte offsets and sizes into out[0..7] (host memory):
+ *   out[0] header: int32 n_work, n_cta, n_part_slots, total_tiles, (cursor), overflow
+ *   out[1] cta_off: int32[n_cta + 1], entries of the work list that belong to the CTAs before c
+ *   out[2] work list: 32-byte entries of int32 {req, tile_begin, tile_end, part_slot (-1: the pair
+ *          is not split), q0, m, L, kv_head}
+ *   out[3] capacity of the work list (entries)
+ *   out[4] pair_nchunks: int32[batch * num_kv_heads], chunks of each pair (0: invalid request)
+ *   out[5] pair_part_base: int32[batch * num_kv_heads], first partial slot of a split pair, else -1
+ *   out[6] capacity in partial slots
+ *   out[7] bytes of the attention part of the workspace
+ * Returns SPX_ERR_INVALID_ARG / SPX_ERR_UNSUPPORTED as spx_workspace_size would refuse the
+ * arguments.  Used by the tests to check the plan's invariants; nothing else depends on it.
+ */
+spx_status_t spx_plan_layout(const spx_attn_args_t *attn, int64_t *out);
+
 #ifdef __cplusplus
 }
 #endif

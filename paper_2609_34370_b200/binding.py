@@ -16,7 +16,7 @@ BF16, F32 = 0, 1
 
 EXPORTS = ("spx_workspace_size", "spx_verify_attention", "spx_rejection_sample", "spx_verify_step",
            "spx_host_step_arena_size", "spx_verify_step_host", "spx_status_string", "spx_last_launch_count",
-           "spx_set_timing_events", "spx_rejection_sample_static", "spx_kv_append", "spx_kv_rollback",
+           "spx_set_timing_events", "spx_plan_layout", "spx_rejection_sample_static", "spx_kv_append", "spx_kv_rollback",
            "spx_draft_confidence_workspace", "spx_draft_confidence", "spx_select_speculation",
            "spx_lookahead_memory", "spx_sp_effective_batch", "spx_selective_batch", "spx_selective_effective_batch",
            "spx_delay_gain", "spx_lm_head")
@@ -112,6 +112,8 @@ def load_library():
         lib.spx_status_string.restype = C.c_char_p
         lib.spx_status_string.argtypes = [C.c_int]
         lib.spx_last_launch_count.restype = C.c_int32
+        lib.spx_plan_layout.restype = C.c_int
+        lib.spx_plan_layout.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
         lib.spx_rejection_sample_static.restype = C.c_int
         lib.spx_rejection_sample_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         lib.spx_kv_append.restype = C.c_int
@@ -303,6 +305,14 @@ def host_step_arena_size(attn: AttnArgs, sample: SampleArgs, kv_pool_elems: int)
     if n == 0:
         raise SpxError(ERR_INVALID_ARG, "invalid arguments for arena sizing")
     return int(n)
+
+
+def plan_layout(attn_args) -> dict:
+    """spx_plan_layout: byte offsets of the attention work plan inside the workspace."""
+    out = (C.c_int64 * 8)()
+    _check(load_library().spx_plan_layout(C.byref(attn_args), out))
+    keys = ("header", "cta_off", "work", "max_work", "pair_nchunks", "pair_part_base", "max_part_slots", "attn_bytes")
+    return dict(zip(keys, (int(v) for v in out)))
 
 
 def last_launch_count() -> int:

@@ -878,6 +878,16 @@ void spx_set_timing_events(void *start_event, void *stop_event) {
 
 int32_t spx_last_launch_count(void) { return t_launches; }
 
+spx_status_t spx_plan_layout(const spx_attn_args_t *attn, int64_t *out) {
+  if (!out) return SPX_ERR_INVALID_ARG;
+  const spx_status_t st = check_attn(attn, false);
+  if (st != SPX_OK) return st;
+  const AttnWs w = attn_ws_layout(attn);
+  out[0] = (int64_t)w.hdr; out[1] = (int64_t)w.cta_off; out[2] = (int64_t)w.work; out[3] = w.max_work;
+  out[4] = (int64_t)w.nchunks; out[5] = (int64_t)w.part_base; out[6] = w.max_part_slots; out[7] = (int64_t)w.total;
+  return SPX_OK;
+}
+
 #if SPX_PROFILE
 // Profiling builds only (not declared in spx.h): per-CTA cycle counters of the attention kernel.
 void spx_debug_set_profile_buffer(long long *device_buffer) { t_prof = device_buffer; }
