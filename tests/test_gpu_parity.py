@@ -117,6 +117,41 @@ def test_verify_step_equals_the_two_halves_and_is_deterministic():
         assert torch.equal(acc, acc_a) and torch.equal(tok, tok_a)
 
 
+def test_verify_step_can_be_captured_in_a_cuda_graph():
+    """The step only enqueues work (its internal stream is forked from and joined to the caller's
+    stream by events), so a stream capture of one call replays it: same outputs, bit for bit."""
+    from paper_2609_34370_b200 import binding
+    spec = W.scaled(W.CONFIGS[1], batch=12, ctx_div=4, vocab=50000)
+    b = W.generate(spec).to(DEV)
+    out = torch.empty_like(b.q)
+    lse = torch.empty(b.q.shape[:2], dtype=torch.float32, device=DEV)
+    acc = torch.empty(b.batch, dtype=torch.int32, device=DEV)
+    tok = torch.empty(b.total_q, dtype=torch.int32, device=DEV)
+    a = binding.make_attn_args(b.q, b.k_cache, b.v_cache, b.kv_strides, b.block_table, b.seq_lens, b.q_indptr,
+                               spec.num_kv_heads, spec.page_size, b.num_pages, out, lse)
+    sa = binding.make_sample_args(b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample,
+                                  acc, tok)
+    ws = spx.Workspace.allocate(spx.workspace_size(a, sa), DEV)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for _ in range(3):                         # warm-up outside the capture (function attributes, side stream)
+            spx.verify_step(a, sa, ws, DEV)
+    torch.cuda.synchronize()
+    want = (out.clone(), lse.clone(), acc.clone(), tok.clone())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        spx.verify_step(a, sa, ws, DEV)
+    torch.cuda.synchronize()
+    for t in (out, lse, acc, tok):
+        t.zero_()
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert int(ws.status.item()) == 0
+    for got, ref in zip((out, lse, acc, tok), want):
+        assert torch.equal(got, ref)
+
+
 def test_edge_cases_k0_minimal_context_and_page_boundaries():
     # hand-made lengths: L = k+1 (no prior context), L exactly on page/tile boundaries, k = 0, k = 15
     import dataclasses
