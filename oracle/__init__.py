@@ -281,10 +281,13 @@ def emit_cdf(r: int, n: int, target_logits: torch.Tensor, draft_logits: torch.Te
 
 def kv_append(new_k: torch.Tensor, new_v: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
               kv_strides: Sequence[int], block_table: torch.Tensor, seq_lens: torch.Tensor, q_indptr: torch.Tensor,
-              page_size: int, num_pages: int) -> None:
-    """Write the new positions' K/V ([TQ, Hkv, D]) into their pages, in place (bit copies)."""
+              page_size: int, num_pages: int, rope_base: float = 0.0) -> None:
+    """Write the new positions' K/V ([TQ, Hkv, D]) into their pages, in place (bit copies).  With
+    rope_base > 0 the K rows are rotated to their absolute positions first (V is not)."""
     lib = _load()
     nk, nv = _cpu(new_k).contiguous(), _cpu(new_v).contiguous()
+    if rope_base > 0.0:
+        nk = round_to(rope(nk, new_positions(seq_lens, q_indptr), rope_base), nk.dtype).contiguous()
     assert nk.dtype == k_cache.dtype == v_cache.dtype == nv.dtype
     _dtype_code(nk)
     TQ, Hkv, D = nk.shape
@@ -296,6 +299,38 @@ def kv_append(new_k: torch.Tensor, new_v: torch.Tensor, k_cache: torch.Tensor, v
                               int(kv_strides[1]), int(kv_strides[2]), _ptr(bt), _ptr(sl), _ptr(qi))
     if st != OK:
         raise OracleError(st)
+
+
+def rope(x: torch.Tensor, positions: torch.Tensor, base: float) -> torch.Tensor:
+    """Rotary embedding of x [rows, H, D] at the given absolute positions; float64 result."""
+    lib = _load()
+    xc = _cpu(x).contiguous()
+    rows, H, D = xc.shape
+    pos = _cpu(positions, torch.int32).contiguous()
+    assert pos.numel() == rows
+    out = torch.empty(rows, H, D, dtype=torch.float64)
+    lib.oracle_rope_rows.argtypes = [c.c_void_p, c.c_int32, c.c_int64, c.c_int32, c.c_int32, c.c_void_p, c.c_double,
+                                     c.c_void_p]
+    st = lib.oracle_rope_rows(_ptr(xc), _dtype_code(xc), rows, H, D, _ptr(pos), float(base), _ptr(out))
+    if st != OK:
+        raise OracleError(st)
+    return out
+
+
+def new_positions(seq_lens: torch.Tensor, q_indptr: torch.Tensor) -> torch.Tensor:
+    """Absolute position of every new row: row q_indptr[r]+j is token L_r-(k_r+1)+j of request r."""
+    sl, qi = _cpu(seq_lens, torch.int32).tolist(), _cpu(q_indptr, torch.int32).tolist()
+    pos = torch.empty(qi[-1], dtype=torch.int32)
+    for r, L in enumerate(sl):
+        m = qi[r + 1] - qi[r]
+        for j in range(m):
+            pos[qi[r] + j] = L - m + j
+    return pos
+
+
+def round_to(x64: torch.Tensor, dtype: torch.dtype) -> torch.Tensor:
+    """double -> binary32 -> dtype, each step round-to-nearest-even (what the CUDA path does)."""
+    return x64.to(torch.float32).to(dtype)
 
 
 def kv_rollback(seq_lens: torch.Tensor, q_indptr: torch.Tensor, accepted_len: torch.Tensor) -> torch.Tensor:

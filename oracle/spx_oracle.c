@@ -902,6 +902,36 @@ int oracle_kv_append(int32_t batch, int32_t Hkv, int32_t D, int32_t P, int64_t n
 }
 
 /*
+ * Rotary position embedding of rows of heads (the optional fusion of the append: the paper is
+ * silent on positional encoding; this is the rotation the Llama / Qwen families it evaluates
+ * use).  For a row at absolute position t, every head vector x of even length D is rotated pairwise,
+ * pair i = (x[i], x[i + D/2]), i < D/2, by the angle t * base^(-2i/D):
+ *   y[i]       = x[i] cos a - x[i + D/2] sin a
+ *   y[i + D/2] = x[i + D/2] cos a + x[i] sin a.
+ * Inputs widened exactly, everything in double, output double [rows, H, D] (the caller rounds to
+ * the cache's type: double -> binary32 -> bf16, each round-to-nearest-even).
+ */
+int oracle_rope_rows(const void *x, int32_t dtype, int64_t rows, int32_t H, int32_t D, const int32_t *pos,
+                     double base, double *out) {
+  if (rows < 0 || H <= 0 || D <= 0 || (D & 1) || !(base > 0.0)) return ORACLE_ERR_ARG;
+  const int half = D / 2;
+  for (int64_t r = 0; r < rows; ++r) {
+    if (pos[r] < 0) return ORACLE_ERR_LEN;
+    for (int h = 0; h < H; ++h) {
+      const int64_t o = (r * H + h) * D;
+      for (int i = 0; i < half; ++i) {
+        const double a = (double)pos[r] * pow(base, -2.0 * (double)i / (double)D);
+        const double c = cos(a), sn = sin(a);
+        const double x0 = widen(x, dtype, o + i), x1 = widen(x, dtype, o + i + half);
+        out[o + i] = x0 * c - x1 * sn;
+        out[o + i + half] = x1 * c + x0 * sn;
+      }
+    }
+  }
+  return ORACLE_OK;
+}
+
+/*
  * Rollback: of the k_r+1 new positions, position 0 (the last committed token) and the n_r accepted
  * drafts stay in the cache; the k_r - n_r rejected drafts' entries are dropped by shrinking the
  * length (Figure 3 of the paper: accepted speculation continues, rejected speculation is
