@@ -207,6 +207,10 @@ def time_extras(spx, binding, spec, b, attn_args, dev, iters: int = 200):
     out["kv_append_us"] = timed(lambda: spx.kv_append(new_k, new_v, k_pool, v_pool, b.kv_strides, b.block_table, b.seq_lens,
                                                       b.q_indptr, spec.page_size, b.num_pages, status=status))
     out["kv_append_bytes"] = 2 * new_k.numel() * new_k.element_size() * 2
+    q_rot = b.q.clone()
+    out["kv_append_rope_us"] = timed(lambda: spx.kv_append(new_k, new_v, k_pool, v_pool, b.kv_strides, b.block_table, b.seq_lens,
+                                                           b.q_indptr, spec.page_size, b.num_pages, status=status,
+                                                           rope_base=500000.0, q_rows=q_rot))
     base = binding.make_sample_args(b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample, acc, tok)
     ws = spx.Workspace.allocate(spx.workspace_size(attn_args, base), dev)
     lib = spx.load_library()

@@ -197,6 +197,17 @@ spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_
  * page id set SPX_DEV_BAD_LEN / SPX_DEV_BAD_PAGE and are skipped.  Pools and strides as in
  * spx_attn_args_t; head_dim * element size must be a multiple of 16 bytes.
  *
+ * Optional rotary embedding on the way (the paper does not discuss positional encoding; this is
+ * the rotation of the Llama and Qwen families it evaluates): with rope_base > 0 every new K row is
+ * rotated to its absolute position t before it is stored - for each head vector x and i < D/2,
+ * with a = t * rope_base^(-2i/D):  y[i] = x[i] cos a - x[i+D/2] sin a,  y[i+D/2] = x[i+D/2] cos a +
+ * x[i] sin a, computed in float64 and rounded float64 -> binary32 -> kv_dtype (nearest-even each).
+ * V is copied as it is.  If q_rows is given ([TQ, num_q_heads, head_dim], kv_dtype, 16-byte
+ * aligned), row q_indptr[r]+j is rotated IN PLACE to the same position, so that the attention that
+ * follows sees rotated Q and K.  rope_base = 0: no rotation, q_rows ignored.  Needs head_dim/2 *
+ * element size to be a multiple of 16 bytes and head_dim <= 512 (SPX_ERR_UNSUPPORTED otherwise); a negative, NaN or
+ * infinite rope_base is SPX_ERR_INVALID_ARG.
+ *
  * spx_kv_rollback computes, AFTER sampling, the lengths that drop the rejected drafts:
  * new_seq_lens[r] = seq_lens[r] - (k_r - accepted_len[r]) (position 0 and the accepted drafts
  * stay; the emitted token is the next step's position 0 and is not cached yet).  An accepted
@@ -212,6 +223,9 @@ typedef struct {
   const int32_t *block_table;         /* [B, max_pages_per_req]                               */
   const int32_t *seq_lens;            /* [B], counts the new positions                        */
   const int32_t *q_indptr;            /* [B+1]                                                */
+  float rope_base;                    /* 0: plain copy; > 0: rotary base (e.g. 10000, 500000) */
+  int32_t num_q_heads;                /* heads of q_rows (ignored when q_rows is NULL)        */
+  void *q_rows;                       /* optional, rotated in place; NULL: none               */
 } spx_kv_append_args_t;
 
 spx_status_t spx_kv_append(const spx_kv_append_args_t *args, int32_t *dev_status, void *cuda_stream);

@@ -54,6 +54,7 @@ class KvAppendArgs(C.Structure):
         ("new_k", C.c_void_p), ("new_v", C.c_void_p), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
         ("kv_stride_page", C.c_int64), ("kv_stride_head", C.c_int64), ("kv_stride_token", C.c_int64),
         ("block_table", C.c_void_p), ("seq_lens", C.c_void_p), ("q_indptr", C.c_void_p),
+        ("rope_base", C.c_float), ("num_q_heads", C.c_int32), ("q_rows", C.c_void_p),
     ]
 
 
@@ -359,8 +360,9 @@ def rejection_sample_static(target_logits, draft_logits, draft_ids, q_indptr, u_
 
 
 def kv_append(new_k, new_v, k_cache, v_cache, kv_strides, block_table, seq_lens, q_indptr, page_size, num_pages,
-              status: Optional[torch.Tensor] = None):
-    """spx_kv_append on the current stream: the new positions' K/V go into their pages, in place."""
+              status: Optional[torch.Tensor] = None, rope_base: float = 0.0, q_rows: Optional[torch.Tensor] = None):
+    """spx_kv_append on the current stream: the new positions' K/V go into their pages, in place.
+    rope_base > 0: the K rows (and q_rows [TQ, Hq, D], in place) are rotated to their positions."""
     _require_cuda(new_k, new_v, k_cache, v_cache, block_table, seq_lens, q_indptr)
     lib = load_library()
     dev = new_k.device
@@ -374,6 +376,12 @@ def kv_append(new_k, new_v, k_cache, v_cache, kv_strides, block_table, seq_lens,
     a.new_k, a.new_v, a.k_cache, a.v_cache = _ptr(new_k), _ptr(new_v), _ptr(k_cache), _ptr(v_cache)
     a.kv_stride_page, a.kv_stride_head, a.kv_stride_token = (int(x) for x in kv_strides)
     a.block_table, a.seq_lens, a.q_indptr = _ptr(block_table), _ptr(seq_lens), q_indptr.data_ptr()
+    a.rope_base = float(rope_base)
+    if q_rows is not None:
+        _require_cuda(q_rows)
+        if q_rows.dtype != new_k.dtype or not q_rows.is_contiguous():
+            raise SpxError(ERR_INVALID_ARG, "q_rows must be contiguous and of the cache's dtype")
+        a.num_q_heads, a.q_rows = q_rows.shape[1], _ptr(q_rows)
     _check(lib.spx_kv_append(C.byref(a), status.data_ptr(), _stream(dev)))
     return status
 

@@ -651,10 +651,15 @@ spx_status_t spx_kv_append(const spx_kv_append_args_t *a, int32_t *dev_status, v
   const int es = a->kv_dtype == SPX_BF16 ? 2 : 4;
   if ((a->head_dim * es) % 16 != 0) return SPX_ERR_UNSUPPORTED;
   if (a->kv_stride_page < 0 || a->kv_stride_head < 0 || a->kv_stride_token < a->head_dim) return SPX_ERR_INVALID_ARG;
+  if (!(a->rope_base >= 0.f) || std::isinf(a->rope_base)) return SPX_ERR_INVALID_ARG;
+  const bool rope = a->rope_base > 0.f;
+  if (rope && ((a->head_dim & 1) || ((a->head_dim / 2) * es) % 16 != 0 || a->head_dim > kRopeMaxHeadDim)) return SPX_ERR_UNSUPPORTED;
+  if (rope && a->q_rows && a->num_q_heads <= 0) return SPX_ERR_INVALID_ARG;
   if (a->batch == 0) return SPX_OK;
   if (!a->new_k || !a->new_v || !a->k_cache || !a->v_cache || !a->block_table || !a->seq_lens || !a->q_indptr)
     return SPX_ERR_INVALID_ARG;
   if (((uintptr_t)a->new_k | (uintptr_t)a->new_v | (uintptr_t)a->k_cache | (uintptr_t)a->v_cache) & 15) return SPX_ERR_INVALID_ARG;
+  if (rope && ((uintptr_t)a->q_rows & 15)) return SPX_ERR_INVALID_ARG;
   if (((a->kv_stride_page * es) | (a->kv_stride_head * es) | (a->kv_stride_token * es)) & 15) return SPX_ERR_INVALID_ARG;
   KvAppendParams p{};
   p.batch = a->batch; p.total_q = a->total_q; p.Hkv = a->num_kv_heads; p.D = a->head_dim; p.P = a->page_size;
@@ -664,6 +669,9 @@ spx_status_t spx_kv_append(const spx_kv_append_args_t *a, int32_t *dev_status, v
   p.k_cache = static_cast<unsigned char *>(a->k_cache); p.v_cache = static_cast<unsigned char *>(a->v_cache);
   p.stride_page = a->kv_stride_page; p.stride_head = a->kv_stride_head; p.stride_token = a->kv_stride_token;
   p.block_table = a->block_table; p.seq_lens = a->seq_lens; p.q_indptr = a->q_indptr; p.dev_status = dev_status;
+  p.rope_base = rope ? (double)a->rope_base : 0.0;
+  p.q_rows = rope ? static_cast<unsigned char *>(a->q_rows) : nullptr;
+  p.Hq = a->num_q_heads;
   kv_append_kernel<<<a->batch, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p);
   ++t_launches;
   return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;

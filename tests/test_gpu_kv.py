@@ -95,3 +95,54 @@ def test_rollback_and_whole_sequence():
     new_len, status = spx.kv_rollback(b.seq_lens, b.q_indptr, bad_acc)
     torch.cuda.synchronize()
     assert int(status.item()) == spx.DEV_BAD_LEN and int(new_len[0]) == -1
+
+
+@pytest.mark.parametrize("layout", ["HND", "NHD"])
+@pytest.mark.parametrize("idx,base", [(0, 10000.0), (1, 500000.0), (3, 1000000.0), (4, 500000.0)])
+def test_append_with_rope_matches_oracle(idx, base, layout):
+    """K rows rotated to their absolute positions on the way into the cache, Q rows in place, V
+    copied.  Both sides compute in float64 and round float64 -> binary32 -> element type, so the
+    stored values agree bit for bit up to the last bit of the two libraries' sin / cos / pow: at
+    most one element in 10^4 may differ, and then by one unit in the last place."""
+    spec = W.CONFIGS[idx] if idx == 0 else W.scaled(W.CONFIGS[idx], batch=9, ctx_div=4 if idx == 3 else 16, vocab=64)
+    b_cpu = W.generate(spec, layout=layout)
+    nk, nv = _new_kv(b_cpu, 5)
+    b = b_cpu.to(DEV)
+    q_dev = b.q.clone()
+    status = spx.kv_append(nk.to(DEV), nv.to(DEV), b.k_cache, b.v_cache, b.kv_strides, b.block_table, b.seq_lens,
+                           b.q_indptr, spec.page_size, b.num_pages, rope_base=base, q_rows=q_dev)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    oracle.kv_append(nk, nv, b_cpu.k_cache, b_cpu.v_cache, b_cpu.kv_strides, b_cpu.block_table, b_cpu.seq_lens,
+                     b_cpu.q_indptr, spec.page_size, b_cpu.num_pages, rope_base=base)
+    assert torch.equal(b.v_cache.cpu(), b_cpu.v_cache)
+    pos = oracle.new_positions(b_cpu.seq_lens, b_cpu.q_indptr)
+    q_ref = oracle.round_to(oracle.rope(b_cpu.q, pos, base), b_cpu.q.dtype)
+
+    def close_to_the_last_bit(got, ref):
+        got, ref = got.cpu(), ref
+        if torch.equal(got, ref):
+            return
+        bits = torch.int16 if got.dtype == torch.bfloat16 else torch.int32
+        d = (got.view(bits).to(torch.int64) - ref.view(bits).to(torch.int64)).abs()
+        assert int(d.max()) <= 1 and float((d > 0).double().mean()) <= 1e-4, (int(d.max()), float((d > 0).double().mean()))
+
+    close_to_the_last_bit(b.k_cache, b_cpu.k_cache)
+    close_to_the_last_bit(q_dev, q_ref)
+    assert not torch.equal(q_dev.cpu(), b_cpu.q)               # the rows were rotated
+    # rope off: q_rows is left alone and the copy is the plain one
+    q2 = b.q.clone()
+    spx.kv_append(nk.to(DEV), nv.to(DEV), b.k_cache, b.v_cache, b.kv_strides, b.block_table, b.seq_lens, b.q_indptr,
+                  spec.page_size, b.num_pages, rope_base=0.0, q_rows=q2)
+    torch.cuda.synchronize()
+    assert torch.equal(q2, b.q)
+
+
+def test_rope_arguments_are_validated():
+    spec = W.CONFIGS[0]
+    b = W.generate(spec).to(DEV)
+    nk, nv = _new_kv(b, 1, DEV)
+    for bad in (-1.0, float("nan"), float("inf")):
+        with pytest.raises(spx.SpxError):
+            spx.kv_append(nk, nv, b.k_cache, b.v_cache, b.kv_strides, b.block_table, b.seq_lens, b.q_indptr,
+                          spec.page_size, b.num_pages, rope_base=bad)
