@@ -3,7 +3,8 @@
 // This is the kernel for kv_dtype = F32: tensor-core tf32 would round the operands to 10-bit
 // mantissas, which does not meet a 1e-4 absolute tolerance, so the fp32 configuration keeps true
 // fp32 products.  It executes the same work plan (chunks of 128-token tiles, partials merged by
-// combine_kernel) as the bf16 tensor-core kernel and also accepts bf16 inputs, which the tests
+// combine_kernel; its blocks take the entries through a shared counter rather than by range) as
+// the bf16 tensor-core kernel and also accepts bf16 inputs, which the tests
 // use to cross-check the two kernels.
 #pragma once
 #include "common.cuh"

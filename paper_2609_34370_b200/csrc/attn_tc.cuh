@@ -10,7 +10,8 @@
 //               grows by more than 2^8), P written back over the score buffer as bf16, epilogue.
 // The G*(k+1) query rows that share a kv-head are packed into the M dimension of one tile, so each
 // K/V byte is fetched once for all of them.  Work items come from the plan (chunks of 128-token
-// tiles); split requests write fp32 partials that combine_kernel merges.
+// tiles of one (request, kv head) pair; CTA c walks its own range of the list); the chunks of a
+// split pair write fp32 partials that combine_kernel merges.
 //
 // Every wait is bounded: on expiry the CTA raises SPX_DEV_TIMEOUT, all roles leave their loops,
 // pending copies get time to land and TMEM is released.

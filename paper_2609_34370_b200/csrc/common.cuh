@@ -11,10 +11,6 @@ namespace spx {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTileTokens = 128;   // KV tokens per attention tile (both attention kernels plan in this unit)
-#ifndef SPX_PLAN_WAVES
-#define SPX_PLAN_WAVES 8
-#endif
-constexpr int kPlanWaves = SPX_PLAN_WAVES;  // target number of work chunks per SM
 
 __device__ __forceinline__ float ld_as_float(const float *p, int64_t i) { return p[i]; }
 __device__ __forceinline__ float ld_as_float(const __nv_bfloat16 *p, int64_t i) { return __bfloat162float(p[i]); }
