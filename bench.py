@@ -295,6 +295,80 @@ def time_extras(spx, binding, spec, b, attn_args, dev, iters: int = 200):
     return out
 
 
+def run_timeline(args):
+    """Where the time of one step goes: every kernel of a timeline build of the library
+    (-DSPX_TIMELINE=1: per-CTA %globaltimer stamps, about 1.5 us per step) reports when its CTAs
+    started and ended.  Steps are launched back to back in windows; the last step of each window is
+    read out, and the median over the windows is printed (us from the first CTA of the step)."""
+    import numpy as np
+    import paper_2609_34370_b200 as spx
+    from paper_2609_34370_b200 import binding, build
+    binding.LIB_PATH = build.build_timeline()
+    spec = W.CONFIGS[args.workload]
+    if args.batch:
+        spec = W.scaled(spec, batch=args.batch)
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    b = W.generate(spec, device=dev)
+    out = torch.empty_like(b.q)
+    lse = torch.empty(b.q.shape[:2], dtype=torch.float32, device=dev)
+    acc = torch.empty(b.batch, dtype=torch.int32, device=dev)
+    tok = torch.empty(b.total_q, dtype=torch.int32, device=dev)
+    a = binding.make_attn_args(b.q, b.k_cache, b.v_cache, b.kv_strides, b.block_table, b.seq_lens, b.q_indptr,
+                               spec.num_kv_heads, spec.page_size, b.num_pages, out, lse, max_q_len=max(b.k_host) + 1)
+    s = binding.make_sample_args(b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample, acc, tok)
+    ws = spx.Workspace.allocate(spx.workspace_size(a, s), dev)
+    for _ in range(max(args.warmup, 3)):
+        spx.verify_step(a, s, ws, dev)
+    torch.cuda.synchronize()
+    names = ["plan", "attention", "combine", "logits statistics", "accept", "residual masses", "residual draw"]
+    windows, per_window = 12, max(50, min(args.steps, 500))
+    rows = {n: [] for n in names}
+    step_us = []
+    for _ in range(windows):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(per_window):
+            spx.verify_step(a, s, ws, dev)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / per_window
+        step_us.append(us)
+        tl = spx.debug_timeline().astype(np.int64)
+        horizon = tl[:, :, 1].max() - int(us * 1e3) - 3000          # CTAs of the last step only
+        spans = {}
+        for k, n in enumerate(names):
+            st, en = tl[k, :, 0], tl[k, :, 1]
+            sel = (en > horizon) & (st > horizon - 200000) & (en >= st)
+            spans[n] = (st[sel], en[sel])
+        starts = [v[0].min() for v in spans.values() if len(v[0])]
+        if not starts:
+            continue
+        t0 = min(starts)
+        for n in names:
+            st, en = spans[n]
+            if len(st) == 0:
+                continue
+            st, en = (st - t0) / 1e3, (en - t0) / 1e3
+            rows[n].append((len(st), st.min(), np.median(st), st.max(), en.min(), np.median(en), en.max(), np.median(en - st)))
+        time.sleep(0.2)
+    table = {}
+    for n in names:
+        if rows[n]:
+            m = np.median(np.array(rows[n]), axis=0)
+            table[n] = {"ctas": int(m[0]), "first_start_us": round(m[1], 1), "median_start_us": round(m[2], 1),
+                        "last_start_us": round(m[3], 1), "first_end_us": round(m[4], 1), "median_end_us": round(m[5], 1),
+                        "last_end_us": round(m[6], 1), "median_cta_us": round(m[7], 1)}
+    print(json.dumps({"timeline": table, "workload": spec.name, "us_per_step_instrumented": round(float(np.median(step_us)), 2),
+                      "windows": windows, "steps_per_window": per_window}))
+    print("%-18s %6s %31s %31s %10s" % ("kernel", "CTAs", "starts (first / median / last)", "ends (first / median / last)", "CTA us"),
+          file=sys.stderr)
+    for n, t in table.items():
+        print("%-18s %6d %9.1f %9.1f %9.1f   %9.1f %9.1f %9.1f %10.1f" % (
+            n, t["ctas"], t["first_start_us"], t["median_start_us"], t["last_start_us"], t["first_end_us"],
+            t["median_end_us"], t["last_end_us"], t["median_cta_us"]), file=sys.stderr)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -309,6 +383,8 @@ def main():
                     help="also time the pieces around the step: KV append / rollback, verification variants")
     ap.add_argument("--extras-iters", type=int, default=200, help="timed calls per extras entry (profiling runs: a few)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling captures of a smaller case)")
+    ap.add_argument("--timeline", action="store_true",
+                    help="per-kernel timeline of the step from a timeline build of the library (prints it and exits)")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 2000:
@@ -318,6 +394,9 @@ def main():
 
     import paper_2609_34370_b200 as spx
     from paper_2609_34370_b200 import binding
+    if args.timeline:
+        run_timeline(args)
+        return
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

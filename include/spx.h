@@ -402,6 +402,17 @@ int32_t spx_last_launch_count(void);
  */
 spx_status_t spx_plan_layout(const spx_attn_args_t *attn, int64_t *out);
 
+/*
+ * Measurement aid of timeline builds of the library (compiled with -DSPX_TIMELINE=1; the regular
+ * build returns SPX_ERR_UNSUPPORTED): every kernel of the step stamps the GPU's global
+ * nanosecond timer per CTA at entry and exit.  Copies the stamps of the most recent launches to
+ * host_out (host memory, uint64 [kernels][ctas_per_kernel][4] = {start ns, end ns, SM id, 0};
+ * kernel index: 0 plan, 1 attention, 2 combine, 3 logits statistics, 4 accept, 5 residual masses,
+ * 6 residual draw).  capacity is in uint64 elements; the two dimensions are always written to
+ * *kernels / *ctas_per_kernel (either may be NULL).  Synchronises the device.
+ */
+spx_status_t spx_debug_timeline(uint64_t *host_out, int64_t capacity, int32_t *kernels, int32_t *ctas_per_kernel);
+
 #ifdef __cplusplus
 }
 #endif

@@ -16,7 +16,7 @@ BF16, F32 = 0, 1
 
 EXPORTS = ("spx_workspace_size", "spx_verify_attention", "spx_rejection_sample", "spx_verify_step",
            "spx_host_step_arena_size", "spx_verify_step_host", "spx_status_string", "spx_last_launch_count",
-           "spx_set_timing_events", "spx_plan_layout", "spx_rejection_sample_static", "spx_kv_append", "spx_kv_rollback",
+           "spx_set_timing_events", "spx_plan_layout", "spx_debug_timeline", "spx_rejection_sample_static", "spx_kv_append", "spx_kv_rollback",
            "spx_draft_confidence_workspace", "spx_draft_confidence", "spx_select_speculation",
            "spx_lookahead_memory", "spx_sp_effective_batch", "spx_selective_batch", "spx_selective_effective_batch",
            "spx_delay_gain", "spx_lm_head")
@@ -114,6 +114,8 @@ def load_library():
         lib.spx_status_string.argtypes = [C.c_int]
         lib.spx_last_launch_count.restype = C.c_int32
         lib.spx_plan_layout.restype = C.c_int
+        lib.spx_debug_timeline.restype = C.c_int
+        lib.spx_debug_timeline.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         lib.spx_plan_layout.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
         lib.spx_rejection_sample_static.restype = C.c_int
         lib.spx_rejection_sample_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
@@ -314,6 +316,18 @@ def plan_layout(attn_args) -> dict:
     _check(load_library().spx_plan_layout(C.byref(attn_args), out))
     keys = ("header", "cta_off", "work", "max_work", "pair_nchunks", "pair_part_base", "max_part_slots", "attn_bytes")
     return dict(zip(keys, (int(v) for v in out)))
+
+
+def debug_timeline():
+    """spx_debug_timeline: numpy uint64 [kernels, ctas, 4] = (start ns, end ns, SM id, 0) of the most
+    recent launches.  Only a timeline build of the library records them (SpxError otherwise)."""
+    import numpy as np
+    lib = load_library()
+    nk, nc = C.c_int32(0), C.c_int32(0)
+    lib.spx_debug_timeline(None, 0, C.byref(nk), C.byref(nc))
+    out = np.zeros((nk.value, nc.value, 4), dtype=np.uint64)
+    _check(lib.spx_debug_timeline(out.ctypes.data, out.size, C.byref(nk), C.byref(nc)))
+    return out
 
 
 def last_launch_count() -> int:

@@ -7,6 +7,7 @@ import subprocess
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 LIB_PATH = os.path.join(_PKG, "libspx.so")
+TIMELINE_LIB_PATH = os.path.join(_PKG, "libspx_timeline.so")
 _SOURCES = [os.path.join(_PKG, "csrc", "spx_api.cu")]
 
 
@@ -18,18 +19,31 @@ def _newest_source_mtime() -> float:
     return newest
 
 
+def _compile(out_path: str, defines=(), verbose: bool = False) -> str:
+    cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+           "--shared", "-Xcompiler", "-fPIC", "-cudart", "static",
+           "-I", os.path.join(_ROOT, "include"), "-I", os.path.join(_PKG, "csrc")]
+    cmd += ["-D" + d for d in defines]
+    cmd += ["-o", out_path] + _SOURCES
+    if verbose:
+        cmd.insert(1, "-Xptxas=-v")
+    subprocess.run(cmd, check=True)
+    return out_path
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile every CUDA source into paper_2609_34370_b200/libspx.so; returns its path."""
     if not force and os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= _newest_source_mtime():
         return LIB_PATH
-    cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "--shared", "-Xcompiler", "-fPIC", "-cudart", "static",
-           "-I", os.path.join(_ROOT, "include"), "-I", os.path.join(_PKG, "csrc"),
-           "-o", LIB_PATH] + _SOURCES
-    if verbose:
-        cmd.insert(1, "-Xptxas=-v")
-    subprocess.run(cmd, check=True)
-    return LIB_PATH
+    return _compile(LIB_PATH, verbose=verbose)
+
+
+def build_timeline(force: bool = False) -> str:
+    """The same sources with per-CTA timestamps compiled in (libspx_timeline.so; see
+    spx_debug_timeline).  Used by `bench.py --timeline` only."""
+    if not force and os.path.exists(TIMELINE_LIB_PATH) and os.path.getmtime(TIMELINE_LIB_PATH) >= _newest_source_mtime():
+        return TIMELINE_LIB_PATH
+    return _compile(TIMELINE_LIB_PATH, defines=("SPX_TIMELINE=1",))
 
 
 if __name__ == "__main__":

@@ -34,6 +34,7 @@ struct SimtSmem {
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads) attn_simt_kernel(AttnParams p) {
+  SPX_TL_SCOPE(kTlAttention);
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ int s_item;
   const SimtSmem lay(p.rows_cap, D);

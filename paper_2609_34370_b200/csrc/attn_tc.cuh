@@ -157,6 +157,7 @@ struct ItemInfo {
 template <int D, int QROWS>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, AttnParams p) {
+  SPX_TL_SCOPE(kTlAttention);
   using Cfg = TcCfg<D, QROWS>;
   using namespace tc;
   extern __shared__ unsigned char smem_dyn[];

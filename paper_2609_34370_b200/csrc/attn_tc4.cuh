@@ -92,6 +92,7 @@ __host__ __device__ constexpr uint32_t idesc_ws(uint32_t m, uint32_t n, bool b_m
 template <int D, int MROWS>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, AttnParams p) {
+  SPX_TL_SCOPE(kTlAttention);
   using Cfg = Tc4Cfg<D, MROWS>;
   using namespace tc;
   constexpr int kSplit = Cfg::kSplit, TPT = Cfg::kTokPerThread;

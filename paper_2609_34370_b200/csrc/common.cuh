@@ -12,6 +12,48 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTileTokens = 128;   // KV tokens per attention tile (both attention kernels plan in this unit)
 
+// ------------------------------------------------------------------------------------------
+// Timeline builds (-DSPX_TIMELINE=1; see build.py and `bench.py --timeline`): every kernel of the
+// step stamps %globaltimer per CTA at entry and exit into a device array that
+// spx_debug_timeline copies out: slot [kernel][cta] = {start ns, end ns, SM id, 0}.  The end is
+// the latest exit of the CTA's warps.  Costs about 1.5 us per step; compiled out otherwise.
+// ------------------------------------------------------------------------------------------
+#ifndef SPX_TIMELINE
+#define SPX_TIMELINE 0
+#endif
+constexpr int kTlKernels = 8;        // plan, attention, combine, logits statistics, accept, residual masses, draw, spare
+constexpr int kTlCtas = 4096;        // CTAs recorded per kernel
+#if SPX_TIMELINE
+__device__ unsigned long long g_timeline[kTlKernels * kTlCtas * 4];
+struct TlScope {
+  unsigned long long *slot;
+  __device__ __forceinline__ static unsigned long long now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+  }
+  __device__ __forceinline__ explicit TlScope(int kernel_id) : slot(nullptr) {
+    const int cta = blockIdx.x + blockIdx.y * gridDim.x;
+    if (cta < kTlCtas) {
+      slot = g_timeline + ((size_t)kernel_id * kTlCtas + cta) * 4;
+      if (threadIdx.x == 0) {
+        unsigned sm;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+        slot[0] = now();
+        slot[2] = sm;
+      }
+    }
+  }
+  __device__ __forceinline__ ~TlScope() {
+    if (slot && (threadIdx.x & 31) == 0) atomicMax(slot + 1, now());
+  }
+};
+#define SPX_TL_SCOPE(id) TlScope spx_tl_scope_(id)
+#else
+#define SPX_TL_SCOPE(id) do { } while (0)
+#endif
+enum { kTlPlan = 0, kTlAttention = 1, kTlCombine = 2, kTlLogitStats = 3, kTlAccept = 4, kTlResidMass = 5, kTlResidPick = 6 };
+
 __device__ __forceinline__ float ld_as_float(const float *p, int64_t i) { return p[i]; }
 __device__ __forceinline__ float ld_as_float(const __nv_bfloat16 *p, int64_t i) { return __bfloat162float(p[i]); }
 

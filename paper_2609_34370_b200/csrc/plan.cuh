@@ -44,6 +44,7 @@ __device__ __forceinline__ int plan_entry_cost(int tiles) { return tiles <= 2 ? 
 // requests' (request, kv head) pairs into n_cta ranges of equal length, lays out partial-result
 // slots for the pairs a cut crosses and emits each range's work entries in axis order.
 __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int n_cta) {
+  SPX_TL_SCOPE(kTlPlan);
   __shared__ int s_scratch[32];
   __shared__ int s_total;
   __shared__ int s_cut[kPlanMaxCta + 1];     // cut c: first tile (axis position) of range c
@@ -231,6 +232,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int n_cta) {
 // (row, 4 columns), chunks walked four at a time so that their loads are in flight together.
 template <typename T>
 __global__ void __launch_bounds__(256) combine_kernel(AttnParams p) {
+  SPX_TL_SCOPE(kTlCombine);
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the attention kernel's partials (no-op without PDL)
   const int r = blockIdx.x / p.Hkv, g = blockIdx.x % p.Hkv;
   const int nch = p.pair_nchunks[blockIdx.x];

@@ -211,6 +211,7 @@ __device__ __forceinline__ void slice_stats(const SubSlice<float> &sl, float &m,
 // bookkeeping cost more than the 22 % of bytes it saved.)
 template <typename T, bool kScaled>
 __global__ void __launch_bounds__(kSampThreads) row_stats_kernel(SampleParams p, int n_units) {
+  SPX_TL_SCOPE(kTlLogitStats);
   const int lane = threadIdx.x & 31;
   const int warp_global = (blockIdx.x * kSampThreads + threadIdx.x) >> 5;
   const int n_warps = (gridDim.x * kSampThreads) >> 5;
@@ -289,6 +290,7 @@ __device__ __forceinline__ bool ring_wait(uint64_t *bar, uint32_t parity, volati
 
 template <bool kScaled>
 __global__ void __launch_bounds__(kRingThreads, 1) row_stats_ring_kernel(SampleParams p, int chunks_per_row, int n_chunks) {
+  SPX_TL_SCOPE(kTlLogitStats);
   extern __shared__ __align__(1024) unsigned char ring_smem[];
   unsigned char *stages = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(ring_smem) + 1023) & ~uintptr_t(1023));
   uint64_t *full = reinterpret_cast<uint64_t *>(stages + kRingStages * kRingStageElems * 2);
@@ -893,6 +895,7 @@ __device__ __forceinline__ void greedy_request(const SampleParams &p, int r) {
 // accepted_len, the accepted ids and the -1 padding; slot n is left for resid_pick_kernel.
 template <typename T, bool kScaled, bool kFiltered>
 __global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_blocks) {
+  SPX_TL_SCOPE(kTlAccept);
   if (kScaled && (int)blockIdx.x >= accept_blocks) {  // variants: one extra block per request for the greedy ones
     greedy_request<T>(p, blockIdx.x - accept_blocks);
     return;
@@ -1073,6 +1076,7 @@ struct ResidCtx {
 constexpr int kResidStageBytes = 2 * kSegElems * 2;  // bf16 logits: the block's segment of both rows
 template <typename T, bool kScaled, bool kFiltered>
 __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 6 : 1) resid_mass_kernel(SampleParams p) {
+  SPX_TL_SCOPE(kTlResidMass);
   const int seg_mine = blockIdx.x, r = blockIdx.y;
   ResidCtx<T, kScaled, kFiltered> c;
   if (!c.init(p, r) || !c.full_pass()) return;
@@ -1157,6 +1161,7 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 6 : 1) resid_m
 // wait, the masses of resid_mass_kernel after it.
 template <typename T, bool kScaled, bool kFiltered>
 __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_pick_kernel(SampleParams p) {
+  SPX_TL_SCOPE(kTlResidPick);
   const int r = blockIdx.x;
   ResidCtx<T, kScaled, kFiltered> c;
   const bool live = c.init(p, r);

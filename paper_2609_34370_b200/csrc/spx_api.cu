@@ -886,6 +886,19 @@ void spx_set_timing_events(void *start_event, void *stop_event) {
 
 int32_t spx_last_launch_count(void) { return t_launches; }
 
+spx_status_t spx_debug_timeline(uint64_t *host_out, int64_t capacity, int32_t *kernels, int32_t *ctas_per_kernel) {
+  if (kernels) *kernels = kTlKernels;
+  if (ctas_per_kernel) *ctas_per_kernel = kTlCtas;
+#if SPX_TIMELINE
+  const int64_t need = (int64_t)kTlKernels * kTlCtas * 4;
+  if (!host_out || capacity < need) return SPX_ERR_INVALID_ARG;
+  return cudaMemcpyFromSymbol(host_out, g_timeline, (size_t)need * sizeof(uint64_t)) == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
+#else
+  (void)host_out; (void)capacity;
+  return SPX_ERR_UNSUPPORTED;
+#endif
+}
+
 spx_status_t spx_plan_layout(const spx_attn_args_t *attn, int64_t *out) {
   if (!out) return SPX_ERR_INVALID_ARG;
   const spx_status_t st = check_attn(attn, false);

@@ -145,3 +145,12 @@ def test_calls_around_the_step_refuse_bad_arguments_before_any_launch(lib):
     la.logits_row_stride = 96
     assert lib.spx_lm_head(C.byref(la), C.byref(status), None) == binding.ERR_INVALID_ARG        # stride below the vocabulary
     assert status.value == 0
+
+
+def test_timeline_is_a_build_option():
+    """The regular build records no per-CTA stamps: the call reports its dimensions and refuses."""
+    import ctypes as C
+    lib = spx.load_library()
+    nk, nc = C.c_int32(0), C.c_int32(0)
+    st = lib.spx_debug_timeline(None, 0, C.byref(nk), C.byref(nc))
+    assert st == binding.ERR_UNSUPPORTED and nk.value >= 7 and nc.value >= 148
