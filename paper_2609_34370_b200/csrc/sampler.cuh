@@ -429,10 +429,10 @@ constexpr int kFilterSmemBytes = 4 * 256 * 32 * 4 + 256 * (8 + 4) * 2 + kFilterL
 
 // Calls f(x) for every element of a row; the block's threads stride over 16-byte vectors and keep
 // kFilterUnroll of them in flight.
-template <typename T, typename F>
+template <typename T, int kThreads = kFilterThreads, typename F>
 __device__ __forceinline__ void sweep_row(const T *base, int vocab, int tid, F f) {
   constexpr int N = Vec<T>::N;
-  constexpr int stride = kFilterThreads * N;
+  constexpr int stride = kThreads * N;
   int v = tid * N;
   for (; v + (kFilterUnroll - 1) * stride + N <= vocab; v += kFilterUnroll * stride) {
     uint4 raw[kFilterUnroll];
@@ -458,6 +458,118 @@ __device__ __forceinline__ void sweep_row(const T *base, int vocab, int tid, F f
   }
 }
 
+// top-k (optionally with top-p on top) of one row per block for K no larger than the number of
+// sub-segments of the row: the K-th largest of the sub-segment maxima (left by the statistics
+// pass) is a lower bound of the K-th largest logit, so one compare-only sweep collects every
+// candidate (a few hundred logits for K = 50 on a 128k vocabulary) and the candidates are ranked
+// by counting - thread i sums count and mass of the keys above and at-or-above its own; no
+// histogram, no atomics on the masses.  256 threads and 16 KB of shared memory per row, so all the
+// rows of a batch are resident at once and the kernel runs at the rate the logits arrive.
+// Rows it cannot take (K larger than that, top-p alone, more than kTopkListCap candidates) are
+// left marked pending (row_z = NaN, set by row_scale_kernel) for filter_rows_kernel.
+constexpr int kTopkThreads = 256;
+constexpr int kTopkListCap = 1024;
+template <typename T>
+__global__ void __launch_bounds__(kTopkThreads, 6) topk_list_kernel(SampleParams p) {
+  __shared__ float s_list[kTopkListCap];
+  __shared__ uint32_t s_key[kTopkListCap];
+  __shared__ unsigned long long s_m[kTopkListCap];
+  __shared__ uint32_t s_n, s_Tk, s_Tf;
+  __shared__ unsigned long long s_Zk, s_Zf;
+  __shared__ int s_found;
+  __shared__ float s_bound;
+  const int row = blockIdx.x, tid = threadIdx.x;
+  const int r = p.row_req[row];
+  if (r < 0) {
+    if (tid == 0) { p.row_thresh[row] = 0; p.row_z[row] = -1.0; }
+    return;
+  }
+  const int tk_raw = p.top_k ? p.top_k[r] : 0;
+  const bool use_k = tk_raw >= 1 && tk_raw < p.vocab;
+  const float tp = p.top_p ? p.top_p[r] : 1.f;
+  const bool use_p = tp < 1.f;
+  if (!use_k || tk_raw > p.nsub || p.nsub > kTopkThreads) return;
+  const float scale = p.row_scale[row];
+  const T *base = row < p.total_q ? reinterpret_cast<const T *>(p.target) + (int64_t)row * p.row_stride
+                                  : reinterpret_cast<const T *>(p.draft) + (int64_t)(row - p.total_q) * p.row_stride;
+  const float2 *st = p.seg_stats + (int64_t)row * p.nsub;
+  float M = -INFINITY;
+  for (int j = 0; j < p.nsub; ++j) M = fmaxf(M, st[j].x);
+  auto mass_of = [&](float x) -> unsigned long long { return __float2ull_rn(fast_exp2(fmaf(x, scale, -M)) * kMassScale); };
+  if (tid < p.nsub) {
+    const float mine = st[tid].x;
+    int rank = 0;
+    for (int j = 0; j < p.nsub; ++j) {
+      const float o = st[j].x;
+      rank += (o > mine || (o == mine && j < tid)) ? 1 : 0;
+    }
+    if (rank == tk_raw - 1) s_bound = mine;
+  }
+  if (tid == 0) { s_n = 0; s_found = 0; }
+  __syncthreads();
+  const float bound = s_bound - (fabsf(s_bound) * 1e-6f + 1e-6f);  // in the scaled (log2) domain, like the statistics
+  sweep_row<T, kTopkThreads>(base, p.vocab, tid, [&](float x) {
+    if (x * scale >= bound) {
+      const uint32_t i = atomicAdd(&s_n, 1u);
+      if (i < (uint32_t)kTopkListCap) s_list[i] = x;
+    }
+  });
+  __syncthreads();
+  const uint32_t n = s_n;
+  if (n > (uint32_t)kTopkListCap) return;   // too many equal logits at the cut: the general kernel takes the row
+  for (uint32_t i = tid; i < n; i += kTopkThreads) { s_key[i] = order_key32(s_list[i]); s_m[i] = mass_of(s_list[i]); }
+  __syncthreads();
+  // the highest key T with count(key >= T) >= K; then, with top-p, the highest key with
+  // mass(key >= T) >= P * kept mass (never below the top-k cut)
+  constexpr int kPer = kTopkListCap / kTopkThreads;
+  uint32_t key[kPer], cnt_ge[kPer];
+  unsigned long long m_gt[kPer], m_ge[kPer];
+#pragma unroll
+  for (int q = 0; q < kPer; ++q) {
+    const uint32_t i = tid + q * kTopkThreads;
+    key[q] = 0; cnt_ge[q] = 0; m_gt[q] = 0ull; m_ge[q] = 0ull;
+    if (i < n) {
+      const uint32_t ki = s_key[i];
+      uint32_t c_gt = 0, c_ge = 0;
+      unsigned long long a_gt = 0ull, a_ge = 0ull;
+      for (uint32_t j = 0; j < n; ++j) {
+        const uint32_t kj = s_key[j];
+        const unsigned long long mj = s_m[j];
+        if (kj > ki) { ++c_gt; a_gt += mj; }
+        if (kj >= ki) { ++c_ge; a_ge += mj; }
+      }
+      key[q] = ki; cnt_ge[q] = c_ge; m_gt[q] = a_gt; m_ge[q] = a_ge;
+      if (c_gt < (uint32_t)tk_raw && c_ge >= (uint32_t)tk_raw) { s_Tk = ki; s_Zk = a_ge; }  // equal keys write equal values
+    }
+  }
+  __syncthreads();
+  const uint32_t Tk = s_Tk;
+  const unsigned long long Zk = s_Zk;
+  uint32_t Tf = Tk;
+  unsigned long long Zf = Zk;
+  if (use_p) {
+    const double need_mass = (double)tp * (double)Zk;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q)
+      if (tid + q * kTopkThreads < (int)n && (double)m_gt[q] < need_mass && (double)m_ge[q] >= need_mass) {
+        s_Tf = key[q]; s_Zf = m_ge[q]; s_found = 1;
+      }
+    __syncthreads();
+    if (!s_found) {  // rounding left the criterion unmet even at the lowest key: take it
+#pragma unroll
+      for (int q = 0; q < kPer; ++q)
+        if (tid + q * kTopkThreads < (int)n && cnt_ge[q] == n) { s_Tf = key[q]; s_Zf = m_ge[q]; }
+      __syncthreads();
+    }
+    Tf = s_Tf; Zf = s_Zf;
+    if (Tf < Tk) { Tf = Tk; Zf = Zk; }
+  }
+  if (tid == 0) {
+    p.row_thresh[row] = Tf;
+    p.row_z[row] = (double)Zf / (double)kMassScale;
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SampleParams p) {
   extern __shared__ __align__(16) unsigned char fsm[];
@@ -474,6 +586,10 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
   __shared__ unsigned long long s_above_mass, s_bin_mass;
   const int row = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  {
+    const double z_in = p.row_z[row];
+    if (z_in == z_in) return;   // not pending (NaN): topk_list_kernel has settled this row
+  }
   const int r = p.row_req[row];
   if (r < 0) {
     if (tid == 0) { p.row_thresh[row] = 0; p.row_z[row] = -1.0; }
@@ -808,8 +924,9 @@ __global__ void row_scale_kernel(SampleParams p) {
   for (int i = 0; i < k; ++i) p.row_scale[p.total_q + t0 - r + i] = sd;
   if (p.row_req) {
     const bool filtered = valid && tau > 0.f && ((tk >= 1 && tk < p.vocab) || tp < 1.f);
-    for (int i = 0; i <= k; ++i) p.row_req[t0 + i] = filtered ? r : -1;
-    for (int i = 0; i < k; ++i) p.row_req[p.total_q + t0 - r + i] = filtered ? r : -1;
+    const double pending = __longlong_as_double(0x7ff8000000000000ll);  // NaN: no threshold yet
+    for (int i = 0; i <= k; ++i) { p.row_req[t0 + i] = filtered ? r : -1; p.row_z[t0 + i] = pending; }
+    for (int i = 0; i < k; ++i) { p.row_req[p.total_q + t0 - r + i] = filtered ? r : -1; p.row_z[p.total_q + t0 - r + i] = pending; }
   }
 }
 

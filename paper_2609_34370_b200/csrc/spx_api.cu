@@ -411,8 +411,9 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
     if constexpr (kFiltered) {
       if (cudaFuncSetAttribute(filter_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFilterSmemBytes) != cudaSuccess)
         return SPX_ERR_CUDA;
+      topk_list_kernel<T><<<rows, kTopkThreads, 0, stream>>>(p);
       filter_rows_kernel<T><<<rows, kFilterThreads, kFilterSmemBytes, stream>>>(p);
-      ++t_launches;
+      t_launches += 2;
     }
     const int accept_blocks = (p.batch * 32 + 127) / 128;
     accept_kernel<T, kScaled, kFiltered><<<accept_blocks + (kScaled ? p.batch : 0), 128, 0, stream>>>(p, accept_blocks);
