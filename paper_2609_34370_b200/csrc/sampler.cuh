@@ -689,11 +689,11 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
     return prefix;
   };
 
-  // top-k with K no larger than the number of sub-segments of the row: the K-th largest of the
-  // sub-segment maxima (known from the statistics pass) is a lower bound of the K-th largest
-  // logit, so one compare-only sweep collects every candidate (a few hundred logits for K = 50
-  // on a 128k vocabulary) and the exact levels run over that list - no histogram of the whole row.
-  // A list that overflows (many equal logits) falls back to the general path below.
+  // top-k with K no larger than the number of sub-segments of the row, for the rows that
+  // topk_list_kernel left (more candidates than its list holds, or more sub-segments than it has
+  // threads): the same lower bound and compare-only sweep into the larger list here, then the
+  // exact key-byte levels over that list.  A list that overflows even here (many equal logits)
+  // falls back to the histogram path below.
   if (use_k && tk_raw <= p.nsub && p.nsub <= kFilterThreads) {
     __shared__ float s_bound;
     const float2 *st = p.seg_stats + (int64_t)row * p.nsub;
@@ -717,54 +717,6 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
     });
     __syncthreads();
     const uint32_t n_list = s_list_n;
-    if (n_list <= (uint32_t)kFilterThreads) {
-      // A list of at most one candidate per thread is ranked by counting, without atomics (the
-      // candidates of a row share the top key byte, and 64-bit shared-memory atomics on one
-      // address cost about 100 cycles each): thread i sums count and mass of the keys above and
-      // at-or-above its own.  The threshold is the highest key T with count(key >= T) >= K, then
-      // (top-p on top) the highest key with mass(key >= T) >= P * kept mass: what the levels find.
-      uint32_t *k_arr = h_cnt;                                                    // the histogram arrays are free here
-      unsigned long long *m_arr = reinterpret_cast<unsigned long long *>(h_cnt + kFilterThreads);
-      __shared__ uint32_t s_Tk, s_Tf;
-      __shared__ unsigned long long s_Zk, s_Zf;
-      __shared__ int s_found;
-      if (tid < (int)n_list) { k_arr[tid] = order_key32(s_list[tid]); m_arr[tid] = mass_of(s_list[tid]); }
-      if (tid == 0) s_found = 0;
-      __syncthreads();
-      uint32_t key = 0, cnt_gt = 0, cnt_ge = 0;
-      unsigned long long m_gt = 0ull, m_ge = 0ull;
-      if (tid < (int)n_list) {
-        key = k_arr[tid];
-        for (uint32_t j = 0; j < n_list; ++j) {
-          const uint32_t kj = k_arr[j];
-          const unsigned long long mj = m_arr[j];
-          if (kj > key) { ++cnt_gt; m_gt += mj; }
-          if (kj >= key) { ++cnt_ge; m_ge += mj; }
-        }
-        if (cnt_gt < (uint32_t)tk_raw && cnt_ge >= (uint32_t)tk_raw) { s_Tk = key; s_Zk = m_ge; }  // equal keys write equal values
-      }
-      __syncthreads();
-      const uint32_t Tk = s_Tk;
-      const unsigned long long Zk = s_Zk;
-      uint32_t Tf = Tk;
-      unsigned long long Zf = Zk;
-      if (use_p) {
-        const double need_mass = (double)tp * (double)Zk;
-        if (tid < (int)n_list && (double)m_gt < need_mass && (double)m_ge >= need_mass) { s_Tf = key; s_Zf = m_ge; s_found = 1; }
-        __syncthreads();
-        if (!s_found) {  // rounding left the criterion unmet even at the lowest key: take it
-          if (tid < (int)n_list && cnt_ge == n_list) { s_Tf = key; s_Zf = m_ge; }
-          __syncthreads();
-        }
-        Tf = s_Tf; Zf = s_Zf;
-        if (Tf < Tk) { Tf = Tk; Zf = Zk; }
-      }
-      if (tid == 0) {
-        p.row_thresh[row] = Tf;
-        p.row_z[row] = (double)Zf / (double)kMassScale;
-      }
-      return;
-    }
     if (n_list <= (uint32_t)kFilterListCap) {
       unsigned long long Zk = 0ull, Zf = 0ull;
       const uint32_t Tk = levels_over_list(true, (uint32_t)tk_raw, 0.0, n_list, &Zk);

@@ -205,6 +205,46 @@ def test_crowded_threshold_bin():
     assert not rep.hard_mismatch, (rep, acc.cpu().tolist(), ref.accepted_len.tolist(), ref.margin.tolist())
 
 
+@pytest.mark.parametrize("tie", [300, 4000, 20000])
+def test_small_top_k_with_a_block_of_equal_logits_at_the_cut(tie):
+    """A small K takes the candidate-list path: every logit at or above a lower bound of the K-th
+    largest is collected and ranked.  A block of equal logits at the cut makes the list a few
+    hundred entries (ranked by counting), a few thousand (exact key-byte levels over the list in the
+    general kernel) or too long for any list (histogram path): same thresholds in all three."""
+    V, B, k = 60000, 4, 1                    # 30 sub-segments of 2048 tokens: K <= 30 qualifies
+    g = torch.Generator().manual_seed(21 + tie)
+    T = (torch.randn(B * (k + 1), V, generator=g)).to(torch.bfloat16)
+    Dr = (torch.randn(B * k, V, generator=g)).to(torch.bfloat16)
+    for rows in (T, Dr):
+        rows[:, 1000:1000 + tie] = 6.0       # the tie: above every Gaussian logit, so it holds the cut for K > 10
+        rows[:, 50000:50010] = 9.0           # ten equal logits above the tie
+    qi = torch.arange(0, (B + 1) * (k + 1), k + 1, dtype=torch.int32)
+    tk = torch.tensor([5, 11, 20, 30], dtype=torch.int32)
+    tp = torch.tensor([1.0, 1.0, 0.9, 0.5])
+    ids = torch.zeros(B * k, dtype=torch.int32)
+    for r in range(B):
+        q, kept, _ = oracle.filtered_row(Dr[r], 1.0, int(tk[r]), float(tp[r]))
+        ids[r] = int(torch.multinomial(q, 1, generator=g))
+    assert oracle.filtered_row(T[0], 1.0, 5, 1.0)[1] == 10             # cut inside the ten equal top logits: all kept
+    assert oracle.filtered_row(T[2], 1.0, 11, 1.0)[1] == 10 + tie      # cut inside the tie: all of it kept
+    ua, us = torch.rand(B * k, generator=g), torch.rand(B, generator=g)
+    ref = oracle.rejection_sample(T, Dr, ids, qi, ua, us, top_k=tk, top_p=tp)
+    acc, tok, _, ws = spx.rejection_sample(T.to(DEV), Dr.to(DEV), ids.to(DEV), qi.to(DEV), ua.to(DEV), us.to(DEV),
+                                           top_k=tk.to(DEV), top_p=tp.to(DEV))
+    torch.cuda.synchronize()
+    assert int(ws.status.item()) in (0, spx.DEV_DEGENERATE)
+
+    class _B:
+        pass
+    bb = _B()
+    bb.batch, bb.q_indptr, bb.u_accept, bb.u_sample = B, qi, ua, us
+    bb.target_logits, bb.draft_logits, bb.draft_ids = T, Dr, ids
+    bb.spec = type("S", (), {"vocab": V})
+    rep = check_sampling(bb, acc, tok, ref, top_k=tk, top_p=tp)
+    assert not rep.hard_mismatch, rep
+    assert rep.exact + rep.cdf_near_tie + rep.cdf_abs_near_tie + rep.accept_near_tie + rep.topp_near_tie == B
+
+
 def test_full_size_filtered():
     spec = W.CONFIGS[1]
     b_cpu = W.generate(spec)
