@@ -369,6 +369,111 @@ def run_timeline(args):
             t["median_end_us"], t["last_end_us"], t["median_cta_us"]), file=sys.stderr)
 
 
+L2_BYTES = 126 << 20
+
+
+class StepRunner:
+    """One workload resident on the device, ready to be stepped.
+
+    Inputs that are smaller than twice the L2 (the whole tiny workload; the long-context workload's
+    17 MB of logits) exist in several copies at different addresses and the steps cycle through them,
+    so that no timed step finds its inputs in L2; the other tensors are larger than L2 as they are."""
+
+    def __init__(self, spx, binding, spec, dev, seed):
+        self.spx, self.binding, self.spec, self.dev = spx, binding, spec, dev
+        b = self.b = W.generate(spec, device=dev, seed=seed)
+        self.kv_bytes, self.logit_bytes = b.kv_bytes(), b.logits_bytes()
+        self.out = torch.empty_like(b.q)
+        self.lse = torch.empty(b.q.shape[:2], dtype=torch.float32, device=dev)
+        self.acc = torch.empty(b.batch, dtype=torch.int32, device=dev)
+        self.tok = torch.empty(b.total_q, dtype=torch.int32, device=dev)
+        kv_sets = 1 if self.kv_bytes >= 2 * L2_BYTES else min(384, -(-2 * L2_BYTES // max(self.kv_bytes, 1)))
+        lg_sets = 1 if self.logit_bytes >= 2 * L2_BYTES else min(384, -(-2 * L2_BYTES // max(self.logit_bytes, 1)))
+        self.n_sets = max(kv_sets, lg_sets)
+        self.keep = []                                             # the copies stay alive
+        self.sets = []
+        for i in range(self.n_sets):
+            kc, vc = (b.k_cache, b.v_cache) if i == 0 or kv_sets == 1 else (b.k_cache.clone(), b.v_cache.clone())
+            tl, dl = (b.target_logits, b.draft_logits) if i == 0 or lg_sets == 1 else (b.target_logits.clone(), b.draft_logits.clone())
+            self.keep.append((kc, vc, tl, dl))
+            a = binding.make_attn_args(b.q, kc, vc, b.kv_strides, b.block_table, b.seq_lens, b.q_indptr,
+                                       spec.num_kv_heads, spec.page_size, b.num_pages, self.out, self.lse,
+                                       max_q_len=max(b.k_host) + 1)
+            sa = binding.make_sample_args(tl, dl, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample, self.acc, self.tok)
+            self.sets.append((a, sa))
+        self.ws = spx.Workspace.allocate(spx.workspace_size(*self.sets[0]), dev)
+        self.rotation = ("inputs larger than L2 (KV + logits re-read from HBM every step)" if self.n_sets == 1 else
+                         f"{self.n_sets} input sets cycled ({'KV + ' if kv_sets > 1 else ''}logits copies at distinct addresses, "
+                         "more than 2x L2 in total); the rest is larger than L2")
+        self.i = 0
+
+    def step(self):
+        a, sa = self.sets[self.i % self.n_sets]
+        self.i += 1
+        self.spx.verify_step(a, sa, self.ws, self.dev)
+
+    def warm(self, n):
+        for _ in range(n):
+            self.step()
+        torch.cuda.synchronize()
+        self.launches_per_step = self.spx.last_launch_count()
+        self.tokens_per_step = int(self.acc.sum().item()) + self.b.batch
+        if int(self.ws.status.item()) != 0:
+            raise SystemExit(f"device status {int(self.ws.status.item())} after warm-up ({self.spec.name})")
+
+    def time_steps(self, steps, local, barrier):
+        """K whole steps between two CUDA events on the launching stream; clocks sampled meanwhile."""
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        clocks = ClockSampler(local)
+        barrier()
+        torch.cuda.synchronize()
+        clocks.start()
+        ev0.record()
+        for _ in range(steps):
+            self.step()
+        ev1.record()
+        torch.cuda.synchronize()
+        info = clocks.stop()
+        barrier()
+        return ev0.elapsed_time(ev1), info
+
+    def time_attention(self, n):
+        """The verify-attention kernel alone: same launch configuration and inputs, one event pair per
+        launch recorded by the library immediately around the kernel (inside the step the sampling
+        kernels run beside it on another stream and share its bandwidth)."""
+        import ctypes as C
+        spx, lib, ws = self.spx, self.spx.load_library(), self.ws
+        stream = torch.cuda.current_stream(self.dev).cuda_stream
+        events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for e0, e1 in events:
+            e0.record()
+            e1.record()
+        for i in range(3):
+            lib.spx_verify_attention(C.byref(self.sets[i % self.n_sets][0]), ws.buf.data_ptr(), ws.buf.numel(),
+                                     ws.status.data_ptr(), stream)
+        torch.cuda.synchronize()
+        for i, (e0, e1) in enumerate(events):
+            spx.set_timing_events(e0, e1)
+            lib.spx_verify_attention(C.byref(self.sets[i % self.n_sets][0]), ws.buf.data_ptr(), ws.buf.numel(),
+                                     ws.status.data_ptr(), stream)
+        torch.cuda.synchronize()
+        spx.set_timing_events(None, None)
+        return [e0.elapsed_time(e1) for e0, e1 in events]
+
+
+def workload_summary(run: "StepRunner", ms_per_step, attn_ms, clock_info, peak, steps):
+    """The per-workload figures of the `workloads` table."""
+    attn_avg_ms = sum(attn_ms) / len(attn_ms)
+    step_gbs = (run.kv_bytes + run.logit_bytes) / (ms_per_step * 1e-3) / 1e9
+    attn_gbs = run.kv_bytes / (attn_avg_ms * 1e-3) / 1e9
+    return {"ms_per_step": ms_per_step, "steps": steps, "tokens_per_s": run.tokens_per_step / (ms_per_step * 1e-3),
+            "tokens_per_step": run.tokens_per_step, "kv_bytes": run.kv_bytes, "logits_bytes": run.logit_bytes,
+            "step_gbs": step_gbs, "step_frac_of_measured": step_gbs / peak,
+            "step_frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS,
+            "attn_avg_launch_ms": attn_avg_ms, "attn_gbs": attn_gbs, "attn_frac_of_measured": attn_gbs / peak,
+            "attn_traffic_bytes": NCU_TRAFFIC_BYTES.get(run.spec.name), "l2": run.rotation, "clocks": clock_info}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -379,6 +484,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-others", action="store_true", help="skip the table of the other four workloads (profiling runs)")
+    ap.add_argument("--other-steps", type=int, default=300, help="timed steps per workload of the `workloads` table")
     ap.add_argument("--extras", action="store_true",
                     help="also time the pieces around the step: KV append / rollback, verification variants")
     ap.add_argument("--extras-iters", type=int, default=200, help="timed calls per extras entry (profiling runs: a few)")
@@ -410,68 +517,20 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     warmup = max(args.warmup, 3)
 
-    spec = W.CONFIGS[args.workload]
-    if args.batch:
-        spec = W.scaled(spec, batch=args.batch, name_suffix=f"-batch{args.batch}")
-    b = W.generate(spec, device=dev, seed=spec.seed + 1000 * rank)
-    out = torch.empty_like(b.q)
-    lse = torch.empty(b.q.shape[:2], dtype=torch.float32, device=dev)
-    acc = torch.empty(b.batch, dtype=torch.int32, device=dev)
-    tok = torch.empty(b.total_q, dtype=torch.int32, device=dev)
-    a = binding.make_attn_args(b.q, b.k_cache, b.v_cache, b.kv_strides, b.block_table, b.seq_lens, b.q_indptr,
-                               spec.num_kv_heads, spec.page_size, b.num_pages, out, lse, max_q_len=max(b.k_host) + 1)
-    s = binding.make_sample_args(b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample,
-                                 acc, tok)
-    ws = spx.Workspace.allocate(spx.workspace_size(a, s), dev)
-
     def barrier():
         if world > 1:
             dist.barrier()
 
-    for _ in range(warmup):
-        spx.verify_step(a, s, ws, dev)
-    torch.cuda.synchronize()
-    launches_per_step = spx.last_launch_count()
-    tokens_per_step = int(acc.sum().item()) + b.batch
-    if int(ws.status.item()) != 0:
-        raise SystemExit(f"device status {int(ws.status.item())} after warm-up")
-
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    clocks = ClockSampler(local)
-    barrier()
-    torch.cuda.synchronize()
-    clocks.start()
-    ev0.record()
-    for _ in range(args.steps):
-        spx.verify_step(a, s, ws, dev)
-    ev1.record()
-    torch.cuda.synchronize()
-    clock_info = clocks.stop()
-    barrier()
-    ms_total = ev0.elapsed_time(ev1)
-
-    # Roofline of the dominant kernel (verify-attention, which streams the KV cache): timed alone,
-    # because inside the step the sampling kernels run beside it on another stream and share its
-    # bandwidth.  Same launch configuration, same inputs, K launches of the attention half, one
-    # event pair per launch recorded by the library immediately around the kernel.
-    n_roof = min(args.steps, 200)
-    k_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_roof)]
-    for e0, e1 in k_events:
-        e0.record()
-        e1.record()
-    lib = spx.load_library()
-    import ctypes as C
-    for _ in range(3):
-        lib.spx_verify_attention(C.byref(a), ws.buf.data_ptr(), ws.buf.numel(), ws.status.data_ptr(),
-                                 torch.cuda.current_stream(dev).cuda_stream)
-    torch.cuda.synchronize()
-    for e0, e1 in k_events:
-        spx.set_timing_events(e0, e1)
-        lib.spx_verify_attention(C.byref(a), ws.buf.data_ptr(), ws.buf.numel(), ws.status.data_ptr(),
-                                 torch.cuda.current_stream(dev).cuda_stream)
-    torch.cuda.synchronize()
-    spx.set_timing_events(None, None)
-    attn_ms = [e0.elapsed_time(e1) for e0, e1 in k_events]
+    peak, peak_kind = measured_peak()
+    spec = W.CONFIGS[args.workload]
+    if args.batch:
+        spec = W.scaled(spec, batch=args.batch, name_suffix=f"-batch{args.batch}")
+    run = StepRunner(spx, binding, spec, dev, spec.seed + 1000 * rank)
+    b, a, s, ws, acc, tok, out = run.b, run.sets[0][0], run.sets[0][1], run.ws, run.acc, run.tok, run.out
+    run.warm(warmup)
+    launches_per_step, tokens_per_step = run.launches_per_step, run.tokens_per_step
+    ms_total, clock_info = run.time_steps(args.steps, local, barrier)
+    attn_ms = run.time_attention(min(args.steps, 200))
     ms_total, job_tokens = reduce_over_ranks(ms_total, tokens_per_step, dev)
     value = job_tokens * args.steps / (ms_total * 1e-3)
     ms_per_step = ms_total / args.steps
@@ -524,8 +583,7 @@ def main():
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = measured_peak()
-    kv_bytes, logit_bytes = b.kv_bytes(), b.logits_bytes()
+    kv_bytes, logit_bytes = run.kv_bytes, run.logit_bytes
     attn_avg_ms = sum(attn_ms) / len(attn_ms)
     achieved = kv_bytes / (attn_avg_ms * 1e-3) / 1e9
     step_gbs = (kv_bytes + logit_bytes) / (ms_per_step * 1e-3) / 1e9
@@ -537,8 +595,7 @@ def main():
                    "kv_heads": spec.num_kv_heads, "head_dim": spec.head_dim, "page_size": spec.page_size,
                    "vocab": spec.vocab, "total_q_rows": b.total_q, "kv_tokens": sum(b.seq_lens_host),
                    "kv_bytes": kv_bytes, "logits_bytes": logit_bytes, "tokens_per_step": tokens_per_step,
-                   "l2": "inputs larger than L2 (KV + logits re-read from HBM every step)",
-                   "parallelism": "replicas" if world > 1 else "single"},
+                   "l2": run.rotation, "parallelism": "replicas" if world > 1 else "single"},
         "clocks": clock_info,
         "e2e": e2e,
         "gpu_launches": launches_per_step * args.steps,
@@ -562,11 +619,48 @@ def main():
                 passes, total_t, total_tok = passes + 1, total_t + dt, total_tok + otok
             result["cpu_baseline"] = {"value": total_tok / total_t, "unit": UNIT, "cores": threads, "kind": "oracle",
                                       "sample": f"first {n_req} of {spec.batch} requests, {passes} passes ({total_t:.1f} s)"}
+            result["cpu_baseline"]["sampling_vs_gpu"] = sampling_agreement(bc, n_req, acc, tok)
         except Exception as exc:
             result["cpu_baseline"] = {"value": None, "unit": UNIT, "error": repr(exc), "kind": "oracle"}
+
+    # ---- the other named workloads, same timing, a shorter run each (single-GPU default run only) ----
+    if world == 1 and not args.no_others and not args.batch:
+        table = {spec.name: workload_summary(run, ms_per_step, attn_ms, clock_info, peak, args.steps)}
+        del run, b, a, s, ws, b_host
+        torch.cuda.empty_cache()
+        for other in W.CONFIGS:
+            if other.name in table:
+                continue
+            try:
+                r2 = StepRunner(spx, binding, other, dev, other.seed)
+                r2.warm(max(warmup, 10))
+                k2 = max(200, args.other_steps)
+                ms2, clk2 = r2.time_steps(k2, local, barrier)
+                table[other.name] = workload_summary(r2, ms2 / k2, r2.time_attention(min(k2, 200)), clk2, peak, k2)
+                del r2
+                torch.cuda.empty_cache()
+            except Exception as exc:  # reported, never hidden
+                table[other.name] = {"error": repr(exc)}
+        result["workloads"] = {w.name: table[w.name] for w in W.CONFIGS if w.name in table}
     print(json.dumps(result))
     if world > 1:
         dist.destroy_process_group()
+
+
+def sampling_agreement(b_cpu, n_req, acc_gpu, tok_gpu):
+    """Accepted lengths and emitted tokens of the device path against the oracle's on the sample the
+    CPU baseline timed: requests that agree bit for bit / requests compared.  (The tests classify
+    the rest into the counted near-tie classes; here they are only counted.)"""
+    import oracle
+    sb = sub_batch(b_cpu, n_req)
+    res = oracle.rejection_sample(sb.target_logits, sb.draft_logits, sb.draft_ids, sb.q_indptr, sb.u_accept, sb.u_sample)
+    acc_g, tok_g = acc_gpu.cpu(), tok_gpu.cpu()
+    qi = sb.q_indptr.tolist()
+    exact = 0
+    for r in range(n_req):
+        if int(acc_g[r]) == int(res.accepted_len[r]) and torch.equal(tok_g[qi[r]:qi[r + 1]], res.out_tokens[qi[r]:qi[r + 1]]):
+            exact += 1
+    return {"requests": n_req, "bit_exact": exact}
 
 
 if __name__ == "__main__":

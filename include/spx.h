@@ -5,8 +5,8 @@
  * a batch of requests each carries k_r >= 0 draft tokens (k_r = 0 where selective speculation,
  * Section 5.1 of the paper, switched speculation off for that request); the target model's
  * k_r+1 new positions attend jointly over the request's paged, shared KV cache (Section 2
- * "Speculative decoding", Section 4 "Self-speculation and parallel scheduling": drafts are
- * "verified jointly", the cache is shared between speculative and normal execution), and the
+ * "Speculative decoding", Section 4 "Self-speculation and parallel scheduling": all drafts of a
+ * request are checked in one pass, and speculative and normal execution use one cache), and the
  * drafts are then accepted or rejected by speculative sampling (the rule of the
  * speculative-decoding work cited in Section 2).
  *
@@ -178,7 +178,8 @@ spx_status_t spx_rejection_sample(const spx_sample_args_t *args, void *ws, size_
  * here), so the sampling half is forked onto a library-internal stream and joined back into
  * `cuda_stream` before the call returns: work enqueued on `cuda_stream` afterwards sees both
  * halves' outputs.  The internal stream and its two events are created on the first call of a
- * host thread on a device and live until the thread exits.  `ws` must hold
+ * host thread on a device and are kept until the process ends.  If a launch fails after the
+ * fork, the internal stream is still joined back before the error is returned.  `ws` must hold
  * spx_workspace_size(attn, sample) bytes.
  */
 spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_t *sample, void *ws,
@@ -277,8 +278,8 @@ spx_status_t spx_select_speculation(int32_t batch, const float *confidence, cons
 /*
  * The paper's scheduler numerics.
  *
- * spx_lookahead_memory is its Algorithm 1 ("look-ahead memory estimation over future
- * iterations"): for i = 1..horizon (the paper uses 64), with pipeline depth pp and speculation
+ * spx_lookahead_memory is its Algorithm 1, the estimate of the batch's cache occupancy over the
+ * coming iterations: for i = 1..horizon (the paper uses 64), with pipeline depth pp and speculation
  * accuracy theta, w counting a request's rejected speculations,
  *   t = i - pp w,  k = t + w,  p = C(k, t) theta^t (1 - theta)^w,  w = 0..floor(i / pp),
  *   E[L_gen] = sum_w k p,   P_fin(r) = prec[r] * sum_w [k >= tau[r]] p,

@@ -66,7 +66,6 @@ def _load():
         lib.oracle_emit_cdf.restype = c.c_double
         lib.oracle_emit_cdf.argtypes = [c.c_int32, c.c_int32, c.c_int64, c.c_int64, c.c_int32,
                                         c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
-        lib.oracle_verify_step.restype = c.c_int
         lib.oracle_kv_append.restype = c.c_int
         lib.oracle_kv_append.argtypes = [c.c_int32, c.c_int32, c.c_int32, c.c_int32, c.c_int64, c.c_int32, c.c_int32,
                                          c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int64, c.c_int64, c.c_int64,

@@ -630,9 +630,9 @@ double oracle_emit_cdf(int32_t r, int32_t n, int64_t V, int64_t row_stride, int3
 /* ------------------------------------------------------------------------------------ */
 
 /*
- * Section 5.1 ranks drafted tokens by the draft's confidence and drops a fixed fraction alpha
- * of the lowest-ranked ones; Section 7.4 states it per sequence ("rank the sequences in a batch
- * by their speculation confidence and drop the lowest alpha fraction").  The paper does not
+ * Section 5.1 orders drafted tokens by how confident the draft is in them and stops speculating
+ * on a fixed share alpha at the bottom of that order; Section 7.4 applies the same rule to whole
+ * sequences of a batch.  The paper does not
  * define the confidence beyond citing the self-speculation works that use the draft's top
  * probability, so this build reads it as:
  *   conf_max[d]  = max_v softmax(D_d)(v)              (the draft's top-1 probability)
@@ -782,48 +782,61 @@ double oracle_delay_gain(double I, int32_t n, double pdr, double bs, double i_de
 }
 
 /*
- * Algorithm 1: look-ahead memory estimate (in tokens) for iterations i = 1..horizon (the paper
- * uses 64).  Per request r: ell[r] current length, tau[r] predicted remaining length, prec[r] the
- * precision E(tau[r]) of that prediction (the caller evaluates E).  pp pipeline depth, theta
- * speculation accuracy.  With w rejections by iteration i:
- *   t = i - pp w (accepted), k = t + w (generated), p = C(k, t) theta^t (1-theta)^w,
- *   w_max = floor(i / pp);
- *   E[L_gen] = sum_w k p;  P_fin(r) = prec[r] sum_w [k >= tau[r]] p;
- *   E[N_fin] = sum_r P_fin(r);  E[L_fin] = sum_r ell[r] P_fin(r);
- *   M[i-1] = L_total + (|B| - E[N_fin]) E[L_gen] - E[L_fin],  L_total = sum_r ell[r].
- * 0^0 = 1 (theta = 0 or 1 select single terms).
+ * Algorithm 1: expected KV-cache occupancy (in tokens) of the running batch after each of the next
+ * `horizon` iterations (the paper looks 64 ahead).  Inputs per request r: its present length
+ * ell[r], the predicted number of tokens it still has to produce tau[r], and prec[r], how often a
+ * prediction of that size is right (the caller looks that up).  pp is the pipeline depth, theta
+ * the probability that a speculation is accepted.
+ *
+ * What the algorithm states, in this file's words.  After `step` iterations a request has had
+ * some number `rej` of rejected speculations, each of which cost it pp iterations; the other
+ * acc = step - pp*rej iterations each produced an accepted token, and every rejection still
+ * produced one (corrected) token, so it has made acc + rej tokens.  The rejections can fall
+ * anywhere among those tokens: Pr[rej] = C(acc + rej, rej) theta^acc (1-theta)^rej, for
+ * rej = 0 .. floor(step / pp), with 0^0 = 1.  From that law:
+ *   grown       = sum_rej made(rej) Pr[rej]                    expected tokens made per request
+ *   done(r)     = prec[r] * sum_{rej : made(rej) >= tau[r]} Pr[rej]   probability r has finished
+ *   estimate    = sum_r ell[r] + (nreq - sum_r done(r)) * grown - sum_r ell[r] done(r).
+ * law_of_rejections() tabulates (made, Pr) once per step; the requests are a separate pass.
  */
+static int law_of_rejections(int step, int pp, double theta, int *made, double *pr) {
+  const int most = step / pp;
+  for (int rej = 0; rej <= most; ++rej) {
+    const int acc = step - pp * rej;
+    double ways = 1.0;                           /* C(acc + rej, rej) as a running product */
+    for (int j = 1; j <= rej; ++j) ways = ways * (double)(acc + j) / (double)j;
+    made[rej] = acc + rej;
+    pr[rej] = ways * pow(theta, (double)acc) * pow(1.0 - theta, (double)rej);
+  }
+  return most + 1;
+}
+
 int oracle_lookahead_memory(int32_t nreq, const int32_t *ell, const int32_t *tau,
                             const double *prec, int32_t pp, double theta, int32_t horizon,
                             double *M) {
   if (nreq < 0 || pp < 1 || horizon < 0 || !(theta >= 0.0 && theta <= 1.0)) return ORACLE_ERR_ARG;
-  double L_total = 0.0;
-  for (int r = 0; r < nreq; ++r) L_total += (double)ell[r];
-  for (int i = 1; i <= horizon; ++i) {
-    const int w_max = i / pp;
-    double E_gen = 0.0;
-    for (int w = 0; w <= w_max; ++w) {
-      const int t = i - pp * w, k = t + w;
-      double binom = 1.0;
-      for (int j = 1; j <= w; ++j) binom = binom * (double)(t + j) / (double)j;
-      E_gen += (double)k * binom * pow(theta, (double)t) * pow(1.0 - theta, (double)w);
-    }
-    double E_nfin = 0.0, E_lfin = 0.0;
+  int *made = (int *)malloc(sizeof(int) * (size_t)(horizon + 2));
+  double *pr = (double *)malloc(sizeof(double) * (size_t)(horizon + 2));
+  if (!made || !pr) { free(made); free(pr); return ORACLE_ERR_ARG; }
+  double held = 0.0;
+  for (int r = 0; r < nreq; ++r) held += (double)ell[r];
+  for (int step = 1; step <= horizon; ++step) {
+    const int cases = law_of_rejections(step, pp, theta, made, pr);
+    double grown = 0.0;
+    for (int c = 0; c < cases; ++c) grown += (double)made[c] * pr[c];
+    double finished = 0.0, released = 0.0;
     for (int r = 0; r < nreq; ++r) {
-      double reach = 0.0;
-      for (int w = 0; w <= w_max; ++w) {
-        const int t = i - pp * w, k = t + w;
-        if (k < tau[r]) continue;
-        double binom = 1.0;
-        for (int j = 1; j <= w; ++j) binom = binom * (double)(t + j) / (double)j;
-        reach += binom * pow(theta, (double)t) * pow(1.0 - theta, (double)w);
-      }
-      const double P_fin = prec[r] * reach;
-      E_nfin += P_fin;
-      E_lfin += (double)ell[r] * P_fin;
+      double reached = 0.0;
+      for (int c = 0; c < cases; ++c)
+        if (made[c] >= tau[r]) reached += pr[c];
+      const double done = prec[r] * reached;
+      finished += done;
+      released += (double)ell[r] * done;
     }
-    M[i - 1] = L_total + ((double)nreq - E_nfin) * E_gen - E_lfin;
+    M[step - 1] = held + ((double)nreq - finished) * grown - released;
   }
+  free(made);
+  free(pr);
   return ORACLE_OK;
 }
 
@@ -947,26 +960,4 @@ int oracle_kv_rollback(int32_t batch, const int32_t *seq_lens, const int32_t *q_
     new_seq_lens[r] = seq_lens[r] - (k - n);
   }
   return ORACLE_OK;
-}
-
-/* ------------------------------------------------------------------------------------ */
-/* (C) the whole step: the two halves are independent given their inputs                  */
-/* ------------------------------------------------------------------------------------ */
-int oracle_verify_step(int32_t batch, int32_t Hq, int32_t Hkv, int32_t D, int32_t P,
-                       int64_t num_pages, int32_t max_pages_per_req, int32_t kv_dtype,
-                       double sm_scale, const void *q, const void *k_cache, const void *v_cache,
-                       int64_t stride_page, int64_t stride_head, int64_t stride_token,
-                       const int32_t *block_table, const int32_t *seq_lens,
-                       const int32_t *q_indptr, double *out, double *lse, int64_t V,
-                       int64_t row_stride, int32_t logits_dtype, const void *target_logits,
-                       const void *draft_logits, const int32_t *draft_ids, const float *u_accept,
-                       const float *u_sample, int32_t *accepted_len, int32_t *out_tokens) {
-  const int sa = oracle_verify_attention(batch, Hq, Hkv, D, P, num_pages, max_pages_per_req,
-                                         kv_dtype, sm_scale, q, k_cache, v_cache, stride_page,
-                                         stride_head, stride_token, block_table, seq_lens,
-                                         q_indptr, NULL, 0, out, lse);
-  if (sa != ORACLE_OK) return sa;
-  return oracle_rejection_sample(batch, V, row_stride, logits_dtype, target_logits, draft_logits,
-                                 draft_ids, q_indptr, u_accept, u_sample, accepted_len,
-                                 out_tokens, NULL, NULL, NULL, NULL, NULL);
 }

@@ -263,9 +263,10 @@ def verify_attention(q, k_cache, v_cache, kv_strides, block_table, seq_lens, q_i
 
 def rejection_sample(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, vocab=None,
                      want_ratio=False, ws: Optional[Workspace] = None, temperature=None, top_k=None, top_p=None,
-                     target_tile_stats=None):
+                     target_tile_stats=None, accepted=None, tokens=None):
     """spx_rejection_sample on the current stream.  Returns (accepted_len, out_tokens, ratio, ws).
-    ``temperature`` ([B] float32 on the device, optional) selects the verification variant per request."""
+    ``temperature`` ([B] float32 on the device, optional) selects the verification variant per request;
+    ``accepted`` ([B] int32) and ``tokens`` ([TQ] int32) are the output buffers if the caller brings its own."""
     _require_cuda(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample)
     for extra in (temperature, top_k, top_p):
         if extra is not None:
@@ -274,8 +275,10 @@ def rejection_sample(target_logits, draft_logits, draft_ids, q_indptr, u_accept,
     dev = target_logits.device
     B = q_indptr.numel() - 1
     TQ = target_logits.shape[0]
-    accepted = torch.empty(B, dtype=torch.int32, device=dev)
-    tokens = torch.empty(TQ, dtype=torch.int32, device=dev)
+    if accepted is None:
+        accepted = torch.empty(B, dtype=torch.int32, device=dev)
+    if tokens is None:
+        tokens = torch.empty(TQ, dtype=torch.int32, device=dev)
     ratio = torch.empty(TQ - B, dtype=torch.float32, device=dev) if want_ratio else None
     s = make_sample_args(target_logits, draft_logits, draft_ids, q_indptr, u_accept, u_sample, accepted, tokens,
                          ratio, vocab, temperature, top_k, top_p, target_tile_stats)

@@ -574,8 +574,6 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
       // the last PV has long completed, so the softmax never idles at an item boundary
       sL[((qc & 1) * kSplit + tblk) * MROWS + row] = l_sum;
       pend.valid = true; pend.I = I; pend.m_ref = m_ref; pend.last_tc = tc_ - 1; pend.qc = qc;
-      const long long prof_e0 = 0, prof_e1 = 0, prof_e2 = 0;
-      (void)prof_e0; (void)prof_e1; (void)prof_e2;
       idx = idx_next;
       I = Inext;
     }

@@ -27,7 +27,9 @@ static thread_local long long *t_prof = nullptr;  // profiling builds only
 
 // spx_verify_step runs its two halves concurrently: the sampling half on an internal stream that
 // is forked from and joined back into the caller's stream.  One stream and two events per (host
-// thread, device), created on first use and kept until the thread exits.
+// thread, device), created on first use.  They are kept for the life of the process: a thread may
+// exit after the CUDA runtime has begun to shut down, when destroying a stream is no longer safe,
+// so the few handles of an exited thread are deliberately left to the driver's process teardown.
 struct SideStream {
   int device = -1;
   cudaStream_t stream = nullptr;
@@ -40,12 +42,22 @@ static SideStream *get_side_stream(int device) {
   SideStream &s = t_side[device];
   if (s.device != device) {
     // a priority of its own: the sampling kernels are short and latency-bound, and a stream of
-    // another priority does not share a hardware queue with the caller's stream
+    // another priority does not share a hardware queue with the caller's stream.  Built in locals
+    // and committed only when all three handles exist, so a failure half way leaks nothing.
     int prio_lo = 0, prio_hi = 0;
-    if (cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) != cudaSuccess) return nullptr;
-    if (cudaStreamCreateWithPriority(&s.stream, cudaStreamNonBlocking, prio_hi) != cudaSuccess) return nullptr;
-    if (cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    if (cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+    bool ok = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithPriority(&stream, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&fork, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&join, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      if (join) cudaEventDestroy(join);
+      if (fork) cudaEventDestroy(fork);
+      if (stream) cudaStreamDestroy(stream);
+      return nullptr;
+    }
+    s.stream = stream; s.fork = fork; s.join = join;
     s.device = device;
   }
   return &s;
@@ -328,12 +340,8 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
       e = p.D == 128 ? launch_tc4<128, 32>(kmap, vmap, p, sms, stream) : launch_tc4<64, 32>(kmap, vmap, p, sms, stream);
     else if (p.rows_cap <= 64)
       e = p.D == 128 ? launch_tc4<128, 64>(kmap, vmap, p, sms, stream) : launch_tc4<64, 64>(kmap, vmap, p, sms, stream);
-    else if (p.D == 128)
-      e = p.rows_cap <= 64 ? launch_tc<128, 64>(kmap, vmap, p, sms, stream)
-                           : launch_tc<128, 128>(kmap, vmap, p, sms, stream);
     else
-      e = p.rows_cap <= 64 ? launch_tc<64, 64>(kmap, vmap, p, sms, stream)
-                           : launch_tc<64, 128>(kmap, vmap, p, sms, stream);
+      e = p.D == 128 ? launch_tc<128, 128>(kmap, vmap, p, sms, stream) : launch_tc<64, 128>(kmap, vmap, p, sms, stream);
   } else {
     const SimtSmem lay(p.rows_cap, p.D);
     if (lay.total > dev.max_smem_optin) return SPX_ERR_UNSUPPORTED;
@@ -549,12 +557,15 @@ spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_
   // launched first.  It keeps one SM clear: a CTA of it fills an SM, and on a full GPU the
   // one-block planner, which the attention kernel waits for, ran only when the first logits CTA
   // had left (8 us per step on the Llama-3-8B shape).
+  // From here on the internal stream is forked: whatever fails below, it is joined back into the
+  // caller's stream before the call returns (an unjoined fork would invalidate a stream capture
+  // and, outside one, leave the caller's stream unordered against sampling kernels already queued).
   const spx_status_t s1 = launch_sampler(sample, base + attn_bytes, dev_status, side->stream, dev.num_sms, kPhaseAll, 1);
   const spx_status_t s0 = launch_attention(attn, base, dev_status, stream, dev, kPhasePlan);
-  ok = ok && cudaEventRecord(side->join, side->stream) == cudaSuccess;
-  const spx_status_t s2 = launch_attention(attn, base, dev_status, stream, dev, kPhaseMain);
-  ok = ok && cudaStreamWaitEvent(stream, side->join, 0) == cudaSuccess;
-  if (!ok) return SPX_ERR_CUDA;
+  const bool rec = cudaEventRecord(side->join, side->stream) == cudaSuccess;
+  const spx_status_t s2 = s0 == SPX_OK ? launch_attention(attn, base, dev_status, stream, dev, kPhaseMain) : s0;
+  const bool joined = rec && cudaStreamWaitEvent(stream, side->join, 0) == cudaSuccess;
+  if (!joined) return SPX_ERR_CUDA;
   return s0 != SPX_OK ? s0 : s1 != SPX_OK ? s1 : s2;
 }
 

@@ -2,8 +2,13 @@
 
 Tolerances (stated where they are used as well):
   * attention, bf16: max abs error <= 2e-2 (contract) and, because that bound is loose next to
-    the signal at long context, also relative RMS error <= 1e-2 and |LSE error| <= 2e-3;
-    fp32: max abs <= 1e-4, relative RMS <= 1e-5, |LSE error| <= 1e-4.
+    the signal at long context, also relative RMS error <= 1e-2 and |LSE error| <= 2e-5;
+    fp32: max abs <= 1e-4, relative RMS <= 1e-5, |LSE error| <= 2e-5.
+    The LSE gate is the one that sees a lost page: leaving 16 of L tokens out of a softmax over
+    N(0,1) scores lowers LSE by about 16/L, i.e. 4e-3 at L = 4096 and 5e-4 at L = 32768, while the
+    output moves by only 3e-3 and 4e-4.  The kernels form the row sums in fp32 from exact bf16
+    products; observed |LSE error| on the five workloads at full size is 1.2e-6 to 1.4e-6, so the
+    gate sits 15x above the arithmetic's noise and 20x below the smallest lost-page signal.
   * sampling: accepted lengths and token ids bit-exact, except requests in which some consulted
     draft has |p/q - u| < 1e-6 (accept-class near tie) or whose target s*R lies within 1e-6*R of
     the CDF interval of the token the GPU chose (cdf-class near tie, an fp32 scan cannot
@@ -31,8 +36,8 @@ import oracle
 import paper_2609_34370_b200 as spx
 
 ATTN_TOL = {
-    torch.bfloat16: dict(max_abs=2e-2, rel_rms=1e-2, lse_abs=2e-3),
-    torch.float32: dict(max_abs=1e-4, rel_rms=1e-5, lse_abs=1e-4),
+    torch.bfloat16: dict(max_abs=2e-2, rel_rms=1e-2, lse_abs=2e-5),
+    torch.float32: dict(max_abs=1e-4, rel_rms=1e-5, lse_abs=2e-5),
 }
 ACCEPT_BAND = 1e-6
 CDF_BAND = 1e-6
@@ -40,11 +45,61 @@ CDF_ABS_BAND = 2.0 ** -22       # variants only: absolute probability mass
 TOPP_BAND = 1e-6                # top-p only: margin of the crossing, in units of the survivors' mass
 
 
+GUARD_BYTES = 4096              # guard band on each side of every buffer the library writes
+GUARD_BYTE = 0xC3
+
+
+class Guarded:
+    """A device buffer with a guard band before and after it.  The bands are filled with a fixed byte
+    and must read back unchanged after the call: the stand-in for a memory checker on the buffers the
+    library writes (workspace, attention output, LSE, accepted lengths, tokens)."""
+
+    def __init__(self, shape, dtype, device, name):
+        self.name = name
+        nbytes = int(torch.tensor([], dtype=dtype).element_size())
+        for d in (shape if isinstance(shape, (tuple, list, torch.Size)) else (shape,)):
+            nbytes *= int(d)
+        self.nbytes = nbytes
+        pad = (-nbytes) % 256                                       # the back band starts on a 256-byte boundary
+        self.raw = torch.full((GUARD_BYTES + nbytes + pad + GUARD_BYTES,), GUARD_BYTE, dtype=torch.uint8, device=device)
+        self.view = self.raw[GUARD_BYTES:GUARD_BYTES + nbytes].view(dtype).view(shape)
+        assert self.raw.device.type != "cuda" or self.view.data_ptr() % 256 == 0   # the library wants 256-byte aligned scratch
+
+    def check(self):
+        front = self.raw[:GUARD_BYTES]
+        back = self.raw[GUARD_BYTES + self.nbytes:]
+        assert bool((front == GUARD_BYTE).all()), f"write before the start of {self.name}"
+        assert bool((back == GUARD_BYTE).all()), f"write past the end of {self.name}"
+
+
+def guarded_workspace(nbytes, device, name="workspace"):
+    g = Guarded((nbytes,), torch.uint8, device, name)
+    return g, spx.Workspace(g.view, torch.zeros(1, dtype=torch.int32, device=device))
+
+
 def gpu_attention(b, ws=None, **kw):
+    """spx_verify_attention with the output, the LSE and (unless the caller brings one) the workspace
+    inside guard bands, which are checked after the call."""
+    from paper_2609_34370_b200 import binding
     s = b.spec
+    dev = b.q.device
+    g_out = Guarded(tuple(b.q.shape), b.q.dtype, dev, "attention output")
+    g_lse = Guarded(tuple(b.q.shape[:2]), torch.float32, dev, "lse")
+    guards = [g_out, g_lse]
+    if ws is None:
+        a = binding.make_attn_args(b.q, b.k_cache, b.v_cache, b.kv_strides, b.block_table, b.seq_lens, b.q_indptr,
+                                   s.num_kv_heads, s.page_size, b.num_pages, g_out.view, g_lse.view,
+                                   kw.get("sm_scale", 0.0), kw.get("max_q_len", 0))
+        g_ws, ws = guarded_workspace(spx.workspace_size(a, None), dev, "attention workspace")
+        ws._guard = g_ws
+    if getattr(ws, "_guard", None) is not None:
+        guards.append(ws._guard)
     out, lse, ws = spx.verify_attention(b.q, b.k_cache, b.v_cache, b.kv_strides, b.block_table, b.seq_lens,
-                                        b.q_indptr, s.num_kv_heads, s.page_size, b.num_pages, ws=ws, **kw)
+                                        b.q_indptr, s.num_kv_heads, s.page_size, b.num_pages, out=g_out.view,
+                                        lse=g_lse.view, ws=ws, **kw)
     torch.cuda.synchronize()
+    for g in guards:
+        g.check()
     return out, lse, ws
 
 
@@ -74,7 +129,9 @@ def check_attention(b, out_gpu, lse_gpu, out_ref, lse_ref, reqs=None):
     max_abs = float((og - orf).abs().max())
     rel_rms = float((og - orf).norm() / orf.norm())
     lse_abs = float((lg - lrf).abs().max())
-    stats = dict(max_abs=max_abs, rel_rms=rel_rms, lse_abs=lse_abs)
+    stats = dict(max_abs=max_abs, rel_rms=rel_rms, lse_abs=lse_abs, rows=int(rows.numel()))
+    print(f"\n[attention parity {getattr(b.spec, 'name', '?')}] " + ", ".join(
+        f"{k} {v:.3e}" if isinstance(v, float) else f"{k} {v}" for k, v in stats.items()))
     assert max_abs <= tol["max_abs"], stats
     assert rel_rms <= tol["rel_rms"], stats
     assert lse_abs <= tol["lse_abs"], stats
@@ -149,7 +206,26 @@ def check_sampling(b_cpu, acc_gpu, tok_gpu, ref: Optional[oracle.SampleResult] =
 
 
 def gpu_sample(b, **kw):
+    """spx_rejection_sample with accepted lengths, tokens and workspace inside checked guard bands."""
+    from paper_2609_34370_b200 import binding
+    dev = b.target_logits.device
+    B, TQ = b.q_indptr.numel() - 1, b.target_logits.shape[0]
+    g_acc = Guarded((B,), torch.int32, dev, "accepted_len")
+    g_tok = Guarded((TQ,), torch.int32, dev, "out_tokens")
+    guards = [g_acc, g_tok]
+    ws = kw.pop("ws", None)
+    if ws is None:
+        sa = binding.make_sample_args(b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr, b.u_accept, b.u_sample,
+                                      g_acc.view, g_tok.view, None, kw.get("vocab"), kw.get("temperature"),
+                                      kw.get("top_k"), kw.get("top_p"), kw.get("target_tile_stats"))
+        g_ws, ws = guarded_workspace(spx.workspace_size(None, sa), dev, "sampling workspace")
+        ws._guard = g_ws
+    if getattr(ws, "_guard", None) is not None:
+        guards.append(ws._guard)
     acc, tok, ratio, ws = spx.rejection_sample(b.target_logits, b.draft_logits, b.draft_ids, b.q_indptr,
-                                               b.u_accept, b.u_sample, **kw)
+                                               b.u_accept, b.u_sample, ws=ws, accepted=g_acc.view, tokens=g_tok.view,
+                                               **kw)
     torch.cuda.synchronize()
+    for g in guards:
+        g.check()
     return acc, tok, ratio, ws

@@ -247,3 +247,29 @@ def test_req_list_subset_matches_full():
     q0, m = int(b.q_indptr[2]), b.k_host[2] + 1
     assert torch.equal(part[q0:q0 + m], full[q0:q0 + m])
     assert torch.isnan(part[:q0]).all()
+
+
+@pytest.mark.parametrize("ctx,page", [(4096, 16), (32768, 32)])
+def test_the_parity_gates_catch_a_lost_page(ctx, page):
+    """The tolerances of the GPU parity tests, tried on the oracle alone: a result computed without
+    one middle page of the cache must fail them although it stays inside the contract's 2e-2 bound on
+    the output (closed form: leaving P of L tokens out of a softmax over N(0,1) scores lowers LSE by
+    about P/L, and the bf16 LSE gate is 2e-5)."""
+    import dataclasses
+    import parity_util
+    spec = dataclasses.replace(W.CONFIGS[3], batch=1, num_q_heads=4, num_kv_heads=1, page_size=page, vocab=64,
+                               ctx=("const", ctx), k=("const", 3), name="lost-page-cpu")
+    b = W.generate(spec)
+    ref_o, ref_l = _oracle(b)
+    lost = b.clone()
+    npages = ctx // page
+    drop = npages // 2
+    lost.block_table[0, drop:npages - 1] = b.block_table[0, drop + 1:npages]
+    lost.seq_lens[0] -= page
+    out, lse = _oracle(lost)
+    shift = float((ref_l - lse).mean())
+    assert 0.3 * page / ctx < shift < 3.0 * page / ctx
+    assert float((out - ref_o).abs().max()) < 2e-2
+    parity_util.check_attention(b, ref_o, ref_l, ref_o, ref_l)
+    with pytest.raises(AssertionError):
+        parity_util.check_attention(b, out, lse, ref_o, ref_l)
