@@ -8,7 +8,8 @@ Tolerances (stated where they are used as well):
     N(0,1) scores lowers LSE by about 16/L, i.e. 4e-3 at L = 4096 and 5e-4 at L = 32768, while the
     output moves by only 3e-3 and 4e-4.  The kernels form the row sums in fp32 from exact bf16
     products; observed |LSE error| on the five workloads at full size is 1.2e-6 to 1.4e-6, so the
-    gate sits 15x above the arithmetic's noise and 20x below the smallest lost-page signal.
+    gate sits 15x above the arithmetic's noise and 20x below the smallest lost-page signal.  (LSE
+    comes back as fp32, so four units in the last place of the value are allowed on top.)
   * sampling: accepted lengths and token ids bit-exact, except requests in which some consulted
     draft has |p/q - u| < 1e-6 (accept-class near tie) or whose target s*R lies within 1e-6*R of
     the CDF interval of the token the GPU chose (cdf-class near tie, an fp32 scan cannot
@@ -128,7 +129,9 @@ def check_attention(b, out_gpu, lse_gpu, out_ref, lse_ref, reqs=None):
     assert torch.isfinite(og).all() and torch.isfinite(lg).all()
     max_abs = float((og - orf).abs().max())
     rel_rms = float((og - orf).norm() / orf.norm())
-    lse_abs = float((lg - lrf).abs().max())
+    # LSE is returned as fp32: beside the absolute gate, four units in the last place of the value
+    # itself (a needle key puts LSE near 60, where one fp32 step is 4e-6)
+    lse_abs = float(((lg - lrf).abs() - lrf.abs() * 2.0 ** -21).clamp(min=0).max())
     stats = dict(max_abs=max_abs, rel_rms=rel_rms, lse_abs=lse_abs, rows=int(rows.numel()))
     print(f"\n[attention parity {getattr(b.spec, 'name', '?')}] " + ", ".join(
         f"{k} {v:.3e}" if isinstance(v, float) else f"{k} {v}" for k, v in stats.items()))
