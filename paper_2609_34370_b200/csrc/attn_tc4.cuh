@@ -91,7 +91,8 @@ __host__ __device__ constexpr uint32_t idesc_ws(uint32_t m, uint32_t n, bool b_m
 
 template <int D, int MROWS>
 __global__ void __launch_bounds__(kTcThreads, 1)
-attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, AttnParams p) {
+attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
+                const __grid_constant__ CUtensorMap qmap, AttnParams p) {
   SPX_TL_SCOPE(kTlAttention);
   using Cfg = Tc4Cfg<D, MROWS>;
   using namespace tc;
@@ -115,7 +116,7 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   if (kProfile) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(prof_g0));
   if (tid == 0) {
     for (int s = 0; s < 4; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->v_full[s], 1); mbar_init(&bars->k_empty[s], 1); mbar_init(&bars->v_empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&bars->s_full[b], 1); mbar_init(&bars->p_full[b], 4); mbar_init(&bars->q_full[b], 4); mbar_init(&bars->q_empty[b], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&bars->s_full[b], 1); mbar_init(&bars->p_full[b], 4); mbar_init(&bars->q_full[b], 1); mbar_init(&bars->q_empty[b], 1); }
     mbar_init(&bars->pv_done[0], 1);
     mbar_init(&bars->pv_done[1], 1);
     mbar_init(&bars->o_free2[0], 4);
@@ -213,12 +214,32 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
     int page_la = load_page(la);
     uint32_t tc_ = 0;
     bool ok = true;
+    // bytes of one Q box pair: G * max_q_len packed rows of D columns (rows past the tensor read as zero)
+    const uint32_t q_bytes = (uint32_t)(p.G * p.q_box_rows) * D * 2;
     while (la.valid && ok && !bars->abort) {
       const GCursor cur = la;
       const int page = page_la;
       advance(la);
       page_la = load_page(la);
       const int g = cur.e.g;
+      if (cur.tile0 == cur.e.tile_begin) {
+        // a new work entry: its packed query rows go into the Q buffer of its parity, as soon as the
+        // last score MMA of the entry that used the buffer before has read it.  The copy is issued
+        // ahead of the entry's first K tile, so it has the tiles still in the ring to arrive.
+        const uint32_t qc = (uint32_t)cur.it;
+        const uint32_t qb = Cfg::kQBufs == 2 ? (qc & 1) : 0;
+        const uint32_t uses = Cfg::kQBufs == 2 ? (qc >> 1) : qc;   // earlier uses of this buffer
+        if (uses >= 1) {
+          ok = warp_wait(&bars->q_empty[qb], (uses - 1) & 1, 2);
+          if (!ok) break;
+        }
+        if (lane == 0) {
+          mbar_expect_tx(&bars->q_full[qb], q_bytes);
+#pragma unroll
+          for (int h = 0; h < Cfg::kHalves; ++h)
+            tma_load_3d(smem_u32(sQ + qb * Cfg::kQBytes + h * Cfg::kQHalfBytes), &qmap, &bars->q_full[qb], h * 64, g * p.G, cur.e.q0);
+        }
+      }
       const int t_end = min(cur.e.tile_end * kTileTokens, cur.e.L);
       for (int ti = 0; ti < tiles_per_group && cur.tile0 + ti < cur.e.tile_end; ++ti, ++tc_) {
         const int tile = cur.tile0 + ti;
@@ -330,41 +351,8 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
     const int row = rgrp * 32 + lane;                       // packed query row
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const int sm_tid = tid - 64;
-    const __nv_bfloat16 *Qg = reinterpret_cast<const __nv_bfloat16 *>(p.q);
     __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(p.out);
-    constexpr int kChunksPerRow = D / 8;
     constexpr int CB = Cfg::kColBlock;
-
-    // Q rows of an item -> shared memory (K-major, 128-byte swizzle), in two halves so that the
-    // global loads can be issued early and stored later: each thread owns up to kQPerThread
-    // 16-byte chunks of the 32 x D tile.
-    constexpr int kQPerThread = (MROWS * kChunksPerRow + 127) / 128;
-    uint4 qreg[kQPerThread];
-    auto q_load = [&](const ItemInfo &J) {
-#pragma unroll
-      for (int u = 0; u < kQPerThread; ++u) {
-        const int i = sm_tid + u * 128;
-        if (i < J.R * kChunksPerRow) {
-          const int r = i / kChunksPerRow, c16 = i % kChunksPerRow;
-          const int j = r / p.G, hg = r % p.G;
-          qreg[u] = *reinterpret_cast<const uint4 *>(Qg + ((int64_t)(J.q0 + j) * p.Hq + J.g * p.G + hg) * D + c16 * 8);
-        }
-      }
-    };
-    auto q_store = [&](const ItemInfo &J, uint32_t qb) {
-      unsigned char *dst = sQ + qb * Cfg::kQBytes;
-#pragma unroll
-      for (int u = 0; u < kQPerThread; ++u) {
-        const int i = sm_tid + u * 128;
-        if (i < J.R * kChunksPerRow) {
-          const int r = i / kChunksPerRow, c16 = i % kChunksPerRow, h = c16 >> 3, c = c16 & 7;
-          *reinterpret_cast<uint4 *>(dst + h * Cfg::kQHalfBytes + (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4)) = qreg[u];
-        }
-      }
-      fence_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->q_full[qb]);
-    };
 
     uint32_t tc_ = 0, qc = 0, ec = 0;
     bool ok = true;
@@ -426,40 +414,14 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
     };
     ItemInfo I, Inext;
     int idx = item_index(0);
-    if (idx >= 0) {
-      I = make_item(entry_of(idx), idx);
-      q_load(I);
-      q_store(I, 0);
-    }
+    if (idx >= 0) I = make_item(entry_of(idx), idx);
     for (int it = 0; idx >= 0 && ok; ++it, ++qc) {
       if (bars->abort) break;
-      // The next item's work entry is requested now, its Q rows after the first tile, and they are
-      // stored after the second tile (or at the end of a shorter item): no load is waited on.
+      // the next item's work entry is requested now and unpacked at the end of this item (the query
+      // rows themselves are fetched by the producer warp)
       const int idx_next = item_index(it + 1);
       WorkEntry e_next;
       if (idx_next >= 0) e_next = entry_of(idx_next);
-      int q_stage = idx_next >= 0 ? 0 : 2;  // 0: nothing yet, 1: loads issued, 2: stored / nothing to do
-      // With one Q buffer the store has to wait for this item's last score MMA, which is only
-      // issued once the softmax has reached the last tile: it then happens after the tile loop.
-      auto q_step = [&](bool item_done) -> bool {
-        if (q_stage == 0) {
-          Inext = make_item(e_next, idx_next);
-          q_load(Inext);
-          q_stage = 1;
-        } else if (q_stage == 1) {
-          if (Cfg::kQBufs == 2) {
-            const uint32_t nb = (qc + 1) & 1;
-            if (qc >= 1 && !warp_wait(&bars->q_empty[nb], ((qc - 1) >> 1) & 1, 3)) return false;
-            q_store(Inext, nb);
-            q_stage = 2;
-          } else if (item_done) {
-            if (!warp_wait(&bars->q_empty[0], qc & 1, 3)) return false;
-            q_store(Inext, 0);
-            q_stage = 2;
-          }
-        }
-        return true;
-      };
       const bool valid_row = row < I.R;
       float m_ref = -INFINITY, l_sum = 0.f;     // m_ref is the same in all four quadrants of a row
       const int limit = I.L - I.m + row / p.G;  // last visible token of this row
@@ -565,10 +527,9 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->p_full[b]);
         if (pend.valid) ok = run_epilogue();  // previous item (its sL became visible at this tile's barrier)
-        if (ok) ok = q_step(false);
       }
-      while (ok && q_stage < 2) ok = q_step(true);
       if (!ok) break;
+      if (idx_next >= 0) Inext = make_item(e_next, idx_next);
 
       // ---- the item's epilogue is deferred: it runs after the first tile of the next item, when
       // the last PV has long completed, so the softmax never idles at an item boundary

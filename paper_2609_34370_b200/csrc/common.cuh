@@ -140,6 +140,7 @@ struct AttnParams {
   float *part_o;           // [slot][rows_cap][D]
   float2 *part_ml;         // [slot][rows_cap]  (m in log2 domain, l)
   int32_t rows_cap;        // G * max_q_len
+  int32_t q_box_rows;      // query positions one Q box of the tensor-core kernel fetches (<= max_q_len)
   int32_t *dev_status;
   long long *prof;         // optional per-CTA cycle counters (profiling builds only), else NULL
 };

@@ -33,12 +33,14 @@ __device__ __forceinline__ int block_exclusive_scan_1024(int v, int *scratch, in
 }
 
 constexpr int kPlanMaxCta = 256;  // ranges the planner can cut the tile axis into
-// Cost of a pair on the axis the cuts are placed on, in quarter tiles: its tiles plus a fixed part
-// that is larger for short pairs, whose tiles do not overlap with anything.  Fitted to per-CTA run
-// times of the attention kernel on the Llama-3-8B, Llama-3-70B and mixed-length shapes: 0.3-0.4
-// tile times per entry, 0.65 for pairs of 3-6 tiles, 1.1-1.6 for pairs of one or two tiles.
-constexpr int kCostPerTile = 4;
-__device__ __forceinline__ int plan_entry_cost(int tiles) { return tiles <= 2 ? 6 : tiles <= 6 ? 3 : 1; }
+// Cost of a pair on the axis the cuts are placed on, in eighths of a tile: its tiles plus a fixed
+// part per work entry (the entry's epilogue and the pipeline's restart on a new set of query rows),
+// a little larger for pairs of one or two tiles, which leave nothing to overlap it with.  Fitted
+// to per-CTA run times of the attention kernel on the Llama-3-8B, Llama-3-70B and mixed-length
+// shapes, whose ranges hold 2 to 32 entries: 1.51 us per tile and 0.65 us per entry on all three
+// (0.43 tile times), pairs of one or two tiles 0.3 tile times more.
+constexpr int kCostPerTile = 8;
+__device__ __forceinline__ int plan_entry_cost(int tiles) { return tiles <= 2 ? 5 : 3; }
 
 // One block.  Validates each request's (k+1, L, page count), cuts the tile axis of the valid
 // requests' (request, kv head) pairs into n_cta ranges of equal length, lays out partial-result

@@ -230,6 +230,21 @@ static bool make_pool_map(CUtensorMap *map, const void *pool, const spx_attn_arg
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 3-D bf16 view of the query rows [TQ, Hq, D]: one box = 64 columns x the G heads of one kv-head x
+// `rows` consecutive query positions, which lands in shared memory as the packed rows j*G + h of a
+// work entry, 128 bytes each, 128-byte swizzle: the K-major A operand of the score MMA.
+static bool make_q_map(CUtensorMap *map, const spx_attn_args_t *a, int rows) {
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) return false;
+  const cuuint64_t D = a->head_dim, H = a->num_q_heads, G = a->num_q_heads / a->num_kv_heads;
+  cuuint64_t dims[3] = {D, H, (cuuint64_t)a->total_q};
+  cuuint64_t strides[2] = {D * 2, H * D * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)rows}, estr[3] = {1, 1, 1};
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(a->q), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // The tensor-core kernel handles bf16 pools whose pages hold at least one 8-row swizzle atom.
 static bool use_tensor_core_path(const spx_attn_args_t *a) {
   return a->kv_dtype == SPX_BF16 && a->page_size >= 8 && a->num_pages > 0 && a->kv_stride_page > 0 &&
@@ -251,8 +266,8 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 }
 
 template <int D, int MROWS>
-static cudaError_t launch_tc4(const CUtensorMap &kmap, const CUtensorMap &vmap, const AttnParams &p, int num_sms,
-                              cudaStream_t stream) {
+static cudaError_t launch_tc4(const CUtensorMap &kmap, const CUtensorMap &vmap, const CUtensorMap &qmap, const AttnParams &p,
+                              int num_sms, cudaStream_t stream) {
   using Cfg = Tc4Cfg<D, MROWS>;
   auto kernel = attn_tc4_kernel<D, MROWS>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
@@ -260,7 +275,7 @@ static cudaError_t launch_tc4(const CUtensorMap &kmap, const CUtensorMap &vmap, 
   // (A programmatic dependent launch behind the planner was measured: no gain, the early-resident
   // CTAs only take registers away from the sampling kernels that run beside them.)
   if (t_ev_start) cudaEventRecord(t_ev_start, stream);
-  kernel<<<num_sms, kTcThreads, Cfg::kSmemBytes, stream>>>(kmap, vmap, p);
+  kernel<<<num_sms, kTcThreads, Cfg::kSmemBytes, stream>>>(kmap, vmap, qmap, p);
   if (t_ev_stop) cudaEventRecord(t_ev_stop, stream);
   ++t_launches;
   return cudaGetLastError();
@@ -336,11 +351,16 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
     CUtensorMap kmap, vmap;
     if (!make_pool_map(&kmap, a->k_cache, a, p.head_inner) || !make_pool_map(&vmap, a->v_cache, a, p.head_inner))
       return SPX_ERR_CUDA;
-    if (p.rows_cap <= 32)
-      e = p.D == 128 ? launch_tc4<128, 32>(kmap, vmap, p, sms, stream) : launch_tc4<64, 32>(kmap, vmap, p, sms, stream);
-    else if (p.rows_cap <= 64)
-      e = p.D == 128 ? launch_tc4<128, 64>(kmap, vmap, p, sms, stream) : launch_tc4<64, 64>(kmap, vmap, p, sms, stream);
-    else
+    if (p.rows_cap <= 64) {
+      // the packed query rows of a work entry arrive by one box pair of a 3-D map over Q
+      CUtensorMap qmap;
+      p.q_box_rows = p.max_q_len < p.total_q ? p.max_q_len : p.total_q;
+      if (!make_q_map(&qmap, a, p.q_box_rows)) return SPX_ERR_CUDA;
+      if (p.rows_cap <= 32)
+        e = p.D == 128 ? launch_tc4<128, 32>(kmap, vmap, qmap, p, sms, stream) : launch_tc4<64, 32>(kmap, vmap, qmap, p, sms, stream);
+      else
+        e = p.D == 128 ? launch_tc4<128, 64>(kmap, vmap, qmap, p, sms, stream) : launch_tc4<64, 64>(kmap, vmap, qmap, p, sms, stream);
+    } else
       e = p.D == 128 ? launch_tc<128, 128>(kmap, vmap, p, sms, stream) : launch_tc<64, 128>(kmap, vmap, p, sms, stream);
   } else {
     const SimtSmem lay(p.rows_cap, p.D);
