@@ -414,6 +414,20 @@ spx_status_t spx_plan_layout(const spx_attn_args_t *attn, int64_t *out);
  */
 spx_status_t spx_debug_timeline(uint64_t *host_out, int64_t capacity, int32_t *kernels, int32_t *ctas_per_kernel);
 
+/*
+ * Test aid of wait-test builds of the library (compiled with -DSPX_WAIT_TEST=1 and a small
+ * -DSPX_WAIT_LIMIT_CYCLES; the regular build returns SPX_ERR_UNSUPPORTED).  Every spin on a
+ * barrier in the library's kernels has a cycle limit, after which the waiting role raises
+ * SPX_DEV_TIMEOUT in *dev_status, sets its CTA's abort flag and returns, so that a lost signal ends
+ * in an error status and not in a hung device.  This call launches one block of four warps in
+ * which the three wait helpers (attention, logits ring, LM head) each wait on a barrier nothing
+ * arrives at.  report (device, int32 [11]): [0..3] 2 = the role's wait gave up (1 would mean it
+ * was satisfied); [4..7] cycles each role waited; [8..10] the three abort flags afterwards.
+ * Role 1 shares its abort flag with role 0 and leaves through it or through its own limit.
+ * Enqueues only; nothing faults, the context stays usable.
+ */
+spx_status_t spx_debug_wait_expiry(int32_t *report, int32_t *dev_status, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

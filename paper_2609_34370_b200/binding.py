@@ -16,7 +16,7 @@ BF16, F32 = 0, 1
 
 EXPORTS = ("spx_workspace_size", "spx_verify_attention", "spx_rejection_sample", "spx_verify_step",
            "spx_host_step_arena_size", "spx_verify_step_host", "spx_status_string", "spx_last_launch_count",
-           "spx_set_timing_events", "spx_plan_layout", "spx_debug_timeline", "spx_rejection_sample_static", "spx_kv_append", "spx_kv_rollback",
+           "spx_set_timing_events", "spx_plan_layout", "spx_debug_timeline", "spx_debug_wait_expiry", "spx_rejection_sample_static", "spx_kv_append", "spx_kv_rollback",
            "spx_draft_confidence_workspace", "spx_draft_confidence", "spx_select_speculation",
            "spx_lookahead_memory", "spx_sp_effective_batch", "spx_selective_batch", "spx_selective_effective_batch",
            "spx_delay_gain", "spx_lm_head")
@@ -117,6 +117,8 @@ def load_library():
         lib.spx_debug_timeline.restype = C.c_int
         lib.spx_debug_timeline.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         lib.spx_plan_layout.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
+        lib.spx_debug_wait_expiry.restype = C.c_int
+        lib.spx_debug_wait_expiry.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         lib.spx_rejection_sample_static.restype = C.c_int
         lib.spx_rejection_sample_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         lib.spx_kv_append.restype = C.c_int

@@ -8,6 +8,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 LIB_PATH = os.path.join(_PKG, "libspx.so")
 TIMELINE_LIB_PATH = os.path.join(_PKG, "libspx_timeline.so")
+WAIT_TEST_LIB_PATH = os.path.join(_PKG, "libspx_waittest.so")
 _SOURCES = [os.path.join(_PKG, "csrc", "spx_api.cu")]
 
 
@@ -44,6 +45,15 @@ def build_timeline(force: bool = False) -> str:
     if not force and os.path.exists(TIMELINE_LIB_PATH) and os.path.getmtime(TIMELINE_LIB_PATH) >= _newest_source_mtime():
         return TIMELINE_LIB_PATH
     return _compile(TIMELINE_LIB_PATH, defines=("SPX_TIMELINE=1",))
+
+
+def build_wait_test(force: bool = False) -> str:
+    """The same sources with every bounded wait limited to 100k cycles (about 50 us) and the kernel
+    behind spx_debug_wait_expiry compiled in (libspx_waittest.so).  Used by the timeout test only:
+    its production kernels would give up on ordinary memory latency."""
+    if not force and os.path.exists(WAIT_TEST_LIB_PATH) and os.path.getmtime(WAIT_TEST_LIB_PATH) >= _newest_source_mtime():
+        return WAIT_TEST_LIB_PATH
+    return _compile(WAIT_TEST_LIB_PATH, defines=("SPX_WAIT_TEST=1", "SPX_WAIT_LIMIT_CYCLES=100000"))
 
 
 if __name__ == "__main__":

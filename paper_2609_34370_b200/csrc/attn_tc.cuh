@@ -71,7 +71,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *b, uint32_t parity) {
                : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after ~2^31 cycles (about a second) or when another role aborted.
+// Bounded wait: gives up after kWaitLimitCycles (about a second) or when another role aborted.
 __device__ __forceinline__ bool mbar_wait(uint64_t *b, uint32_t parity, TcBarriers *bars, int32_t *dev_status) {
   if (mbar_try_wait(b, parity)) return true;
   const long long t0 = clock64();
@@ -79,7 +79,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *b, uint32_t parity, TcBarrie
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(b, parity)) return true;
     if (bars->abort) return false;
-    if (clock64() - t0 > (1ll << 31)) {
+    if (clock64() - t0 > kWaitLimitCycles) {
       bars->abort = 1;
       atomicOr(dev_status, SPX_DEV_TIMEOUT);
       return false;

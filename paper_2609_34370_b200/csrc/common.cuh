@@ -145,6 +145,18 @@ struct AttnParams {
   long long *prof;         // optional per-CTA cycle counters (profiling builds only), else NULL
 };
 
+// Every spin on a barrier in this library gives up after this many clock cycles (about a second at
+// the default), raises SPX_DEV_TIMEOUT and makes the other roles of its CTA leave too.  The
+// wait-test build (build.py: build_wait_test) compiles a limit of some tens of microseconds and a
+// small kernel that lets each of the wait helpers run out on purpose (spx_debug_wait_expiry).
+#ifndef SPX_WAIT_LIMIT_CYCLES
+#define SPX_WAIT_LIMIT_CYCLES (1ll << 31)
+#endif
+constexpr long long kWaitLimitCycles = SPX_WAIT_LIMIT_CYCLES;
+#ifndef SPX_WAIT_TEST
+#define SPX_WAIT_TEST 0
+#endif
+
 #ifndef SPX_PROFILE
 #define SPX_PROFILE 0
 #endif

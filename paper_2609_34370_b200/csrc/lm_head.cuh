@@ -51,7 +51,7 @@ __device__ __forceinline__ bool lm_wait(uint64_t *b, uint32_t parity, LmBarriers
     for (int i = 0; i < 64; ++i)
       if (tc::mbar_try_wait(b, parity)) return true;
     if (bars->abort) return false;
-    if (clock64() - t0 > (1ll << 31)) {  // about a second
+    if (clock64() - t0 > kWaitLimitCycles) {  // about a second
       bars->abort = 1;
       atomicOr(dev_status, SPX_DEV_TIMEOUT);
       return false;

@@ -280,7 +280,7 @@ __device__ __forceinline__ bool ring_wait(uint64_t *bar, uint32_t parity, volati
       if (ok) return true;
     }
     if (*abort) return false;
-    if (clock64() - t0 > (1ll << 31)) {  // about a second: give up, report, let the others leave too
+    if (clock64() - t0 > kWaitLimitCycles) {  // about a second: give up, report, let the others leave too
       *abort = 1;
       atomicOr(dev_status, SPX_DEV_TIMEOUT);
       return false;

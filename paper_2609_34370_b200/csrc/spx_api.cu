@@ -18,6 +18,9 @@
 #include "plan.cuh"
 #include "sampler.cuh"
 #include "spx.h"
+#if SPX_WAIT_TEST
+#include "wait_test.cuh"
+#endif
 
 namespace spx {
 
@@ -927,6 +930,17 @@ spx_status_t spx_debug_timeline(uint64_t *host_out, int64_t capacity, int32_t *k
   return cudaMemcpyFromSymbol(host_out, g_timeline, (size_t)need * sizeof(uint64_t)) == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
 #else
   (void)host_out; (void)capacity;
+  return SPX_ERR_UNSUPPORTED;
+#endif
+}
+
+spx_status_t spx_debug_wait_expiry(int32_t *report, int32_t *dev_status, void *cuda_stream) {
+#if SPX_WAIT_TEST
+  if (!report || !dev_status) return SPX_ERR_INVALID_ARG;
+  wait_expiry_kernel<<<1, 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(report, dev_status);
+  return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
+#else
+  (void)report; (void)dev_status; (void)cuda_stream;
   return SPX_ERR_UNSUPPORTED;
 #endif
 }
