@@ -266,7 +266,7 @@ def time_extras(spx, binding, spec, b, attn_args, dev, iters: int = 200):
     H = torch.randn((b.total_q, hid), generator=gh, device=dev).to(torch.bfloat16)
     Wt = (torch.randn((spec.vocab, hid), generator=gh, device=dev) * (3.0 / hid ** 0.5)).to(torch.bfloat16)
     lg = torch.empty((b.total_q, spec.vocab + (-spec.vocab) % 8), dtype=torch.bfloat16, device=dev)
-    ts = torch.empty((b.total_q, (spec.vocab + 255) // 256, 2), dtype=torch.float32, device=dev)
+    ts = torch.empty((b.total_q, (spec.vocab + binding.LM_TILE_COLS - 1) // binding.LM_TILE_COLS, 2), dtype=torch.float32, device=dev)
     lm_iters = max(3, min(iters, 20))
     saved, iters = iters, lm_iters
     out["lm_head_us"] = timed(lambda: spx.lm_head(H, Wt, logits=lg, tile_stats=ts, status=status))

@@ -310,8 +310,8 @@ double spx_delay_gain(double iterations, int32_t n_evictions, double pdr, double
  * stored at logits[m * logits_row_stride + v].  hidden is [rows, hidden_dim] and weight is
  * [vocab, hidden_dim], both row-major and dense; all device pointers, 16-byte aligned;
  * hidden_dim and logits_row_stride multiples of 8.  tile_stats (optional) receives, for every row
- * and every block of 256 vocabulary columns, (max * log2 e, sum_v 2^((x_v - max) log2 e)) of the
- * values AS STORED: [rows][ceil(vocab / 256)] pairs of floats.  Passed as
+ * and every block of 128 vocabulary columns, (max * log2 e, sum_v 2^((x_v - max) log2 e)) of the
+ * values AS STORED: [rows][ceil(vocab / 128)] pairs of floats.  Passed as
  * spx_sample_args_t.target_tile_stats they replace the sampling half's own read of the target
  * logits for its statistics (temperature 1, no filters; ignored otherwise).
  * Errors: SPX_ERR_INVALID_ARG / SPX_ERR_UNSUPPORTED for bad shapes or alignment; a bounded wait
@@ -323,7 +323,7 @@ typedef struct {
   const void *weight;          /* [vocab, hidden_dim] bf16                                     */
   void *logits;                /* [rows, logits_row_stride] bf16, written                      */
   int64_t logits_row_stride;   /* elements                                                     */
-  float *tile_stats;           /* optional [rows][ceil(vocab/256)][2], written                 */
+  float *tile_stats;           /* optional [rows][ceil(vocab/128)][2], written                 */
 } spx_lm_head_args_t;
 
 spx_status_t spx_lm_head(const spx_lm_head_args_t *args, int32_t *dev_status, void *cuda_stream);

@@ -491,7 +491,7 @@ def delay_gain(iterations: float, pdr: float, running: float, i_delay: float, i_
     return float(load_library().spx_delay_gain(float(iterations), len(i_wait), float(pdr), float(running), float(i_delay), w))
 
 
-LM_TILE_COLS = 256
+LM_TILE_COLS = 128
 
 
 def lm_head(hidden, weight, logits: Optional[torch.Tensor] = None, want_stats: bool = True,

@@ -426,8 +426,8 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
         // the target rows' statistics came out of the LM-head epilogue, per 256-column tile: fold them
         // into sub-segments; only the draft rows are read here
         const int n = p.first_row * p.nsub;
-        lm_stats_merge_kernel<<<(n + 255) / 256, 256, 0, stream>>>(tile_stats, p.first_row, (p.vocab + kLmBN - 1) / kLmBN, p.nsub,
-                                                                  kSubElems / kLmBN, p.seg_stats);
+        lm_stats_merge_kernel<<<(n + 255) / 256, 256, 0, stream>>>(tile_stats, p.first_row, (p.vocab + kLmStatCols - 1) / kLmStatCols, p.nsub,
+                                                                  kSubElems / kLmStatCols, p.seg_stats);
         ++t_launches;
       }
       if (n_chunks > 0)
@@ -847,23 +847,39 @@ spx_status_t spx_lm_head(const spx_lm_head_args_t *a, int32_t *dev_status, void 
   if (((uintptr_t)a->hidden | (uintptr_t)a->weight | (uintptr_t)a->logits) & 15) return SPX_ERR_INVALID_ARG;
   DeviceInfo info;
   if (!get_device_info(&info)) return SPX_ERR_CUDA;
-  CUtensorMap hmap, wmap;
-  if (!make_matrix_map(&hmap, a->hidden, a->rows, a->hidden_dim, kLmBM) ||
-      !make_matrix_map(&wmap, a->weight, a->vocab, a->hidden_dim, kLmBN))
-    return SPX_ERR_CUDA;
   LmParams p{};
   p.M = a->rows; p.K = a->hidden_dim; p.V = a->vocab;
-  p.m_tiles = (a->rows + kLmBM - 1) / kLmBM;
-  p.n_tiles = (a->vocab + kLmBN - 1) / kLmBN;
+  // the rows are cut into equal token tiles of at most 512 (the TMEM columns); a tile of more than
+  // 256 tokens is covered by two MMAs per k-step and has one accumulator instead of two in rotation
+  p.tok_tiles = (a->rows + kLmMaxTileTok - 1) / kLmMaxTileTok;
+  const int per_tile = (a->rows + p.tok_tiles - 1) / p.tok_tiles;
+  p.n_sub = per_tile > kLmMaxNT ? 2 : 1;
+  p.NT = ((per_tile + p.n_sub - 1) / p.n_sub + 31) / 32 * 32;
+  p.tile_tok = p.n_sub * p.NT;
+  p.n_buf = p.tile_tok <= kLmMaxNT ? 2 : 1;
+  p.stage_bytes = (kLmABytes + p.n_sub * (p.NT / 2) * kLmBK * 2 + 1023) / 1024 * 1024;
+  p.n_stages = kLmRingBytes / p.stage_bytes < kLmMaxStages ? kLmRingBytes / p.stage_bytes : kLmMaxStages;
+  p.v_tiles = (a->vocab + 2 * kLmVB - 1) / (2 * kLmVB);
   p.k_blocks = (a->hidden_dim + kLmBK - 1) / kLmBK;
+  p.stat_tiles = (a->vocab + kLmStatCols - 1) / kLmStatCols;
   p.logits = static_cast<__nv_bfloat16 *>(a->logits);
   p.row_stride = a->logits_row_stride;
   p.tile_stats = reinterpret_cast<float2 *>(a->tile_stats);
   p.dev_status = dev_status;
+  CUtensorMap hmap, wmap;
+  if (!make_matrix_map(&hmap, a->hidden, a->rows, a->hidden_dim, p.NT / 2) ||
+      !make_matrix_map(&wmap, a->weight, a->vocab, a->hidden_dim, kLmVB))
+    return SPX_ERR_CUDA;
   if (cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLmSmemBytes) != cudaSuccess) return SPX_ERR_CUDA;
-  const long long tiles = (long long)p.m_tiles * p.n_tiles;
-  const int grid = tiles < info.num_sms ? (int)tiles : info.num_sms;
-  lm_head_kernel<<<grid, kLmThreads, kLmSmemBytes, static_cast<cudaStream_t>(cuda_stream)>>>(hmap, wmap, p);
+  // one resident CTA pair per two SMs of a GPC (a GPC with an odd SM count leaves one SM out)
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(info.num_sms / 2 * 2); cfg.blockDim = dim3(kLmThreads); cfg.dynamicSmemBytes = kLmSmemBytes;
+  cfg.stream = static_cast<cudaStream_t>(cuda_stream);
+  int max_pairs = 0;
+  if (cudaOccupancyMaxActiveClusters(&max_pairs, lm_head_kernel, &cfg) != cudaSuccess || max_pairs < 1) return SPX_ERR_CUDA;
+  const long long tiles = (long long)p.v_tiles * p.tok_tiles;
+  const int pairs = tiles < max_pairs ? (int)tiles : max_pairs;
+  lm_head_kernel<<<2 * pairs, kLmThreads, kLmSmemBytes, static_cast<cudaStream_t>(cuda_stream)>>>(hmap, wmap, p);
   ++t_launches;
   return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
 }

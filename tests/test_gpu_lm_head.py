@@ -11,6 +11,7 @@ import torch
 
 import oracle
 import paper_2609_34370_b200 as spx
+from paper_2609_34370_b200 import binding
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -34,7 +35,7 @@ def _check_logits(H, W, cols=None):
     return logits, stats
 
 
-@pytest.mark.parametrize("M,K,V", [(1, 64, 256), (7, 72, 100), (128, 512, 1024), (200, 520, 1000), (384, 1024, 5000)])
+@pytest.mark.parametrize("M,K,V", [(1, 64, 256), (7, 72, 100), (128, 512, 1024), (200, 520, 1000), (384, 1024, 5000), (300, 256, 700), (520, 128, 900)])
 def test_small_shapes_match_oracle(M, K, V):
     g = torch.Generator().manual_seed(M + K + V)
     H = torch.randn(M, K, generator=g).to(torch.bfloat16)
@@ -42,9 +43,11 @@ def test_small_shapes_match_oracle(M, K, V):
     logits, stats = _check_logits(H, W)
     # the statistics describe the stored values: recompute them from the same launch's logits on the host
     x = logits[:, :V].float().cpu().double()
-    n_tiles = (V + 255) // 256
+    cols = binding.LM_TILE_COLS
+    n_tiles = (V + cols - 1) // cols
+    assert stats.shape[1] == n_tiles
     for t in range(n_tiles):
-        blk = x[:, t * 256:min(V, (t + 1) * 256)]
+        blk = x[:, t * cols:min(V, (t + 1) * cols)]
         mx = blk.max(dim=1).values
         s = torch.exp(blk - mx[:, None]).sum(dim=1)
         assert torch.allclose(stats[:, t, 0].cpu().double(), mx * 1.4426950408889634, rtol=1e-6, atol=1e-6)
