@@ -33,9 +33,13 @@ METRIC = "verified_tokens_per_s"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one verify-attention launch, from the ncu
-# captures summarised under profiles/ (None until captured for that workload).
-NCU_TRAFFIC_BYTES = {"llama3-8b": 625.2e6}  # profiles/launch_list_llama3-8b.txt: 621.7 MB read + 3.5 MB written
+# dram__bytes_read.sum + dram__bytes_write.sum of one verify-attention launch, from the ncu captures
+# summarised in profiles/attention_traffic.txt (two launches each, averaged).  The mixed-length
+# workload was captured on its first 64 requests (1186.8 MB for 1176.1 MB of KV) and scaled to the
+# full batch by the KV bytes: the traffic beyond the KV bytes (query and output rows, block
+# tables, partials of split pairs) grows with the batch like the KV bytes do.
+NCU_TRAFFIC_BYTES = {"tiny-fp32": 0.621e6, "llama3-8b": 626.7e6, "llama3-70b": 761.1e6, "long-context": 2154.5e6,
+                     "selective-mix": 4309.4e6}
 
 
 def measured_peak():
