@@ -661,6 +661,57 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
     __syncthreads();
   };
 
+  // One level's histogram (count, mass per key byte) of the listed logits that match the prefix.
+  // The listed logits lie within a fraction of a logit unit of each other, so at the first levels
+  // all of them fall into one bin and at the later ones into a few dozen: 64-bit shared-memory
+  // atomics (a compare-and-swap loop) on so few addresses queue up for hundreds of cycles each.  The
+  // masses are therefore added as three 15-bit pieces with native 32-bit atomics (a list holds at
+  // most kFilterListCap logits: no piece overflows), into the first rows of the per-lane arrays,
+  // which are idle here; and a warp whose lanes all agree on the bin adds its 32 masses up with
+  // shuffles and issues one set of atomics.
+  auto level_hist_of_list = [&](int level, int shift, uint32_t prefix, uint32_t n_list) {
+    if (tid < 256) { s_cnt[tid] = 0; h_m0[tid] = 0; h_m1[tid] = 0; h_m2[tid] = 0; }
+    __syncthreads();
+    for (uint32_t i0 = (uint32_t)(tid & ~31); i0 < n_list; i0 += kFilterThreads) {   // warp-uniform bounds
+      const uint32_t i = i0 + lane;
+      bool use = i < n_list;
+      float x = 0.f;
+      uint32_t key = 0;
+      if (use) {
+        x = s_list[i];
+        key = order_key32(x);
+        use = level == 1 || (key >> (shift + 8)) == (prefix >> (shift + 8));
+      }
+      const uint32_t bin = use ? ((key >> shift) & 255u) : 0xffffffffu;
+      unsigned long long m = use ? mass_of(x) : 0ull;
+      uint32_t c = use ? 1u : 0u;
+      int same = 0;
+      __match_all_sync(0xffffffffu, bin, &same);
+      if (same) {
+        if (bin == 0xffffffffu) continue;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          m += __shfl_xor_sync(0xffffffffu, m, o);
+          c += __shfl_xor_sync(0xffffffffu, c, o);
+        }
+        if (lane == 0) {   // up to 32 masses: the pieces are cut from the sum, 20 bits suffice for the top one
+          atomicAdd(&s_cnt[bin], c);
+          atomicAdd(&h_m0[bin], (uint32_t)(m & 0x7fffull));
+          atomicAdd(&h_m1[bin], (uint32_t)((m >> 15) & 0x7fffull));
+          atomicAdd(&h_m2[bin], (uint32_t)(m >> 30));
+        }
+      } else if (use) {
+        atomicAdd(&s_cnt[bin], 1u);
+        atomicAdd(&h_m0[bin], (uint32_t)(m & 0x7fffull));
+        atomicAdd(&h_m1[bin], (uint32_t)((m >> 15) & 0x7fffull));
+        atomicAdd(&h_m2[bin], (uint32_t)(m >> 30));
+      }
+    }
+    __syncthreads();
+    if (tid < 256)
+      s_mass[tid] = (unsigned long long)h_m0[tid] + ((unsigned long long)h_m1[tid] << 15) + ((unsigned long long)h_m2[tid] << 30);
+  };
+
   // Exact key-byte levels over the n_list logits in s_list (every level narrows the key by one
   // byte; after the last the key is complete).  Returns the threshold key, *Z the mass at or above it.
   auto levels_over_list = [&](bool by_count, uint32_t need, double need_mass, uint32_t n_list, unsigned long long *Z) -> uint32_t {
@@ -670,14 +721,7 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
       const int shift = kKeyShift + 8 * (kLevels - level);
       if (tid < 256) { s_cnt[tid] = 0; s_mass[tid] = 0ull; }
       __syncthreads();
-      for (uint32_t i = tid; i < n_list; i += kFilterThreads) {
-        const float x = s_list[i];
-        const uint32_t key = order_key32(x);
-        if (level > 1 && (key >> (shift + 8)) != (prefix >> (shift + 8))) continue;
-        const uint32_t bin = (key >> shift) & 255u;
-        atomicAdd(&s_cnt[bin], 1u);
-        atomicAdd(&s_mass[bin], mass_of(x));
-      }
+      level_hist_of_list(level, shift, prefix, n_list);
       __syncthreads();
       pick(by_count, need, need_mass, above);
       prefix |= s_bin << shift;
@@ -804,7 +848,7 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
         atomicAdd(&s_mass[bin], mass_of(x));
       };
       if (listed) {
-        for (uint32_t i = tid; i < n_list; i += kFilterThreads) add(s_list[i]);
+        level_hist_of_list(level, shift, prefix, n_list);
       } else {
         sweep_row<T>(base, p.vocab, tid, [&](float x) { if (bin0_of(x) == b0) add(x); });
       }
