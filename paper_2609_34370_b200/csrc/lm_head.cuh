@@ -19,11 +19,14 @@
 //   warp 1      leader CTA only: MMA issuer (one lane) into the TMEM accumulator (two of them,
 //               alternating, when a tile has at most 256 tokens);
 //   warps 2-9   epilogue, two warps per TMEM lane quadrant taking alternate chunks of 32 tokens.
-//               A chunk comes out of the accumulator one vocabulary row per lane; a partial
-//               shuffle transpose hands every lane eight consecutive columns of four tokens,
-//               which it rounds to bf16, stores as 16-byte vectors (64 contiguous bytes per
-//               token and warp) and reduces - as stored - to (max, sum 2^((x - max) log2 e));
-//               the four quadrants' pairs of a token are merged through shared memory.
+//               A warp first reads its chunks out of the accumulator (one vocabulary row per
+//               lane), rounds them to bf16 pairs that stay in registers and hands the accumulator
+//               back: a tile of more than 256 tokens has no second accumulator, and the next
+//               tile's MMAs wait for exactly this.  Then, beside those MMAs, a partial transpose
+//               across the warp hands every lane eight consecutive columns of four tokens, which
+//               it stores as 16-byte vectors (64 contiguous bytes per token and warp) and
+//               reduces - as stored - to (max, sum 2^((x - max) log2 e)); the four quadrants'
+//               pairs of a token are merged through shared memory.
 // The MMA's completions are committed twice, once to the leader's barrier and once to the peer's
 // (a commit takes a shared::cluster address); the epilogue's "accumulator drained" signals of the
 // peer are plain remote mbarrier arrivals on the leader's barrier.  No copy and no commit is sent
@@ -157,26 +160,38 @@ __device__ __forceinline__ void mma_pair_commit(uint32_t bar_cluster) {
 __host__ __device__ constexpr uint32_t idesc_pair(uint32_t n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((256u >> 4) << 24);
 }
-// Partial transpose across the warp: exchanges the low three bits of the lane index with the low
-// three bits of the register index (three butterfly steps of 16 shuffles).  Before, lane l holds
-// x[t] = value (row l, column t); after, lane (a, b) = 8 a + b holds x[8 i + v] = value (row 8 a + v,
-// column 8 i + b): eight consecutive rows of one column per group of eight registers.
-__device__ __forceinline__ void warp_transpose8(float (&x)[32], int lane) {
+// Partial transpose across the warp of a chunk held as bf16 pairs.  Before, lane l (a row of the
+// accumulator) holds u[i] = (columns 2 i, 2 i + 1 of row l); the column's bit 0 sits in the half,
+// its bits 1-4 in the register index, the row's bits 0-4 in the lane index.  Three exchanges swap
+// the column's bits 0-2 with the row's bits 0-2: halves against lane bit 0 (16 shuffles and byte
+// permutes), register bits 0 and 1 against lane bits 1 and 2 (8 shuffles each).  After, lane
+// (a, b) = 8 a + b holds u[4 g + i] = (rows 8 a + 2 i, 8 a + 2 i + 1 of column 8 g + b): eight
+// consecutive rows of one column per group of four registers.
+__device__ __forceinline__ void warp_transpose_pairs(uint32_t (&u)[16], int lane) {
+  const bool odd = (lane & 1) != 0;
 #pragma unroll
-  for (int o = 4; o >= 1; o >>= 1) {
-    const bool upper = (lane & o) != 0;
+  for (int i = 0; i < 16; ++i) {
+    const uint32_t o = __shfl_xor_sync(0xffffffffu, u[i], 1);
+    u[i] = odd ? __byte_perm(o, u[i], 0x7632) : __byte_perm(u[i], o, 0x5410);
+  }
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
+  for (int o = 1; o <= 2; o <<= 1) {
+    const bool upper = (lane & (2 * o)) != 0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
       if ((j & o) == 0) {
-        const float send = upper ? x[j] : x[j + o];
-        const float recv = __shfl_xor_sync(0xffffffffu, send, o);
-        if (upper) x[j] = recv; else x[j + o] = recv;
+        const uint32_t send = upper ? u[j] : u[j + o];
+        const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 2 * o);
+        if (upper) u[j] = recv; else u[j + o] = recv;
       }
     }
   }
 }
 }  // namespace lm
 
+// kCh: chunks of 32 tokens an epilogue warp holds at most (tile_tok <= 64 kCh); the rounded
+// accumulator stays in 16 kCh registers per thread while it is stored.
+template <int kCh>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kLmThreads, 1)
 lm_head_kernel(const __grid_constant__ CUtensorMap hmap, const __grid_constant__ CUtensorMap wmap, LmParams p) {
   using namespace tc;
@@ -302,38 +317,50 @@ lm_head_kernel(const __grid_constant__ CUtensorMap hmap, const __grid_constant__
       const uint32_t taddr = tmem + b * kLmMaxNT + ((uint32_t)(q * 32) << 16);
       const int vrow0 = vt * 2 * kLmVB + (int)rank * kLmVB + q * 32;  // first vocabulary index of this warp
       const int v_left = p.V - vrow0;                                  // valid columns among the warp's 32 (may be <= 0)
-      // Per chunk of 32 tokens: the accumulator comes out one vocabulary row per lane.  A partial
-      // transpose across the warp leaves lane (a, b) with eight consecutive vocabulary columns
-      // 8a..8a+7 of the tokens b, 8 + b, 16 + b, 24 + b: 16 bytes of a logits row per token, so that
-      // one store instruction writes 64 contiguous bytes of eight rows; the statistics of a
-      // token's 32 values are finished by two shuffle steps across its four lanes.
-      const int va = lane >> 3, tb = lane & 7;
-      const int v_mine = v_left - 8 * va;   // valid columns among this lane's eight (may be <= 0)
-#pragma unroll 1
-      for (int c = c_first; c < n_chunks; c += kLmEpiWarps / 4) {
-        float x[32];
-        {
+      // The accumulator is drained first: per chunk of 32 tokens it comes out one vocabulary row
+      // per lane and is rounded to bf16 pairs that stay in registers, so that the MMAs of the next
+      // tile start while this one is still being transposed, stored and reduced.
+      uint32_t u[kCh][16];
+#pragma unroll
+      for (int ci = 0; ci < kCh; ++ci) {
+        const int c = c_first + ci * (kLmEpiWarps / 4);
+        if (c < n_chunks) {
           uint32_t r[32];
           tmem_ld32(taddr + c * 32, r);
           wait_ld();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) x[i] = __uint_as_float(r[i]);
+          for (int i = 0; i < 16; ++i) u[ci][i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
         }
-        lm::warp_transpose8(x, lane);
-        uint32_t pk[4][4];
+      }
+      fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if (leader) mbar_arrive(&bars->acc_empty[b]);
+        else lm::remote_arrive(&bars->acc_empty[b], 0);
+      }
+      // Per chunk: a partial transpose across the warp leaves lane (a, b) with eight consecutive
+      // vocabulary columns 8a..8a+7 of the tokens b, 8 + b, 16 + b, 24 + b: 16 bytes of a logits row
+      // per token, so that one store instruction writes 64 contiguous bytes of eight rows; the
+      // statistics of a token's 32 values are finished by two shuffle steps across its four lanes.
+      const int va = lane >> 3, tb = lane & 7;
+      const int v_mine = v_left - 8 * va;   // valid columns among this lane's eight (may be <= 0)
+#pragma unroll
+      for (int ci = 0; ci < kCh; ++ci) {
+        const int c = c_first + ci * (kLmEpiWarps / 4);
+        if (c >= n_chunks) break;
+        lm::warp_transpose_pairs(u[ci], lane);
+        uint32_t (&pk)[16] = u[ci];
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           const int tok = tok0 + c * 32 + g * 8 + tb;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) pk[g][i] = pack_bf16(x[g * 8 + 2 * i], x[g * 8 + 2 * i + 1]);
           if (tok < p.M && v_mine > 0) {
             __nv_bfloat16 *dst = p.logits + (int64_t)tok * p.row_stride + vrow0 + 8 * va;
             if (v_mine >= 8) {
-              *reinterpret_cast<uint4 *>(dst) = make_uint4(pk[g][0], pk[g][1], pk[g][2], pk[g][3]);
+              *reinterpret_cast<uint4 *>(dst) = make_uint4(pk[g * 4], pk[g * 4 + 1], pk[g * 4 + 2], pk[g * 4 + 3]);
             } else {
 #pragma unroll
               for (int i = 0; i < 8; ++i)
-                if (i < v_mine) dst[i] = __ushort_as_bfloat16((unsigned short)((i & 1) ? (pk[g][i >> 1] >> 16) : (pk[g][i >> 1] & 0xffffu)));
+                if (i < v_mine) dst[i] = __ushort_as_bfloat16((unsigned short)((i & 1) ? (pk[g * 4 + (i >> 1)] >> 16) : (pk[g * 4 + (i >> 1)] & 0xffffu)));
             }
           }
         }
@@ -346,8 +373,8 @@ lm_head_kernel(const __grid_constant__ CUtensorMap hmap, const __grid_constant__
             mx[g] = -INFINITY;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              if (2 * i < v_mine) mx[g] = fmaxf(mx[g], __uint_as_float(pk[g][i] << 16));
-              if (2 * i + 1 < v_mine) mx[g] = fmaxf(mx[g], __uint_as_float(pk[g][i] & 0xffff0000u));
+              if (2 * i < v_mine) mx[g] = fmaxf(mx[g], __uint_as_float(pk[g * 4 + i] << 16));
+              if (2 * i + 1 < v_mine) mx[g] = fmaxf(mx[g], __uint_as_float(pk[g * 4 + i] & 0xffff0000u));
             }
           }
 #pragma unroll
@@ -361,8 +388,8 @@ lm_head_kernel(const __grid_constant__ CUtensorMap hmap, const __grid_constant__
             sum[g] = 0.f;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              if (2 * i < v_mine) sum[g] += fast_exp2(fmaf(__uint_as_float(pk[g][i] << 16), kLog2e, -m2));
-              if (2 * i + 1 < v_mine) sum[g] += fast_exp2(fmaf(__uint_as_float(pk[g][i] & 0xffff0000u), kLog2e, -m2));
+              if (2 * i < v_mine) sum[g] += fast_exp2(fmaf(__uint_as_float(pk[g * 4 + i] << 16), kLog2e, -m2));
+              if (2 * i + 1 < v_mine) sum[g] += fast_exp2(fmaf(__uint_as_float(pk[g * 4 + i] & 0xffff0000u), kLog2e, -m2));
             }
           }
 #pragma unroll
@@ -374,13 +401,6 @@ lm_head_kernel(const __grid_constant__ CUtensorMap hmap, const __grid_constant__
             for (int g = 0; g < 4; ++g) s_ms[(c * 4 + q) * 32 + g * 8 + tb] = make_float2(mx[g] * kLog2e, sum[g]);
           }
         }
-      }
-      // the accumulator has been read for the last time: hand it back to the leader's MMA issuer
-      fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        if (leader) mbar_arrive(&bars->acc_empty[b]);
-        else lm::remote_arrive(&bars->acc_empty[b], 0);
       }
       if (p.tile_stats) {
         ok = epi_sync();

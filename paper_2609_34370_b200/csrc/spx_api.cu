@@ -870,16 +870,19 @@ spx_status_t spx_lm_head(const spx_lm_head_args_t *a, int32_t *dev_status, void 
   if (!make_matrix_map(&hmap, a->hidden, a->rows, a->hidden_dim, p.NT / 2) ||
       !make_matrix_map(&wmap, a->weight, a->vocab, a->hidden_dim, kLmVB))
     return SPX_ERR_CUDA;
-  if (cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLmSmemBytes) != cudaSuccess) return SPX_ERR_CUDA;
+  // the epilogue keeps a tile's rounded accumulator in registers: 6 chunks of 32 tokens per warp for
+  // tiles of at most 384 tokens, 8 beyond
+  auto kernel = p.tile_tok <= 384 ? lm_head_kernel<6> : lm_head_kernel<8>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLmSmemBytes) != cudaSuccess) return SPX_ERR_CUDA;
   // one resident CTA pair per two SMs of a GPC (a GPC with an odd SM count leaves one SM out)
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(info.num_sms / 2 * 2); cfg.blockDim = dim3(kLmThreads); cfg.dynamicSmemBytes = kLmSmemBytes;
   cfg.stream = static_cast<cudaStream_t>(cuda_stream);
   int max_pairs = 0;
-  if (cudaOccupancyMaxActiveClusters(&max_pairs, lm_head_kernel, &cfg) != cudaSuccess || max_pairs < 1) return SPX_ERR_CUDA;
+  if (cudaOccupancyMaxActiveClusters(&max_pairs, kernel, &cfg) != cudaSuccess || max_pairs < 1) return SPX_ERR_CUDA;
   const long long tiles = (long long)p.v_tiles * p.tok_tiles;
   const int pairs = tiles < max_pairs ? (int)tiles : max_pairs;
-  lm_head_kernel<<<2 * pairs, kLmThreads, kLmSmemBytes, static_cast<cudaStream_t>(cuda_stream)>>>(hmap, wmap, p);
+  kernel<<<2 * pairs, kLmThreads, kLmSmemBytes, static_cast<cudaStream_t>(cuda_stream)>>>(hmap, wmap, p);
   ++t_launches;
   return cudaGetLastError() == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
 }
