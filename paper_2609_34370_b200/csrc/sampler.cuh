@@ -426,6 +426,11 @@ constexpr int kFilterWarps = kFilterThreads / 32;
 constexpr int kFilterListCap = 12288;
 constexpr float kMassScale = 17592186044416.f;  // 2^44
 constexpr int kFilterSmemBytes = 4 * 256 * 32 * 4 + 256 * (8 + 4) * 2 + kFilterListCap * 4 + 64;
+constexpr int kExactUnroll = 4;                                   // 16-byte loads per thread and round
+constexpr int kExactPerThread = 35;                               // odd: a thread's run of counters starts in its own bank
+constexpr int kExactBins = kFilterThreads * kExactPerThread;      // counters of the exact-value histogram (bf16 rows)
+constexpr int kExactListCap = (kFilterSmemBytes - kExactBins * 4) / 2;   // 16-bit distances of the occupied counters
+static_assert(kExactBins <= 65536 && kExactListCap >= 16384, "the exact-value histogram and its list reuse the general path's shared memory");
 
 // Calls f(x) for every element of a row; the block's threads stride over 16-byte vectors and keep
 // kFilterUnroll of them in flight.
@@ -570,6 +575,36 @@ __global__ void __launch_bounds__(kTopkThreads, 6) topk_list_kernel(SampleParams
   }
 }
 
+// Calls f_pair(w) for every aligned pair of bf16 logits of a row (one 32-bit word, the element of the
+// lower index in the low half) and f_one(x) for the elements of a ragged end.  Rounds of kUnroll
+// 16-byte loads per thread, predicated at the end of the row; the loads of the next round are in
+// flight while a round is processed (two register buffers in turn).
+template <int kUnroll, typename F, typename G>
+__device__ __forceinline__ void sweep_row_pairs(const __nv_bfloat16 *base, int vocab, int tid, F f_pair, G f_one) {
+  const int n_vec = vocab >> 3;
+  const uint4 *b4 = reinterpret_cast<const uint4 *>(base);
+  constexpr int kRound = kUnroll * kFilterThreads;
+  auto load = [&](uint4 (&raw)[kUnroll], int v0) {
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u)
+      if (v0 + u * kFilterThreads < n_vec) raw[u] = __ldg(b4 + v0 + u * kFilterThreads);
+  };
+  auto work = [&](const uint4 (&raw)[kUnroll], int v0) {
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u)
+      if (v0 + u * kFilterThreads < n_vec) { f_pair(raw[u].x); f_pair(raw[u].y); f_pair(raw[u].z); f_pair(raw[u].w); }
+  };
+  uint4 ra[kUnroll], rb[kUnroll];
+  load(ra, tid);
+  for (int v0 = tid; v0 < n_vec; v0 += 2 * kRound) {
+    load(rb, v0 + kRound);
+    work(ra, v0);
+    load(ra, v0 + 2 * kRound);
+    work(rb, v0 + kRound);
+  }
+  for (int i = (n_vec << 3) + tid; i < vocab; i += kFilterThreads) f_one(__bfloat162float(base[i]));
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SampleParams p) {
   extern __shared__ __align__(16) unsigned char fsm[];
@@ -586,35 +621,227 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
   __shared__ unsigned long long s_above_mass, s_bin_mass;
   const int row = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  {
-    const double z_in = p.row_z[row];
-    if (z_in == z_in) return;   // not pending (NaN): topk_list_kernel has settled this row
-  }
-  const int r = p.row_req[row];
+  // what the block needs of the row, fetched in two round trips instead of a chain of five: the
+  // loads that do not depend on the request first, all at once
+  const float2 *st = p.seg_stats + (int64_t)row * p.nsub;
+  const double z_in = __ldg(p.row_z + row);
+  const int r = __ldg(p.row_req + row);
+  const float scale = __ldg(p.row_scale + row);
+  float M = -INFINITY;   // the row maximum (scaled) out of the sub-segment statistics: every warp reduces them for itself
+  for (int j = lane; j < p.nsub; j += 32) M = fmaxf(M, __ldg(&st[j].x));
+  if (z_in == z_in) return;   // not pending (NaN): topk_list_kernel has settled this row
   if (r < 0) {
     if (tid == 0) { p.row_thresh[row] = 0; p.row_z[row] = -1.0; }
     return;
   }
   constexpr int kLevels = sizeof(T) == 2 ? 2 : 4;      // exact key bytes after level 0
   constexpr int kKeyShift = sizeof(T) == 2 ? 16 : 0;   // bf16: the low 16 bits of the fp32 key carry nothing
-  const int tk_raw = p.top_k ? p.top_k[r] : 0;
+  const int tk_raw = p.top_k ? __ldg(p.top_k + r) : 0;
+  const float tp = p.top_p ? __ldg(p.top_p + r) : 1.f;
+  if constexpr (sizeof(T) == 2) {
+    // the exact-value histogram below is cleared while those two are on their way
+    uint32_t *h = reinterpret_cast<uint32_t *>(fsm);
+    for (int i = tid; i < kExactBins; i += kFilterThreads) h[i] = 0;
+  }
   const bool use_k = tk_raw >= 1 && tk_raw < p.vocab;
-  const float tp = p.top_p ? p.top_p[r] : 1.f;
   const bool use_p = tp < 1.f;
-  const float scale = p.row_scale[row];
   const float inv_w = 8.f / scale;   // distance in log2 units -> eighths of a logit unit
   const T *base = row < p.total_q ? reinterpret_cast<const T *>(p.target) + (int64_t)row * p.row_stride
                                   : reinterpret_cast<const T *>(p.draft) + (int64_t)(row - p.total_q) * p.row_stride;
-  float M = -INFINITY;
-  {
-    const float2 *st = p.seg_stats + (int64_t)row * p.nsub;
-    for (int j = 0; j < p.nsub; ++j) M = fmaxf(M, st[j].x);
-  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
   auto bin0_of = [&](float x) -> uint32_t {
     const float d = fmaxf(fmaf(x, -scale, M), 0.f) * inv_w;
     return 255u - (uint32_t)fminf(d, 255.f);
   };
   auto mass_of = [&](float x) -> unsigned long long { return __float2ull_rn(fast_exp2(fmaf(x, scale, -M)) * kMassScale); };
+
+  // bf16 rows: one histogram of COUNTS over the exact values.  A bf16 logit has a 16-bit key, and the
+  // keys of a row lie within a few ten thousand steps below the key of its maximum (128 per binade:
+  // from 16 down through zero to -16 are 38 k keys), so one counter per key fits in shared memory.
+  // Equal values have equal masses, so the mass of a key is its count times the mass of its value -
+  // the same integer as the sum over its elements - and the thresholds follow from one scan over the
+  // counters in descending key order: no masses are added per element, no second sweep, no further
+  // levels.  A row with a value outside the counters' range (never seen with logits) takes the
+  // general path below.
+  if constexpr (sizeof(T) == 2) {
+    uint32_t *h = reinterpret_cast<uint32_t *>(fsm);   // [kExactBins], index = key distance below the reference
+    uint16_t *nzl = reinterpret_cast<uint16_t *>(fsm + kExactBins * 4);   // [kExactListCap] distances of the occupied counters
+    __shared__ uint32_t s_over, s_tail, s_dk, s_df, s_found, s_nn, s_tc, s_wc[kFilterWarps];
+    __shared__ unsigned long long s_wm[kFilterWarps], s_zk, s_zf, s_tm;
+    if (tid == 0) { s_over = 0; s_tail = 0; s_found = 0; }
+    // reference: a bf16 value at or above every value of the row (the maximum of the statistics is
+    // the row's largest logit times the scale, rounded)
+    uint32_t key_ref;
+    {
+      float xub = M / scale;
+      xub = xub >= 0.f ? xub * (1.f + 0x1p-20f) : xub * (1.f - 0x1p-20f);
+      const uint32_t fb = __float_as_uint(xub);
+      const uint32_t b16 = (fb & 0x80000000u) ? (fb >> 16) : ((fb + 0xffffu) >> 16);   // towards +inf
+      const uint32_t k = order_key32(__uint_as_float(b16 << 16)) >> 16;
+      key_ref = k < 0xffffu ? k + 1u : k;
+    }
+    __syncthreads();
+    // a value below the counters (masked tokens at -inf, typically) is harmless while it carries no
+    // mass and no threshold falls among such values; the lanes that get here together add once
+    auto below = [&](float x) {
+      const bool massless = (order_key32(x) >> 16) <= key_ref && mass_of(x) == 0ull;
+      const uint32_t act = __activemask();
+      const uint32_t zl = __ballot_sync(act, massless);
+      if (lane == __ffs(act) - 1) {
+        if (zl) atomicAdd(&s_tail, (uint32_t)__popc(zl));
+        if (zl != act) atomicAdd(&s_over, (uint32_t)__popc(act & ~zl));
+      }
+    };
+    // Two logits per step of integer arithmetic: the sign of each half spread over the half (one
+    // byte permute), the order key of both (one logic operation), both distances by one
+    // subtraction - the reference is at or above every value, so no half borrows from the other.
+    const uint32_t ref2 = key_ref * 0x10001u;
+    sweep_row_pairs<kExactUnroll>(reinterpret_cast<const __nv_bfloat16 *>(base), p.vocab, tid,
+        [&](uint32_t w) {
+          uint32_t sm;
+          asm("prmt.b32 %0, %1, 0, 0xBB99;" : "=r"(sm) : "r"(w));
+          const uint32_t d2 = ref2 - (w ^ (sm | 0x80008000u));
+          const uint32_t dl = d2 & 0xffffu, dh = d2 >> 16;
+          if (dl < (uint32_t)kExactBins) atomicAdd(&h[dl], 1u); else below(__uint_as_float(w << 16));
+          if (dh < (uint32_t)kExactBins) atomicAdd(&h[dh], 1u); else below(__uint_as_float(w & 0xffff0000u));
+        },
+        [&](float x) {
+          const uint32_t d = key_ref - (order_key32(x) >> 16);
+          if (d < (uint32_t)kExactBins) atomicAdd(&h[d], 1u); else below(x);
+        });
+    __syncthreads();
+    if (s_over == 0) {
+      auto value_of = [&](uint32_t d) -> float {
+        const uint32_t k = key_ref - d;
+        const uint32_t b16 = (k & 0x8000u) ? (k & 0x7fffu) : (~k & 0xffffu);
+        return __uint_as_float(b16 << 16);
+      };
+      // The occupied counters lie in two or three dense stretches of the key axis, so their keys
+      // are first written out as a list (descending): every thread counts the occupied counters
+      // of its own run, a scan gives it its place in the list, and then every thread takes an
+      // equal share of the LIST - masses are evaluated three or so per thread instead of a
+      // whole run by the few threads whose runs are occupied.
+      const uint32_t d0 = (uint32_t)tid * kExactPerThread;
+      static_assert(kExactPerThread % 5 == 0, "runs are read five counters at a time");
+      uint32_t nz_t = 0;
+#pragma unroll
+      for (int j = 0; j < kExactPerThread; ++j) nz_t += h[d0 + j] != 0u ? 1u : 0u;
+      // exclusive scan over the block: within the warps, then warp 0 over the warps' totals
+      uint32_t nzi = nz_t;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, nzi, o);
+        if (lane >= o) nzi += v;
+      }
+      if (lane == 31) s_wc[warp] = nzi;
+      __syncthreads();
+      if (warp == 0) {
+        const uint32_t v = s_wc[lane];
+        uint32_t vi = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t x = __shfl_up_sync(0xffffffffu, vi, o);
+          if (lane >= o) vi += x;
+        }
+        s_wc[lane] = vi - v;
+        if (lane == 31) s_nn = vi;
+      }
+      __syncthreads();
+      const uint32_t n_nz = s_nn;
+      if (n_nz >= 1u && n_nz <= (uint32_t)kExactListCap) {
+        uint32_t off = nzi - nz_t + s_wc[warp];
+        for (int j = 0; j < kExactPerThread; ++j)
+          if (h[d0 + j]) nzl[off++] = (uint16_t)(d0 + j);
+        __syncthreads();
+        const uint32_t per = (n_nz + kFilterThreads - 1) / kFilterThreads;
+        const uint32_t e0 = min((uint32_t)tid * per, n_nz), e1 = min(e0 + per, n_nz);
+        uint32_t c_t = 0;
+        unsigned long long m_t = 0ull;
+        for (uint32_t e = e0; e < e1; ++e) {
+          const uint32_t d = nzl[e], c = h[d];
+          c_t += c;
+          m_t += (unsigned long long)c * mass_of(value_of(d));
+        }
+        uint32_t ci = c_t;
+        unsigned long long mi = m_t;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t cn = __shfl_up_sync(0xffffffffu, ci, o);
+          const unsigned long long mn = __shfl_up_sync(0xffffffffu, mi, o);
+          if (lane >= o) { ci += cn; mi += mn; }
+        }
+        if (lane == 31) { s_wc[warp] = ci; s_wm[warp] = mi; }
+        __syncthreads();
+        if (warp == 0) {
+          const uint32_t v = s_wc[lane];
+          const unsigned long long w = s_wm[lane];
+          uint32_t vi = v;
+          unsigned long long wi = w;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t x = __shfl_up_sync(0xffffffffu, vi, o);
+            const unsigned long long y = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) { vi += x; wi += y; }
+          }
+          s_wc[lane] = vi - v;
+          s_wm[lane] = wi - w;
+          if (lane == 31) { s_tc = vi; s_tm = wi; }
+        }
+        __syncthreads();
+        const uint32_t ce = ci - c_t + s_wc[warp], total_c = s_tc;   // counts / masses of the keys above this thread's share
+        const unsigned long long me = mi - m_t + s_wm[warp], total = s_tm;
+        // a top-k cut among the tokens below the counters is left to the general path
+        if (!use_k || total_c >= (uint32_t)tk_raw) {
+          unsigned long long Zk = total;
+          if (use_k) {
+            if (ce < (uint32_t)tk_raw && ce + c_t >= (uint32_t)tk_raw) {   // exactly one thread
+              uint32_t cc = ce;
+              unsigned long long mm = me;
+              for (uint32_t e = e0; e < e1; ++e) {
+                const uint32_t d = nzl[e], c = h[d];
+                cc += c;
+                mm += (unsigned long long)c * mass_of(value_of(d));
+                if (cc >= (uint32_t)tk_raw) { s_dk = d; s_zk = mm; break; }
+              }
+            }
+            __syncthreads();
+            Zk = s_zk;
+          }
+          if (use_p) {
+            const double need_mass = (double)tp * (double)Zk;
+            if (!((double)me >= need_mass) && (double)(me + m_t) >= need_mass) {   // at most one thread
+              unsigned long long mm = me;
+              for (uint32_t e = e0; e < e1; ++e) {
+                const uint32_t d = nzl[e];
+                mm += (unsigned long long)h[d] * mass_of(value_of(d));
+                if ((double)mm >= need_mass) { s_df = d; s_zf = mm; s_found = 1; break; }
+              }
+            }
+            __syncthreads();
+          }
+          // rounding can leave the mass criterion unmet even at the lowest key, which is then taken:
+          // with tokens below the counters that key is not known here
+          if (!use_p || s_found || s_tail == 0) {
+            if (tid == 0) {
+              uint32_t d_f;
+              unsigned long long Zf;
+              if (use_p) {
+                if (s_found) { d_f = s_df; Zf = s_zf; } else { d_f = nzl[n_nz - 1]; Zf = total; }
+                if (use_k && d_f > s_dk) { d_f = s_dk; Zf = s_zk; }   // the sets stay nested
+              } else {
+                d_f = s_dk; Zf = s_zk;
+              }
+              p.row_thresh[row] = order_key32(value_of(d_f));
+              p.row_z[row] = (double)Zf / (double)kMassScale;
+            }
+            return;
+          }
+        }
+      }
+    }
+    __syncthreads();
+  }
 
   // warp 0: the highest bin b such that (count or mass of bins >= b, plus what lies above the
   // prefix) reaches the target; leaves the bin, and count / mass of the bins above it, in shared memory
