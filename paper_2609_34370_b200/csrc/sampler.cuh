@@ -399,6 +399,10 @@ __device__ __forceinline__ uint32_t order_key32(float f) {
 
 // top-k / top-p thresholds of one logits row per block (kFilterThreads threads).
 //
+// bf16 rows are settled by one histogram of counts over their exact 16-bit keys (see the kernel);
+// what follows is the general way, which fp32 rows take, and bf16 rows with values outside that
+// histogram's range.
+//
 // The kept set is {v : key(x_v) >= T}.  T is found by a descent from the top, level by level; each
 // level is a 256-bin histogram (count, mass) of the elements still in play, and warp 0 picks the
 // bin where the running count reaches top_k, or the running mass reaches top_p times the survivors'
@@ -429,7 +433,7 @@ constexpr int kFilterSmemBytes = 4 * 256 * 32 * 4 + 256 * (8 + 4) * 2 + kFilterL
 constexpr int kExactUnroll = 4;                                   // 16-byte loads per thread and round
 constexpr int kExactPerThread = 35;                               // odd: a thread's run of counters starts in its own bank
 constexpr int kExactBins = kFilterThreads * kExactPerThread;      // counters of the exact-value histogram (bf16 rows)
-constexpr int kExactListCap = (kFilterSmemBytes - kExactBins * 4) / 2;   // 16-bit distances of the occupied counters
+constexpr int kExactListCap = (kFilterSmemBytes - (kExactBins + 32) * 4) / 2;   // 16-bit distances of the occupied counters
 static_assert(kExactBins <= 65536 && kExactListCap >= 16384, "the exact-value histogram and its list reuse the general path's shared memory");
 
 // Calls f(x) for every element of a row; the block's threads stride over 16-byte vectors and keep
@@ -641,7 +645,7 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
   if constexpr (sizeof(T) == 2) {
     // the exact-value histogram below is cleared while those two are on their way
     uint32_t *h = reinterpret_cast<uint32_t *>(fsm);
-    for (int i = tid; i < kExactBins; i += kFilterThreads) h[i] = 0;
+    for (int i = tid; i < kExactBins + 32; i += kFilterThreads) h[i] = 0;
   }
   const bool use_k = tk_raw >= 1 && tk_raw < p.vocab;
   const bool use_p = tp < 1.f;
@@ -658,15 +662,17 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
 
   // bf16 rows: one histogram of COUNTS over the exact values.  A bf16 logit has a 16-bit key, and the
   // keys of a row lie within a few ten thousand steps below the key of its maximum (128 per binade:
-  // from 16 down through zero to -16 are 38 k keys), so one counter per key fits in shared memory.
+  // from 16 down through zero to -16 are 34 k keys), so one counter per key fits in shared memory.
   // Equal values have equal masses, so the mass of a key is its count times the mass of its value -
   // the same integer as the sum over its elements - and the thresholds follow from one scan over the
-  // counters in descending key order: no masses are added per element, no second sweep, no further
-  // levels.  A row with a value outside the counters' range (never seen with logits) takes the
-  // general path below.
+  // occupied counters in descending key order: no masses are added per element, no second sweep,
+  // no further levels.  What bounds the sweep are the shared-memory atomics: 32 random counters per
+  // instruction meet in about four bank conflicts.  Values below the counters are tolerated while
+  // they carry no mass (masked tokens at -inf) and no threshold falls among them; any other row
+  // with values outside the counters' range takes the general path below.
   if constexpr (sizeof(T) == 2) {
     uint32_t *h = reinterpret_cast<uint32_t *>(fsm);   // [kExactBins], index = key distance below the reference
-    uint16_t *nzl = reinterpret_cast<uint16_t *>(fsm + kExactBins * 4);   // [kExactListCap] distances of the occupied counters
+    uint16_t *nzl = reinterpret_cast<uint16_t *>(fsm + (kExactBins + 32) * 4);   // [kExactListCap] distances of the occupied counters
     __shared__ uint32_t s_over, s_tail, s_dk, s_df, s_found, s_nn, s_tc, s_wc[kFilterWarps];
     __shared__ unsigned long long s_wm[kFilterWarps], s_zk, s_zf, s_tm;
     if (tid == 0) { s_over = 0; s_tail = 0; s_found = 0; }
@@ -682,35 +688,41 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
       key_ref = k < 0xffffu ? k + 1u : k;
     }
     __syncthreads();
-    // a value below the counters (masked tokens at -inf, typically) is harmless while it carries no
-    // mass and no threshold falls among such values; the lanes that get here together add once
-    auto below = [&](float x) {
-      const bool massless = (order_key32(x) >> 16) <= key_ref && mass_of(x) == 0ull;
-      const uint32_t act = __activemask();
-      const uint32_t zl = __ballot_sync(act, massless);
-      if (lane == __ffs(act) - 1) {
-        if (zl) atomicAdd(&s_tail, (uint32_t)__popc(zl));
-        if (zl != act) atomicAdd(&s_over, (uint32_t)__popc(act & ~zl));
-      }
-    };
     // Two logits per step of integer arithmetic: the sign of each half spread over the half (one
     // byte permute), the order key of both (one logic operation), both distances by one
     // subtraction - the reference is at or above every value, so no half borrows from the other.
+    // A value below the counters is counted in one of 32 spare counters behind them (the lane's own:
+    // a row full of masked tokens must not queue up on one address), so the loop has no branch.
     const uint32_t ref2 = key_ref * 0x10001u;
+    const uint32_t spare = (uint32_t)kExactBins + (uint32_t)lane;
     sweep_row_pairs<kExactUnroll>(reinterpret_cast<const __nv_bfloat16 *>(base), p.vocab, tid,
         [&](uint32_t w) {
           uint32_t sm;
           asm("prmt.b32 %0, %1, 0, 0xBB99;" : "=r"(sm) : "r"(w));
           const uint32_t d2 = ref2 - (w ^ (sm | 0x80008000u));
-          const uint32_t dl = d2 & 0xffffu, dh = d2 >> 16;
-          if (dl < (uint32_t)kExactBins) atomicAdd(&h[dl], 1u); else below(__uint_as_float(w << 16));
-          if (dh < (uint32_t)kExactBins) atomicAdd(&h[dh], 1u); else below(__uint_as_float(w & 0xffff0000u));
+          atomicAdd(&h[min(d2 & 0xffffu, spare)], 1u);
+          atomicAdd(&h[min(d2 >> 16, spare)], 1u);
         },
-        [&](float x) {
-          const uint32_t d = key_ref - (order_key32(x) >> 16);
-          if (d < (uint32_t)kExactBins) atomicAdd(&h[d], 1u); else below(x);
-        });
+        [&](float x) { atomicAdd(&h[min(key_ref - (order_key32(x) >> 16), spare)], 1u); });
     __syncthreads();
+    const bool outside = tid < 32 && h[kExactBins + tid] != 0u;
+    if (__syncthreads_or(outside)) {
+      // Values below the counters (masked tokens at -inf, typically) are harmless while they carry
+      // no mass and no threshold falls among them: one more sweep tells which kind they are.
+      sweep_row<T>(base, p.vocab, tid, [&](float x) {
+        const uint32_t k = order_key32(x) >> 16;
+        if (k > key_ref || key_ref - k >= (uint32_t)kExactBins) {
+          const bool massless = k <= key_ref && mass_of(x) == 0ull;
+          const uint32_t act = __activemask();
+          const uint32_t zl = __ballot_sync(act, massless);
+          if (lane == __ffs(act) - 1) {   // the lanes that got here together add once
+            if (zl) atomicAdd(&s_tail, (uint32_t)__popc(zl));
+            if (zl != act) atomicAdd(&s_over, (uint32_t)__popc(act & ~zl));
+          }
+        }
+      });
+      __syncthreads();
+    }
     if (s_over == 0) {
       auto value_of = [&](uint32_t d) -> float {
         const uint32_t k = key_ref - d;

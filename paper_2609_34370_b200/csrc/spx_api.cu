@@ -442,9 +442,12 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
     if constexpr (kFiltered) {
       if (cudaFuncSetAttribute(filter_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFilterSmemBytes) != cudaSuccess)
         return SPX_ERR_CUDA;
-      topk_list_kernel<T><<<rows, kTopkThreads, 0, stream>>>(p);
+      if (p.top_k) {   // the short way for small K; without a top-k array every row is the general kernel's
+        topk_list_kernel<T><<<rows, kTopkThreads, 0, stream>>>(p);
+        ++t_launches;
+      }
       filter_rows_kernel<T><<<rows, kFilterThreads, kFilterSmemBytes, stream>>>(p);
-      t_launches += 2;
+      ++t_launches;
     }
     const int accept_blocks = (p.batch * 32 + 127) / 128;
     accept_kernel<T, kScaled, kFiltered><<<accept_blocks + (kScaled ? p.batch : 0), 128, 0, stream>>>(p, accept_blocks);

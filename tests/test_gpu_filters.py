@@ -245,6 +245,49 @@ def test_small_top_k_with_a_block_of_equal_logits_at_the_cut(tie):
     assert rep.exact + rep.cdf_near_tie + rep.cdf_abs_near_tie + rep.accept_near_tie + rep.topp_near_tie == B
 
 
+@pytest.mark.parametrize("masked", [float("-inf"), float(torch.finfo(torch.bfloat16).min), -3.0e4])
+def test_masked_tokens_below_the_value_histogram(masked):
+    """bf16 rows are settled by a histogram over the exact values that reaches a few ten thousand
+    keys below the row maximum.  Masked tokens lie below it: they carry no mass, so cuts among the
+    other tokens are still taken from the histogram; a top-k that reaches into the masked block, or a
+    masked value that is still inside the histogram, must give the oracle's answer as well."""
+    V, B, k = 40000, 6, 1
+    g = torch.Generator().manual_seed(33)
+    T = (torch.randn(B * (k + 1), V, generator=g) * 2.5).to(torch.bfloat16)
+    Dr = (torch.randn(B * k, V, generator=g) * 2.5).to(torch.bfloat16)
+    for rows in (T, Dr):
+        rows[:, 28000:] = masked                 # 12000 masked tokens
+        rows[:, 100:103] = 0.0                   # exact zeros of both signs
+        rows[:, 103:105] = -0.0
+        rows[:, 105] = 1e-30                     # values next to zero: thousands of keys from the other logits
+        rows[:, 106] = -1e-30
+    qi = torch.arange(0, (B + 1) * (k + 1), k + 1, dtype=torch.int32)
+    tk = torch.tensor([0, 500, 35000, 0, 28000, 27999], dtype=torch.int32)   # 35000: the cut lies among the masked tokens
+    tp = torch.tensor([0.9, 1.0, 1.0, 0.5, 0.999, 1.0])
+    ids = torch.zeros(B * k, dtype=torch.int32)
+    for r in range(B):
+        q, kept, _ = oracle.filtered_row(Dr[r], 1.0, int(tk[r]), float(tp[r]))
+        ids[r] = int(torch.multinomial(q, 1, generator=g))
+    assert oracle.filtered_row(T[2 * 2], 1.0, 35000, 1.0)[1] == V
+    ua, us = torch.rand(B * k, generator=g), torch.rand(B, generator=g)
+    ref = oracle.rejection_sample(T, Dr, ids, qi, ua, us, top_k=tk, top_p=tp)
+    acc, tok, _, ws = spx.rejection_sample(T.to(DEV), Dr.to(DEV), ids.to(DEV), qi.to(DEV), ua.to(DEV), us.to(DEV),
+                                           top_k=tk.to(DEV), top_p=tp.to(DEV))
+    torch.cuda.synchronize()
+    assert int(ws.status.item()) in (0, spx.DEV_DEGENERATE)
+
+    class _B:
+        pass
+    bb = _B()
+    bb.batch, bb.q_indptr, bb.u_accept, bb.u_sample = B, qi, ua, us
+    bb.target_logits, bb.draft_logits, bb.draft_ids = T, Dr, ids
+    bb.spec = type("S", (), {"vocab": V})
+    rep = check_sampling(bb, acc, tok, ref, top_k=tk, top_p=tp)
+    _report(f"masked at {masked}", rep)
+    assert not rep.hard_mismatch, (rep, acc.cpu().tolist(), ref.accepted_len.tolist(), ref.margin.tolist())
+    assert rep.exact + rep.cdf_near_tie + rep.cdf_abs_near_tie + rep.accept_near_tie + rep.topp_near_tie == B
+
+
 def test_full_size_filtered():
     spec = W.CONFIGS[1]
     b_cpu = W.generate(spec)
