@@ -631,13 +631,13 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
   const double z_in = __ldg(p.row_z + row);
   const int r = __ldg(p.row_req + row);
   const float scale = __ldg(p.row_scale + row);
-  float M = -INFINITY;   // the row maximum (scaled) out of the sub-segment statistics: every warp reduces them for itself
-  for (int j = lane; j < p.nsub; j += 32) M = fmaxf(M, __ldg(&st[j].x));
   if (z_in == z_in) return;   // not pending (NaN): topk_list_kernel has settled this row
   if (r < 0) {
     if (tid == 0) { p.row_thresh[row] = 0; p.row_z[row] = -1.0; }
     return;
   }
+  float M = -INFINITY;   // the row maximum (scaled) out of the sub-segment statistics: every warp reduces them for itself
+  for (int j = lane; j < p.nsub; j += 32) M = fmaxf(M, __ldg(&st[j].x));
   constexpr int kLevels = sizeof(T) == 2 ? 2 : 4;      // exact key bytes after level 0
   constexpr int kKeyShift = sizeof(T) == 2 ? 16 : 0;   // bf16: the low 16 bits of the fp32 key carry nothing
   const int tk_raw = p.top_k ? __ldg(p.top_k + r) : 0;
