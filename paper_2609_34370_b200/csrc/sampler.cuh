@@ -467,19 +467,60 @@ __device__ __forceinline__ void sweep_row(const T *base, int vocab, int tid, F f
   }
 }
 
+// Calls f_vec(v) for every aligned group of eight bf16 logits of a row (one 16-byte vector, the
+// element of the lowest index in the low half of v.x) and f_one(x) for the elements of a ragged
+// end.  Rounds of kUnroll 16-byte loads per thread, predicated at the end of the row; the loads of
+// the next round are in flight while a round is processed (two register buffers in turn).
+template <int kUnroll, int kThreads, typename F, typename G>
+__device__ __forceinline__ void sweep_row_vecs(const __nv_bfloat16 *base, int vocab, int tid, F f_vec, G f_one) {
+  const int n_vec = vocab >> 3;
+  const uint4 *b4 = reinterpret_cast<const uint4 *>(base);
+  constexpr int kRound = kUnroll * kThreads;
+  auto load = [&](uint4 (&raw)[kUnroll], int v0) {
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u)
+      if (v0 + u * kThreads < n_vec) raw[u] = __ldg(b4 + v0 + u * kThreads);
+  };
+  auto work = [&](const uint4 (&raw)[kUnroll], int v0) {
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u)
+      if (v0 + u * kThreads < n_vec) f_vec(raw[u]);
+  };
+  uint4 ra[kUnroll], rb[kUnroll];
+  load(ra, tid);
+  for (int v0 = tid; v0 < n_vec; v0 += 2 * kRound) {
+    load(rb, v0 + kRound);
+    work(ra, v0);
+    load(ra, v0 + 2 * kRound);
+    work(rb, v0 + kRound);
+  }
+  for (int i = (n_vec << 3) + tid; i < vocab; i += kThreads) f_one(__bfloat162float(base[i]));
+}
+// The same, word by word: f_pair(w) for every aligned pair of logits.
+template <int kUnroll, int kThreads, typename F, typename G>
+__device__ __forceinline__ void sweep_row_pairs(const __nv_bfloat16 *base, int vocab, int tid, F f_pair, G f_one) {
+  sweep_row_vecs<kUnroll, kThreads>(base, vocab, tid, [&](const uint4 &v) { f_pair(v.x); f_pair(v.y); f_pair(v.z); f_pair(v.w); }, f_one);
+}
+
 // top-k (optionally with top-p on top) of one row per block for K no larger than the number of
 // sub-segments of the row: the K-th largest of the sub-segment maxima (left by the statistics
-// pass) is a lower bound of the K-th largest logit, so one compare-only sweep collects every
-// candidate (a few hundred logits for K = 50 on a 128k vocabulary) and the candidates are ranked
-// by counting - thread i sums count and mass of the keys above and at-or-above its own; no
-// histogram, no atomics on the masses.  256 threads and 16 KB of shared memory per row, so all the
-// rows of a batch are resident at once and the kernel runs at the rate the logits arrive.
-// Rows it cannot take (K larger than that, top-p alone, more than kTopkListCap candidates) are
-// left marked pending (row_z = NaN, set by row_scale_kernel) for filter_rows_kernel.
+// pass) is a lower bound of the K-th largest logit, so one compare-only sweep finds every
+// candidate (a few hundred logits for K = 50 on a 128k vocabulary).  256 threads and a few KB of
+// shared memory per row, so all the rows of a batch are resident at once and the kernel runs at
+// the rate the logits arrive.
+//   bf16 rows: the candidates lie within a few dozen 16-bit keys of the row maximum, so they are
+//   counted per exact value in a window of kTopkWindow keys below it (mass of a key = count times
+//   the mass of its value), and one scan over the window gives both thresholds; no list, so a
+//   block of equal logits at the cut costs nothing.
+//   fp32 rows: the candidates are listed and ranked by counting - thread i sums count and mass of
+//   the keys above and at-or-above its own; no histogram, no atomics on the masses.
+// Rows it cannot take (K larger than that, top-p alone, candidates beyond the window or the list)
+// are left marked pending (row_z = NaN, set by row_scale_kernel) for filter_rows_kernel.
 constexpr int kTopkThreads = 256;
 constexpr int kTopkListCap = 1024;
+constexpr int kTopkWindow = 1024;   // keys below the row maximum counted by the bf16 path (four per thread)
 template <typename T>
-__global__ void __launch_bounds__(kTopkThreads, 6) topk_list_kernel(SampleParams p) {
+__global__ void __launch_bounds__(kTopkThreads, 5) topk_list_kernel(SampleParams p) {
   __shared__ float s_list[kTopkListCap];
   __shared__ uint32_t s_key[kTopkListCap];
   __shared__ unsigned long long s_m[kTopkListCap];
@@ -501,22 +542,146 @@ __global__ void __launch_bounds__(kTopkThreads, 6) topk_list_kernel(SampleParams
   const float scale = p.row_scale[row];
   const T *base = row < p.total_q ? reinterpret_cast<const T *>(p.target) + (int64_t)row * p.row_stride
                                   : reinterpret_cast<const T *>(p.draft) + (int64_t)(row - p.total_q) * p.row_stride;
+  // the sub-segment maxima, once from memory (one per thread), then out of shared memory
+  __shared__ float s_max[kTopkThreads];
   const float2 *st = p.seg_stats + (int64_t)row * p.nsub;
+  if (tid < p.nsub) s_max[tid] = st[tid].x;
+  if (tid == 0) { s_n = 0; s_found = 0; }
+  __syncthreads();
   float M = -INFINITY;
-  for (int j = 0; j < p.nsub; ++j) M = fmaxf(M, st[j].x);
+  for (int j = 0; j < p.nsub; ++j) M = fmaxf(M, s_max[j]);
   auto mass_of = [&](float x) -> unsigned long long { return __float2ull_rn(fast_exp2(fmaf(x, scale, -M)) * kMassScale); };
   if (tid < p.nsub) {
-    const float mine = st[tid].x;
+    const float mine = s_max[tid];
     int rank = 0;
     for (int j = 0; j < p.nsub; ++j) {
-      const float o = st[j].x;
+      const float o = s_max[j];
       rank += (o > mine || (o == mine && j < tid)) ? 1 : 0;
     }
     if (rank == tk_raw - 1) s_bound = mine;
   }
-  if (tid == 0) { s_n = 0; s_found = 0; }
   __syncthreads();
   const float bound = s_bound - (fabsf(s_bound) * 1e-6f + 1e-6f);  // in the scaled (log2) domain, like the statistics
+  if constexpr (sizeof(T) == 2) {
+    __shared__ uint32_t s_hist[kTopkWindow];
+    __shared__ uint32_t s_wc[kTopkThreads / 32], s_dk, s_df;
+    __shared__ unsigned long long s_wm[kTopkThreads / 32], s_zk, s_zf;
+    const int lane = tid & 31, warp = tid >> 5;
+    // keys: the reference one step above a bf16 value at or above the row maximum, the bound one
+    // step below a bf16 value at or below the bound (in logit units)
+    uint32_t key_ref, key_lo;
+    {
+      float xub = M / scale;
+      xub = xub >= 0.f ? xub * (1.f + 0x1p-20f) : xub * (1.f - 0x1p-20f);
+      const uint32_t fu = __float_as_uint(xub);
+      const uint32_t bu = (fu & 0x80000000u) ? (fu >> 16) : ((fu + 0xffffu) >> 16);   // towards +inf
+      const uint32_t ku = order_key32(__uint_as_float(bu << 16)) >> 16;
+      key_ref = ku < 0xffffu ? ku + 1u : ku;
+      const uint32_t fl = __float_as_uint(bound / scale);
+      const uint32_t bl = (fl & 0x80000000u) ? ((fl + 0xffffu) >> 16) : (fl >> 16);   // towards -inf
+      const uint32_t kl = order_key32(__uint_as_float(bl << 16)) >> 16;
+      key_lo = kl > 0u ? kl - 1u : kl;
+    }
+    if (key_lo > key_ref || key_ref - key_lo >= (uint32_t)kTopkWindow) return;   // (uniform) the general kernel takes the row
+#pragma unroll
+    for (int i = 0; i < kTopkWindow / kTopkThreads; ++i) s_hist[tid + i * kTopkThreads] = 0;
+    __syncthreads();
+    bool above = false;
+    auto take = [&](uint32_t k) {
+      if (k >= key_lo) {
+        const uint32_t d = key_ref - k;
+        if (d < (uint32_t)kTopkWindow) atomicAdd(&s_hist[d], 1u); else above = true;   // above the reference: never with sound statistics
+      }
+    };
+    // eight logits per test: their maximum by packed bf16 instructions against the bound as a value
+    // (a superset of the key test: -0 and +0 compare equal); the rare vector that passes is taken
+    // apart key by key
+    const float x_lo = __uint_as_float(((key_lo & 0x8000u) ? (key_lo & 0x7fffu) : (~key_lo & 0xffffu)) << 16);
+    sweep_row_vecs<kFilterUnroll, kTopkThreads>(reinterpret_cast<const __nv_bfloat16 *>(base), p.vocab, tid,
+        [&](const uint4 &v) {
+          auto b2 = [](uint32_t w) { return *reinterpret_cast<const __nv_bfloat162 *>(&w); };
+          const __nv_bfloat162 m2 = __hmax2(__hmax2(b2(v.x), b2(v.y)), __hmax2(b2(v.z), b2(v.w)));
+          if (fmaxf(__low2float(m2), __high2float(m2)) >= x_lo) {
+            const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              uint32_t sm;
+              asm("prmt.b32 %0, %1, 0, 0xBB99;" : "=r"(sm) : "r"(w4[i]));
+              const uint32_t k2 = w4[i] ^ (sm | 0x80008000u);
+              take(k2 & 0xffffu);
+              take(k2 >> 16);
+            }
+          }
+        },
+        [&](float x) { take(order_key32(x) >> 16); });
+    if (__syncthreads_or(above)) return;
+    auto value_of = [&](uint32_t d) -> float {
+      const uint32_t k = key_ref - d;
+      const uint32_t b16 = (k & 0x8000u) ? (k & 0x7fffu) : (~k & 0xffffu);
+      return __uint_as_float(b16 << 16);
+    };
+    // every thread takes four consecutive keys of the window (descending), then a block scan
+    constexpr int kPerT = kTopkWindow / kTopkThreads;
+    const uint32_t d0 = (uint32_t)tid * kPerT;
+    uint32_t cb[kPerT], c_t = 0;
+    unsigned long long mb[kPerT], m_t = 0ull;
+#pragma unroll
+    for (int j = 0; j < kPerT; ++j) {
+      cb[j] = s_hist[d0 + j];
+      mb[j] = cb[j] ? (unsigned long long)cb[j] * mass_of(value_of(d0 + j)) : 0ull;
+      c_t += cb[j];
+      m_t += mb[j];
+    }
+    uint32_t ci = c_t;
+    unsigned long long mi = m_t;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t cn = __shfl_up_sync(0xffffffffu, ci, o);
+      const unsigned long long mn = __shfl_up_sync(0xffffffffu, mi, o);
+      if (lane >= o) { ci += cn; mi += mn; }
+    }
+    if (lane == 31) { s_wc[warp] = ci; s_wm[warp] = mi; }
+    __syncthreads();
+    uint32_t ce = ci - c_t, total_c = 0;   // counts / masses of the keys above this thread's four
+    unsigned long long me = mi - m_t;
+#pragma unroll
+    for (int w = 0; w < kTopkThreads / 32; ++w) {
+      if (w < warp) { ce += s_wc[w]; me += s_wm[w]; }
+      total_c += s_wc[w];
+    }
+    if (total_c < (uint32_t)tk_raw) return;   // (uniform; cannot happen: the K largest sub-segment maxima are candidates)
+    if (ce < (uint32_t)tk_raw && ce + c_t >= (uint32_t)tk_raw) {   // exactly one thread
+      uint32_t cc = ce;
+      unsigned long long mm = me;
+#pragma unroll
+      for (int j = 0; j < kPerT; ++j) {
+        cc += cb[j];
+        mm += mb[j];
+        if (cb[j] && cc >= (uint32_t)tk_raw) { s_dk = d0 + j; s_zk = mm; s_df = d0 + j; s_zf = mm; break; }
+      }
+    }
+    __syncthreads();
+    const unsigned long long Zk = s_zk;
+    if (use_p) {
+      // the highest key with mass(key >= T) >= P * kept mass: at or above the top-k cut, where the
+      // running mass equals the kept mass
+      const double need_mass = (double)tp * (double)Zk;
+      if (!((double)me >= need_mass) && (double)(me + m_t) >= need_mass) {   // exactly one thread
+        unsigned long long mm = me;
+#pragma unroll
+        for (int j = 0; j < kPerT; ++j) {
+          mm += mb[j];
+          if (cb[j] && (double)mm >= need_mass) { s_df = d0 + j; s_zf = mm; break; }
+        }
+      }
+      __syncthreads();
+    }
+    if (tid == 0) {
+      p.row_thresh[row] = order_key32(value_of(s_df));
+      p.row_z[row] = (double)s_zf / (double)kMassScale;
+    }
+    return;
+  }
   sweep_row<T, kTopkThreads>(base, p.vocab, tid, [&](float x) {
     if (x * scale >= bound) {
       const uint32_t i = atomicAdd(&s_n, 1u);
@@ -577,36 +742,6 @@ __global__ void __launch_bounds__(kTopkThreads, 6) topk_list_kernel(SampleParams
     p.row_thresh[row] = Tf;
     p.row_z[row] = (double)Zf / (double)kMassScale;
   }
-}
-
-// Calls f_pair(w) for every aligned pair of bf16 logits of a row (one 32-bit word, the element of the
-// lower index in the low half) and f_one(x) for the elements of a ragged end.  Rounds of kUnroll
-// 16-byte loads per thread, predicated at the end of the row; the loads of the next round are in
-// flight while a round is processed (two register buffers in turn).
-template <int kUnroll, typename F, typename G>
-__device__ __forceinline__ void sweep_row_pairs(const __nv_bfloat16 *base, int vocab, int tid, F f_pair, G f_one) {
-  const int n_vec = vocab >> 3;
-  const uint4 *b4 = reinterpret_cast<const uint4 *>(base);
-  constexpr int kRound = kUnroll * kFilterThreads;
-  auto load = [&](uint4 (&raw)[kUnroll], int v0) {
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u)
-      if (v0 + u * kFilterThreads < n_vec) raw[u] = __ldg(b4 + v0 + u * kFilterThreads);
-  };
-  auto work = [&](const uint4 (&raw)[kUnroll], int v0) {
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u)
-      if (v0 + u * kFilterThreads < n_vec) { f_pair(raw[u].x); f_pair(raw[u].y); f_pair(raw[u].z); f_pair(raw[u].w); }
-  };
-  uint4 ra[kUnroll], rb[kUnroll];
-  load(ra, tid);
-  for (int v0 = tid; v0 < n_vec; v0 += 2 * kRound) {
-    load(rb, v0 + kRound);
-    work(ra, v0);
-    load(ra, v0 + 2 * kRound);
-    work(rb, v0 + kRound);
-  }
-  for (int i = (n_vec << 3) + tid; i < vocab; i += kFilterThreads) f_one(__bfloat162float(base[i]));
 }
 
 template <typename T>
@@ -695,7 +830,7 @@ __global__ void __launch_bounds__(kFilterThreads, 1) filter_rows_kernel(SamplePa
     // a row full of masked tokens must not queue up on one address), so the loop has no branch.
     const uint32_t ref2 = key_ref * 0x10001u;
     const uint32_t spare = (uint32_t)kExactBins + (uint32_t)lane;
-    sweep_row_pairs<kExactUnroll>(reinterpret_cast<const __nv_bfloat16 *>(base), p.vocab, tid,
+    sweep_row_pairs<kExactUnroll, kFilterThreads>(reinterpret_cast<const __nv_bfloat16 *>(base), p.vocab, tid,
         [&](uint32_t w) {
           uint32_t sm;
           asm("prmt.b32 %0, %1, 0, 0xBB99;" : "=r"(sm) : "r"(w));
