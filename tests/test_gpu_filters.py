@@ -207,10 +207,10 @@ def test_crowded_threshold_bin():
 
 @pytest.mark.parametrize("tie", [300, 4000, 20000])
 def test_small_top_k_with_a_block_of_equal_logits_at_the_cut(tie):
-    """A small K takes the candidate-list path: every logit at or above a lower bound of the K-th
-    largest is collected and ranked.  A block of equal logits at the cut makes the list a few
-    hundred entries (ranked by counting), a few thousand (exact key-byte levels over the list in the
-    general kernel) or too long for any list (histogram path): same thresholds in all three."""
+    """A small K takes the short way: every logit at or above a lower bound of the K-th largest is a
+    candidate, counted per exact value in a window of keys below the row maximum (bf16).  A block of
+    equal logits at the cut - a few hundred, a few thousand, more than any list could hold - must
+    not change the thresholds."""
     V, B, k = 60000, 4, 1                    # 30 sub-segments of 2048 tokens: K <= 30 qualifies
     g = torch.Generator().manual_seed(21 + tie)
     T = (torch.randn(B * (k + 1), V, generator=g)).to(torch.bfloat16)
