@@ -208,7 +208,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     I.t_end = min(we.tile_end * kTileTokens, I.L);
   };
   const int pages_per_tile = kTileTokens >> p.log2P;
-  // warp-uniform bounded wait (all lanes poll; the verdict is shared so that the warp never
+  // warp-uniform bounded wait (all lanes poll; the outcome is shared so that the warp never
   // diverges around the .sync.aligned tensor-memory instructions)
   auto warp_wait = [&](uint64_t *bar, uint32_t parity) -> bool {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, bars, p.dev_status));

@@ -288,6 +288,58 @@ def test_masked_tokens_below_the_value_histogram(masked):
     assert rep.exact + rep.cdf_near_tie + rep.cdf_abs_near_tie + rep.accept_near_tie + rep.topp_near_tie == B
 
 
+@pytest.mark.parametrize("V", [5003, 40001])
+def test_ragged_vocabulary_and_unusual_rows(V):
+    """A vocabulary that is no multiple of eight (the rows' padding holds poison the kernels must not
+    read), and rows the named workloads do not have: all-negative logits, magnitudes next to zero, a
+    wide spread, sharp and flat temperatures, coarse values with many ties, one dominant token."""
+    B, k = 8, 2
+    VS = (V + 7) // 8 * 8
+    g = torch.Generator().manual_seed(77 + V)
+
+    def rows(n):
+        x = torch.randn(n, V, generator=g) * 2.5
+        return x
+
+    T, Dr = rows(B * (k + 1)), rows(B * k)
+    for X, per in ((T, k + 1), (Dr, k)):
+        X[1 * per:2 * per] = -20.0 + 5.0 * torch.randn(per, V, generator=g).clamp(-1.9, 1.9)     # all negative
+        X[2 * per:3 * per] *= 1e-3                                                               # next to zero
+        X[3 * per:4 * per] *= 3.2                                                                # wide
+        X[6 * per:7 * per] = torch.randint(-4, 5, (per, V), generator=g).float()                 # ties
+        X[7 * per:8 * per, 17] = 40.0                                                            # one dominant token
+    T, Dr = T.to(torch.bfloat16), Dr.to(torch.bfloat16)
+    Tp = torch.full((T.shape[0], VS), 1e4, dtype=torch.bfloat16)
+    Dp = torch.full((Dr.shape[0], VS), 1e4, dtype=torch.bfloat16)
+    Tp[:, :V], Dp[:, :V] = T, Dr
+    qi = torch.arange(0, (B + 1) * (k + 1), k + 1, dtype=torch.int32)
+    tk = torch.tensor([3, 0, 200, 0, 2, 1000, 0, 3], dtype=torch.int32)
+    tp = torch.tensor([1.0, 0.9, 0.8, 0.3, 1.0, 0.95, 0.5, 0.9])
+    tau = torch.tensor([1.0, 1.0, 1.0, 1.0, 0.05, 4.0, 1.0, 1.0])
+    ids = torch.zeros(B * k, dtype=torch.int32)
+    for r in range(B):
+        for i in range(k):
+            q, _, _ = oracle.filtered_row(Dr[r * k + i], float(tau[r]), int(tk[r]), float(tp[r]))
+            ids[r * k + i] = int(torch.multinomial(q, 1, generator=g))
+    ua, us = torch.rand(B * k, generator=g), torch.rand(B, generator=g)
+    ref = oracle.rejection_sample(T, Dr, ids, qi, ua, us, temperature=tau, top_k=tk, top_p=tp)
+    acc, tok, _, ws = spx.rejection_sample(Tp.to(DEV), Dp.to(DEV), ids.to(DEV), qi.to(DEV), ua.to(DEV), us.to(DEV), vocab=V,
+                                           temperature=tau.to(DEV), top_k=tk.to(DEV), top_p=tp.to(DEV))
+    torch.cuda.synchronize()
+    assert int(ws.status.item()) in (0, spx.DEV_DEGENERATE)
+
+    class _B:
+        pass
+    bb = _B()
+    bb.batch, bb.q_indptr, bb.u_accept, bb.u_sample = B, qi, ua, us
+    bb.target_logits, bb.draft_logits, bb.draft_ids = T, Dr, ids
+    bb.spec = type("S", (), {"vocab": V})
+    rep = check_sampling(bb, acc, tok, ref, temperature=tau, top_k=tk, top_p=tp)
+    _report(f"ragged vocabulary {V}", rep)
+    assert not rep.hard_mismatch, (rep, acc.cpu().tolist(), ref.accepted_len.tolist(), ref.margin.tolist())
+    assert int(tok.max()) < V
+
+
 def test_full_size_filtered():
     spec = W.CONFIGS[1]
     b_cpu = W.generate(spec)
