@@ -36,7 +36,7 @@ static thread_local long long *t_prof = nullptr;  // profiling builds only
 struct SideStream {
   int device = -1;
   cudaStream_t stream = nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr, mid = nullptr;
 };
 static thread_local SideStream t_side[16];
 
@@ -46,21 +46,23 @@ static SideStream *get_side_stream(int device) {
   if (s.device != device) {
     // a priority of its own: the sampling kernels are short and latency-bound, and a stream of
     // another priority does not share a hardware queue with the caller's stream.  Built in locals
-    // and committed only when all three handles exist, so a failure half way leaks nothing.
+    // and committed only when all four handles exist, so a failure half way leaks nothing.
     int prio_lo = 0, prio_hi = 0;
     cudaStream_t stream = nullptr;
-    cudaEvent_t fork = nullptr, join = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr, mid = nullptr;
     bool ok = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) == cudaSuccess;
     ok = ok && cudaStreamCreateWithPriority(&stream, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&fork, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&join, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&mid, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) {
+      if (mid) cudaEventDestroy(mid);
       if (join) cudaEventDestroy(join);
       if (fork) cudaEventDestroy(fork);
       if (stream) cudaStreamDestroy(stream);
       return nullptr;
     }
-    s.stream = stream; s.fork = fork; s.join = join;
+    s.stream = stream; s.fork = fork; s.join = join; s.mid = mid;
     s.device = device;
   }
   return &s;
@@ -303,7 +305,8 @@ static cudaError_t launch_tc(const CUtensorMap &kmap, const CUtensorMap &vmap, c
 // ---------------------------------------------------------------------------------------------
 // launches
 // ---------------------------------------------------------------------------------------------
-enum { kPhasePlan = 1, kPhaseMain = 2, kPhaseStats = 1, kPhaseTail = 2, kPhaseAll = 3 };
+enum { kPhasePlan = 1, kPhaseMain = 2, kPhaseAll = 3 };                        // attention: planner, kernels behind it
+enum { kPhaseStats = 1, kPhaseTail = 2, kPhaseFilter = 4, kPhaseSampAll = 7 };  // sampling: statistics, top-k / top-p thresholds, the rest
 
 static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws, int32_t *dev_status,
                                      cudaStream_t stream, const DeviceInfo &dev, int phases = kPhaseAll) {
@@ -438,8 +441,8 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
     }
     ++t_launches;
   }
-  if (phases & kPhaseTail) {
-    if constexpr (kFiltered) {
+  if constexpr (kFiltered) {
+    if (phases & kPhaseFilter) {
       if (cudaFuncSetAttribute(filter_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFilterSmemBytes) != cudaSuccess)
         return SPX_ERR_CUDA;
       if (p.top_k) {   // the short way for small K; without a top-k array every row is the general kernel's
@@ -449,6 +452,8 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
       filter_rows_kernel<T><<<rows, kFilterThreads, kFilterSmemBytes, stream>>>(p);
       ++t_launches;
     }
+  }
+  if (phases & kPhaseTail) {
     const int accept_blocks = (p.batch * 32 + 127) / 128;
     accept_kernel<T, kScaled, kFiltered><<<accept_blocks + (kScaled ? p.batch : 0), 128, 0, stream>>>(p, accept_blocks);
     resid_mass_kernel<T, kScaled, kFiltered><<<dim3(p.nseg, p.batch), kResidThreads, sizeof(T) == 2 ? kResidStageBytes : 0, stream>>>(p);
@@ -460,7 +465,7 @@ static spx_status_t launch_sampler_t(const SampleParams &p, cudaStream_t stream,
 }
 
 static spx_status_t launch_sampler(const spx_sample_args_t *s, unsigned char *ws, int32_t *dev_status,
-                                   cudaStream_t stream, int num_sms, int phases = kPhaseAll, int spare_sms = 0) {
+                                   cudaStream_t stream, int num_sms, int phases = kPhaseSampAll, int spare_sms = 0) {
   if (s->batch == 0) return SPX_OK;
   if (s->batch > 65535) return SPX_ERR_UNSUPPORTED;  // grid.y limit of the residual pass
   const SampleWs w = sample_ws_layout(s);
@@ -586,12 +591,24 @@ spx_status_t spx_verify_step(const spx_attn_args_t *attn, const spx_sample_args_
   // From here on the internal stream is forked: whatever fails below, it is joined back into the
   // caller's stream before the call returns (an unjoined fork would invalidate a stream capture
   // and, outside one, leave the caller's stream unordered against sampling kernels already queued).
-  const spx_status_t s1 = launch_sampler(sample, base + attn_bytes, dev_status, side->stream, dev.num_sms, kPhaseAll, 1);
+  // With top-k / top-p the threshold kernels sweep the logits once more, with blocks that do not fit
+  // beside the attention CTAs: left to themselves the two halves take the SMs from each other and the
+  // step is longer than their sum.  The attention kernel is therefore held back until the thresholds
+  // are known; accept, residual and draw then run beside and behind it as in the base rule.
+  const bool filtered = sample->top_k || sample->top_p;
+  spx_status_t s1 = launch_sampler(sample, base + attn_bytes, dev_status, side->stream, dev.num_sms,
+                                   filtered ? (kPhaseStats | kPhaseFilter) : kPhaseSampAll, 1);
   const spx_status_t s0 = launch_attention(attn, base, dev_status, stream, dev, kPhasePlan);
+  bool held = true;
+  if (filtered) {
+    held = cudaEventRecord(side->mid, side->stream) == cudaSuccess && cudaStreamWaitEvent(stream, side->mid, 0) == cudaSuccess;
+    const spx_status_t s1b = launch_sampler(sample, base + attn_bytes, dev_status, side->stream, dev.num_sms, kPhaseTail, 1);
+    if (s1 == SPX_OK) s1 = s1b;
+  }
   const bool rec = cudaEventRecord(side->join, side->stream) == cudaSuccess;
-  const spx_status_t s2 = s0 == SPX_OK ? launch_attention(attn, base, dev_status, stream, dev, kPhaseMain) : s0;
+  const spx_status_t s2 = s0 == SPX_OK && held ? launch_attention(attn, base, dev_status, stream, dev, kPhaseMain) : s0;
   const bool joined = rec && cudaStreamWaitEvent(stream, side->join, 0) == cudaSuccess;
-  if (!joined) return SPX_ERR_CUDA;
+  if (!joined || !held) return SPX_ERR_CUDA;
   return s0 != SPX_OK ? s0 : s1 != SPX_OK ? s1 : s2;
 }
 
