@@ -15,7 +15,7 @@
  *     _host.  The structs themselves, `ws_bytes` and all scalars live on the host.
  *   - The caller owns every buffer and the CUDA stream (`cuda_stream` is a cudaStream_t passed
  *     as void*; NULL = the legacy default stream).  The library allocates no device memory
- *     (spx_verify_step keeps one internal stream and two events per host thread and device).
+ *     (spx_verify_step keeps one internal stream and three events per host thread and device).
  *   - Calls only enqueue work on the stream and return; nothing synchronises the device.
  *   - Host-visible argument errors return a non-zero spx_status_t and launch nothing.
  *   - Errors in device-resident data (a page id out of range, a draft token id >= vocab, a
@@ -177,8 +177,10 @@ spx_status_t spx_rejection_sample(const spx_sample_args_t *args, void *ws, size_
  * The whole verify step.  The halves are independent given their inputs (logits are inputs
  * here), so the sampling half is forked onto a library-internal stream and joined back into
  * `cuda_stream` before the call returns: work enqueued on `cuda_stream` afterwards sees both
- * halves' outputs.  The internal stream and its two events are created on the first call of a
- * host thread on a device and are kept until the process ends.  If a launch fails after the
+ * halves' outputs.  With top_k / top_p the attention kernel additionally waits (one event) for
+ * the thresholds, whose kernels do not share an SM with it.  The internal stream and its three
+ * events are created on the first call of a host thread on a device and are kept until the
+ * process ends.  If a launch fails after the
  * fork, the internal stream is still joined back before the error is returned.  `ws` must hold
  * spx_workspace_size(attn, sample) bytes.
  */
