@@ -391,7 +391,7 @@ int32_t spx_last_launch_count(void);
  * the workspace of spx_verify_step).  The plan cuts the 128-token tiles of all (request, kv head)
  * pairs, in (request, head) order, into one contiguous range per CTA of the persistent attention
  * kernel.  Writes byte offsets and sizes into out[0..7] (host memory):
- *   out[0] header: int32 n_work, n_cta, n_part_slots, total_tiles, (cursor), overflow
+ *   out[0] header: int32 n_work, n_cta, n_part_slots, total_tiles, (cursor), overflow, n_combine
  *   out[1] cta_off: int32[n_cta + 1], entries of the work list that belong to the CTAs before c
  *   out[2] work list: 32-byte entries of int32 {req, tile_begin, tile_end, part_slot (-1: the pair
  *          is not split), q0, m, L, kv_head}

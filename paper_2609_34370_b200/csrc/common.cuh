@@ -98,7 +98,8 @@ struct PlanHeader {
   int32_t total_tiles;   // sum over requests of tiles (one kv-head)
   int32_t work_counter;  // dynamic scheduler cursor (SIMT kernel), zeroed by the planner
   int32_t overflow;      // 1 if the plan did not fit the workspace (nothing is executed then)
-  int32_t pad[2];
+  int32_t n_combine;     // pairs the combine kernel has work for (split pairs, pairs of invalid requests)
+  int32_t pad[1];
 };
 
 struct __align__(16) WorkEntry {
@@ -128,6 +129,7 @@ struct AttnParams {
   PlanHeader *hdr;
   int32_t *pair_nchunks;   // [B*Hkv]  chunks of the pair, 0 = invalid request
   int32_t *pair_part_base; // [B*Hkv]  first partial slot of a split pair
+  int32_t *combine_list;   // [B*Hkv]  the pairs the combine kernel has work for, n_combine of them
   int32_t *tile_prefix;    // [B+1]  tiles of the requests before r (one kv head)
   int32_t *valid_prefix;   // [B+1]  valid requests before r
   int32_t *cost_prefix;    // [B+1]  planning cost (one kv head) of the requests before r

@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int n_cta) {
   __shared__ int s_cut_vq[kPlanMaxCta + 1];  // index, among the valid requests' pairs, of the first pair that ends after cut c
   __shared__ int s_cut_in[kPlanMaxCta + 1];  // 1: cut c lies strictly inside that pair
   __shared__ int s_off[kPlanMaxCta + 1];     // work entries of the ranges before c
-  __shared__ int s_carry_t, s_carry_v, s_carry_c, s_carry_p, s_bad;
+  __shared__ int s_carry_t, s_carry_v, s_carry_c, s_carry_p, s_carry_l, s_bad;
   // The prefix sums of a batch of up to kPlanSmemReqs requests stay in shared memory: the searches
   // below would otherwise be chains of global loads, each a memory round trip beside the
   // bandwidth-bound kernel that runs while the plan is made (29 us instead of 6 for 64 requests).
@@ -67,7 +67,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int n_cta) {
   const int tid = threadIdx.x;
   const int Hkv = p.Hkv;
   if (n_cta > kPlanMaxCta) n_cta = kPlanMaxCta;
-  if (tid == 0) { s_carry_t = 0; s_carry_v = 0; s_carry_c = 0; s_carry_p = 0; s_bad = 0; }
+  if (tid == 0) { s_carry_t = 0; s_carry_v = 0; s_carry_c = 0; s_carry_p = 0; s_carry_l = 0; s_bad = 0; }
   __syncthreads();
 
   // pass 1: validate; prefix sums of tiles and of valid requests
@@ -191,6 +191,11 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int n_cta) {
     }
     const int part = block_exclusive_scan_1024(nch > 1 ? nch : 0, s_scratch, &s_total) + s_carry_p;
     const int tot_p = s_total;
+    // the pairs the combine kernel has work for: split ones, and those of invalid requests (sentinel rows)
+    const bool listed = pair < n_pairs && nch != 1;
+    const int lpos = block_exclusive_scan_1024(listed ? 1 : 0, s_scratch, &s_total) + s_carry_l;
+    const int tot_l = s_total;
+    if (listed) p.combine_list[lpos] = pair;
     if (pair < n_pairs) {
       const bool split = nch > 1 && part + nch <= p.max_part_slots;
       if (nch > 1 && !split) s_bad = 2;  // cannot happen: at most n_cta - 1 cuts, two slots each
@@ -213,7 +218,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int n_cta) {
       }
     }
     __syncthreads();
-    if (tid == 0) s_carry_p += tot_p;
+    if (tid == 0) { s_carry_p += tot_p; s_carry_l += tot_l; }
     __syncthreads();
   }
   if (tid == 0) {
@@ -224,94 +229,106 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int n_cta) {
     p.hdr->total_tiles = (int)total_tiles;
     p.hdr->work_counter = 0;
     p.hdr->overflow = bad;
+    p.hdr->n_combine = s_carry_l;
     if (bad) atomicOr(p.dev_status, SPX_DEV_BAD_LEN);
   }
 }
 
 // Merge the chunk partials of split pairs: m* = max_c m_c, l* = sum_c 2^(m_c-m*) l_c,
 // O = sum_c 2^(m_c-m*) O_c / l*, LSE = (m* + log2 l*) ln 2.  Also writes the sentinel rows of
-// invalid requests.  grid = (B * Hkv, ceil(rows_cap * D/4 / 256)), block = 256: one thread per
-// (row, 4 columns), chunks walked four at a time so that their loads are in flight together.
+// invalid requests.  The planner lists the pairs with such work (a cut of the tile axis makes at
+// most one: a hundred or so of the thousands of pairs of a large batch); blocks (b, y) take
+// entries b, b + gridDim.x, ... of the list, thread t of block (b, y) the item (row, 4 columns)
+// y * 256 + t of a pair - one item per thread, since the items of a thread would run one after
+// the other, a memory round trip each - with the chunks walked four at a time so that their loads
+// are in flight together.
+constexpr int kCombineThreads = 256;
 template <typename T>
-__global__ void __launch_bounds__(256) combine_kernel(AttnParams p) {
+__global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) {
   SPX_TL_SCOPE(kTlCombine);
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the attention kernel's partials (no-op without PDL)
-  const int r = blockIdx.x / p.Hkv, g = blockIdx.x % p.Hkv;
-  const int nch = p.pair_nchunks[blockIdx.x];
-  const int q0 = p.q_indptr[r];
-  int m = p.q_indptr[r + 1] - q0;
+  const int n_list = p.hdr->n_combine;
+  const bool overflow = p.hdr->overflow != 0;
   T *out = reinterpret_cast<T *>(p.out);
   const int D = p.D, G = p.G;
   const int vecs = D / 4;
-  const int item = blockIdx.y * blockDim.x + threadIdx.x;  // (row, dv)
-  if (nch == 0 || p.hdr->overflow || p.req_bad[r]) {
-    // invalid request (or unusable plan): zero rows, NaN lse; clamp the row range to the tensor
-    if (m < 0) m = 0;
-    if (m > p.max_q_len) m = p.max_q_len;
-    if (q0 < 0 || q0 + m > p.total_q) return;
-    if (item < m * G * vecs) {
-      const int row = item / vecs, dv = item % vecs, j = row / G, hg = row % G;
+  for (int li = blockIdx.x; li < n_list; li += gridDim.x) {
+    const int pair = p.combine_list[li];
+    const int r = pair / p.Hkv, g = pair % p.Hkv;
+    const int nch = p.pair_nchunks[pair];
+    const int q0 = p.q_indptr[r];
+    int m = p.q_indptr[r + 1] - q0;
+    if (nch == 0 || overflow || p.req_bad[r]) {
+      // invalid request (or unusable plan): zero rows, NaN lse; clamp the row range to the tensor
+      if (m < 0) m = 0;
+      if (m > p.max_q_len) m = p.max_q_len;
+      if (q0 < 0 || q0 + m > p.total_q) continue;
+      for (int item = blockIdx.y * blockDim.x + threadIdx.x; item < m * G * vecs; item += gridDim.y * blockDim.x) {
+        const int row = item / vecs, dv = item % vecs, j = row / G, hg = row % G;
+        const int64_t o_idx = ((int64_t)(q0 + j) * p.Hq + g * G + hg) * D + dv * 4;
+        for (int i = 0; i < 4; ++i) st_from_float(out, o_idx + i, 0.f);
+        if (dv == 0 && p.lse) p.lse[(int64_t)(q0 + j) * p.Hq + g * G + hg] = __int_as_float(0x7fc00000);
+      }
+      continue;
+    }
+    if (nch == 1) continue;  // written directly by the attention kernel (not listed; kept for safety)
+    const int64_t slot_base = (int64_t)p.pair_part_base[pair] * p.rows_cap;
+    const int64_t slot_step = p.rows_cap;
+    for (int item = blockIdx.y * blockDim.x + threadIdx.x; item < m * G * vecs; item += gridDim.y * blockDim.x) {
+      const int row = item / vecs, dv = item % vecs;
+      const int64_t slot0 = slot_base + row;
+      float lstar = 0.f, mstar = -INFINITY;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (nch <= 4) {
+        // the common case: every load of the item is issued at once (one memory round trip)
+        float2 ml[4];
+        float4 o[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int c = min(u, nch - 1);
+          ml[u] = p.part_ml[slot0 + c * slot_step];
+          o[u] = *reinterpret_cast<const float4 *>(p.part_o + (slot0 + c * slot_step) * D + dv * 4);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (u < nch) mstar = fmaxf(mstar, ml[u].x);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (u >= nch || ml[u].x == -INFINITY) continue;
+          const float w = fast_exp2(ml[u].x - mstar);
+          lstar += w * ml[u].y;
+          acc.x += w * o[u].x; acc.y += w * o[u].y; acc.z += w * o[u].z; acc.w += w * o[u].w;
+        }
+      } else {
+        for (int c = 0; c < nch; ++c) mstar = fmaxf(mstar, p.part_ml[slot0 + c * slot_step].x);
+        for (int c0 = 0; c0 < nch; c0 += 4) {
+          float2 ml[4];
+          float4 o[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int c = min(c0 + u, nch - 1);
+            ml[u] = p.part_ml[slot0 + c * slot_step];
+            o[u] = *reinterpret_cast<const float4 *>(p.part_o + (slot0 + c * slot_step) * D + dv * 4);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            if (c0 + u >= nch || ml[u].x == -INFINITY) continue;
+            const float w = fast_exp2(ml[u].x - mstar);
+            lstar += w * ml[u].y;
+            acc.x += w * o[u].x; acc.y += w * o[u].y; acc.z += w * o[u].z; acc.w += w * o[u].w;
+          }
+        }
+      }
+      const float inv = 1.f / lstar;
+      const int j = row / G, hg = row % G;
       const int64_t o_idx = ((int64_t)(q0 + j) * p.Hq + g * G + hg) * D + dv * 4;
-      for (int i = 0; i < 4; ++i) st_from_float(out, o_idx + i, 0.f);
-      if (dv == 0 && p.lse) p.lse[(int64_t)(q0 + j) * p.Hq + g * G + hg] = __int_as_float(0x7fc00000);
-    }
-    return;
-  }
-  if (nch == 1) return;  // written directly by the attention kernel
-  if (item >= m * G * vecs) return;
-  const int row = item / vecs, dv = item % vecs;
-  const int64_t slot0 = (int64_t)p.pair_part_base[blockIdx.x] * p.rows_cap + row;
-  const int64_t slot_step = p.rows_cap;
-  float lstar = 0.f, mstar = -INFINITY;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (nch <= 4) {
-    // the common case: every load of the item is issued at once (one memory round trip)
-    float2 ml[4];
-    float4 o[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int c = min(u, nch - 1);
-      ml[u] = p.part_ml[slot0 + c * slot_step];
-      o[u] = *reinterpret_cast<const float4 *>(p.part_o + (slot0 + c * slot_step) * D + dv * 4);
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-      if (u < nch) mstar = fmaxf(mstar, ml[u].x);
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      if (u >= nch || ml[u].x == -INFINITY) continue;
-      const float w = fast_exp2(ml[u].x - mstar);
-      lstar += w * ml[u].y;
-      acc.x += w * o[u].x; acc.y += w * o[u].y; acc.z += w * o[u].z; acc.w += w * o[u].w;
-    }
-  } else {
-    for (int c = 0; c < nch; ++c) mstar = fmaxf(mstar, p.part_ml[slot0 + c * slot_step].x);
-    for (int c0 = 0; c0 < nch; c0 += 4) {
-      float2 ml[4];
-      float4 o[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int c = min(c0 + u, nch - 1);
-        ml[u] = p.part_ml[slot0 + c * slot_step];
-        o[u] = *reinterpret_cast<const float4 *>(p.part_o + (slot0 + c * slot_step) * D + dv * 4);
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (c0 + u >= nch || ml[u].x == -INFINITY) continue;
-        const float w = fast_exp2(ml[u].x - mstar);
-        lstar += w * ml[u].y;
-        acc.x += w * o[u].x; acc.y += w * o[u].y; acc.z += w * o[u].z; acc.w += w * o[u].w;
-      }
+      st_from_float(out, o_idx + 0, acc.x * inv);
+      st_from_float(out, o_idx + 1, acc.y * inv);
+      st_from_float(out, o_idx + 2, acc.z * inv);
+      st_from_float(out, o_idx + 3, acc.w * inv);
+      if (dv == 0 && p.lse) p.lse[(int64_t)(q0 + j) * p.Hq + g * G + hg] = (mstar + log2f(lstar)) * kLn2;
     }
   }
-  const float inv = 1.f / lstar;
-  const int j = row / G, hg = row % G;
-  const int64_t o_idx = ((int64_t)(q0 + j) * p.Hq + g * G + hg) * D + dv * 4;
-  st_from_float(out, o_idx + 0, acc.x * inv);
-  st_from_float(out, o_idx + 1, acc.y * inv);
-  st_from_float(out, o_idx + 2, acc.z * inv);
-  st_from_float(out, o_idx + 3, acc.w * inv);
-  if (dv == 0 && p.lse) p.lse[(int64_t)(q0 + j) * p.Hq + g * G + hg] = (mstar + log2f(lstar)) * kLn2;
 }
 
 }  // namespace spx

@@ -40,6 +40,7 @@ struct SampleParams {
   float2 *seg_stats;   // [(TQ+TD)][nsub]  per sub-segment (max in log2 domain, sum)
   float *seg_resid;    // [B][nseg]        residual mass of each segment of row n (units of 1)
   float4 *req_norm;    // [B]  (Mt, 1/St, Md, 1/Sd) of row n, log2 domain maxima; Md = NaN => bonus
+  int32_t *req_done;   // [B]  residual-mass blocks of the request that have written their sum (zeroed by the accept kernel)
   int32_t *dev_status;
   // verification variants (both NULL: temperature 1 everywhere)
   const float *temperature;  // [B]  > 0: sample at that temperature; 0: greedy (NULL with filters: 1)
@@ -1390,6 +1391,7 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_
   const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (r >= p.batch) return;
+  if (lane == 0) p.req_done[r] = 0;   // counted up by the residual-mass blocks of this call
   const int t0 = p.q_indptr[r];
   const int k = p.q_indptr[r + 1] - t0 - 1;
   const int d0 = t0 - r;
@@ -1564,6 +1566,8 @@ constexpr int kResidStageBytes = 2 * kSegElems * 2;  // bf16 logits: the block's
 template <typename T, bool kScaled, bool kFiltered>
 __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 6 : 1) resid_mass_kernel(SampleParams p) {
   SPX_TL_SCOPE(kTlResidMass);
+  // the draw kernel may start once every block of this one runs: it waits per request, on req_done
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int seg_mine = blockIdx.x, r = blockIdx.y;
   ResidCtx<T, kScaled, kFiltered> c;
   if (!c.init(p, r) || !c.full_pass()) return;
@@ -1639,13 +1643,16 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 6 : 1) resid_m
       for (int w = 0; w < kResidThreads / 32; ++w) totp += s_wp[w];
       p.seg_pmass[(int64_t)r * p.nseg + seg_mine] = totp;
     }
+    __threadfence();
+    atomicAdd(p.req_done + r, 1);
   }
 }
 
 // The final draw of request r = blockIdx.x: segment choice in float64 over the segment masses,
 // token choice by an fp32 scan of the chosen segment (thread t owns tokens [32t, 32t+32) of it).
-// Launched with programmatic stream serialization: what the accept kernel left is read before the
-// wait, the masses of resid_mass_kernel after it.
+// Launched with programmatic stream serialization behind resid_mass_kernel, whose blocks release it
+// as they start: what the accept kernel left is read at once, the masses of the request's own
+// segments after its blocks have counted themselves done.
 template <typename T, bool kScaled, bool kFiltered>
 __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_pick_kernel(SampleParams p) {
   SPX_TL_SCOPE(kTlResidPick);
@@ -1653,8 +1660,23 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_p
   ResidCtx<T, kScaled, kFiltered> c;
   const bool live = c.init(p, r);
   const float u = p.u_sample[r];
-  asm volatile("griddepcontrol.wait;" ::: "memory");  // a no-op under a plain launch
   if (!live) return;
+  // The masses of this request's segments: the draw is launched while the mass blocks still run
+  // (every one of them is resident or done by then, so waiting for them cannot starve them) and
+  // waits for its own request's blocks only, with a limit like every wait of the library.
+  if (c.full_pass()) {
+    if (threadIdx.x == 0) {
+      const long long t_start = clock64();
+      for (;;) {
+        int done;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(done) : "l"(p.req_done + r) : "memory");
+        if (done >= p.nseg) break;
+        if (clock64() - t_start > kWaitLimitCycles) { atomicOr(p.dev_status, SPX_DEV_TIMEOUT); break; }
+        __nanosleep(64);
+      }
+    }
+    __syncthreads();
+  }
   const bool bonus = c.bonus, masked = c.masked;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float2 *tstats = p.seg_stats + (int64_t)(c.t0 + c.n) * p.nsub;

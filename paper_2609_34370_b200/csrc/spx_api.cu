@@ -92,7 +92,7 @@ constexpr int kPlanSmCount = 148;  // workspace sizing must not depend on a devi
 // workspace layout
 // ---------------------------------------------------------------------------------------------
 struct AttnWs {
-  size_t hdr, nchunks, part_base, tile_prefix, valid_prefix, cost_prefix, cta_off, req_bad, work, part_ml, part_o, total;
+  size_t hdr, nchunks, part_base, combine_list, tile_prefix, valid_prefix, cost_prefix, cta_off, req_bad, work, part_ml, part_o, total;
   int32_t max_work, max_part_slots, rows_cap;
 };
 
@@ -134,6 +134,7 @@ static AttnWs attn_ws_layout(const spx_attn_args_t *a) {
   w.hdr = off; off = align_up(off + sizeof(PlanHeader), 256);
   w.nchunks = off; off = align_up(off + sizeof(int32_t) * pairs, 256);
   w.part_base = off; off = align_up(off + sizeof(int32_t) * pairs, 256);
+  w.combine_list = off; off = align_up(off + sizeof(int32_t) * pairs, 256);
   w.tile_prefix = off; off = align_up(off + sizeof(int32_t) * ((size_t)a->batch + 1), 256);
   w.valid_prefix = off; off = align_up(off + sizeof(int32_t) * ((size_t)a->batch + 1), 256);
   w.cost_prefix = off; off = align_up(off + sizeof(int32_t) * ((size_t)a->batch + 1), 256);
@@ -148,7 +149,7 @@ static AttnWs attn_ws_layout(const spx_attn_args_t *a) {
 }
 
 struct SampleWs {
-  size_t seg_stats, seg_resid, req_norm, row_scale, row_req, row_thresh, row_z, req_thresh, seg_pmass, total;
+  size_t seg_stats, seg_resid, req_norm, req_done, row_scale, row_req, row_thresh, row_z, req_thresh, seg_pmass, total;
   int32_t nseg, nsub;
 };
 
@@ -177,6 +178,7 @@ static SampleWs sample_ws_layout(const spx_sample_args_t *s) {
   w.seg_stats = off; off = align_up(off + sizeof(float2) * rows * w.nsub, 256);
   w.seg_resid = off; off = align_up(off + sizeof(float) * (size_t)s->batch * w.nseg, 256);
   w.req_norm = off; off = align_up(off + sizeof(float4) * (size_t)s->batch, 256);
+  w.req_done = off; off = align_up(off + sizeof(int32_t) * (size_t)s->batch, 256);
   w.row_scale = off;
   const bool filtered = s->top_k || s->top_p;
   if (s->temperature || filtered) off = align_up(off + sizeof(float) * rows, 256);
@@ -328,6 +330,7 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
   p.hdr = reinterpret_cast<PlanHeader *>(ws + w.hdr);
   p.pair_nchunks = reinterpret_cast<int32_t *>(ws + w.nchunks);
   p.pair_part_base = reinterpret_cast<int32_t *>(ws + w.part_base);
+  p.combine_list = reinterpret_cast<int32_t *>(ws + w.combine_list);
   p.tile_prefix = reinterpret_cast<int32_t *>(ws + w.tile_prefix);
   p.valid_prefix = reinterpret_cast<int32_t *>(ws + w.valid_prefix);
   p.cost_prefix = reinterpret_cast<int32_t *>(ws + w.cost_prefix);
@@ -390,9 +393,12 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
       e = p.D == 64 ? launch_simt(attn_simt_kernel<__nv_bfloat16, 64>) : launch_simt(attn_simt_kernel<__nv_bfloat16, 128>);
   }
   if (e != cudaSuccess) return SPX_ERR_CUDA;
-  const dim3 cgrid(p.batch * p.Hkv, (p.rows_cap * (p.D / 4) + 255) / 256);
-  e = a->kv_dtype == SPX_F32 ? launch_pdl(combine_kernel<float>, cgrid, dim3(256), 0, stream, p)
-                             : launch_pdl(combine_kernel<__nv_bfloat16>, cgrid, dim3(256), 0, stream, p);
+  // one row of blocks per listed pair on the named workloads (a cut of the tile axis lists at most one
+  // pair); longer lists - many invalid requests - are walked
+  const int pairs_all = p.batch * p.Hkv;
+  const dim3 cgrid(pairs_all < kPlanSmCount ? pairs_all : kPlanSmCount, (p.rows_cap * (p.D / 4) + kCombineThreads - 1) / kCombineThreads);
+  e = a->kv_dtype == SPX_F32 ? launch_pdl(combine_kernel<float>, cgrid, dim3(kCombineThreads), 0, stream, p)
+                             : launch_pdl(combine_kernel<__nv_bfloat16>, cgrid, dim3(kCombineThreads), 0, stream, p);
   ++t_launches;
   return e == cudaSuccess ? SPX_OK : SPX_ERR_CUDA;
 }
@@ -479,6 +485,7 @@ static spx_status_t launch_sampler(const spx_sample_args_t *s, unsigned char *ws
   p.seg_stats = reinterpret_cast<float2 *>(ws + w.seg_stats);
   p.seg_resid = reinterpret_cast<float *>(ws + w.seg_resid);
   p.req_norm = reinterpret_cast<float4 *>(ws + w.req_norm);
+  p.req_done = reinterpret_cast<int32_t *>(ws + w.req_done);
   p.dev_status = dev_status;
   if (s->top_k || s->top_p) {
     p.temperature = s->temperature; p.top_k = s->top_k; p.top_p = s->top_p;
