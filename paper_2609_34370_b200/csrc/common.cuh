@@ -102,6 +102,16 @@ struct PlanHeader {
   int32_t pad[1];
 };
 
+// What the combine kernel needs to know of a pair, in one load.
+struct __align__(16) CombineEntry {
+  int32_t pair;       // request * Hkv + kv head; -1: past the end of the list
+  int32_t nch;        // chunks of the pair (0: invalid request, sentinel rows)
+  int32_t part_base;  // first partial slot
+  int32_t q0, m;      // first query row and number of query rows of the request
+  int32_t pad[3];
+};
+constexpr int kCombineListPad = 148;   // entries the planner always writes (the combine kernel's blocks read their first entry unconditionally)
+
 struct __align__(16) WorkEntry {
   int32_t req;         // request index
   int32_t tile_begin;  // first tile of the chunk
@@ -129,7 +139,7 @@ struct AttnParams {
   PlanHeader *hdr;
   int32_t *pair_nchunks;   // [B*Hkv]  chunks of the pair, 0 = invalid request
   int32_t *pair_part_base; // [B*Hkv]  first partial slot of a split pair
-  int32_t *combine_list;   // [B*Hkv]  the pairs the combine kernel has work for, n_combine of them
+  CombineEntry *combine_list;  // [max(B*Hkv, kCombineListPad)]  the pairs the combine kernel has work for: n_combine entries, then pair = -1
   int32_t *tile_prefix;    // [B+1]  tiles of the requests before r (one kv head)
   int32_t *valid_prefix;   // [B+1]  valid requests before r
   int32_t *cost_prefix;    // [B+1]  planning cost (one kv head) of the requests before r

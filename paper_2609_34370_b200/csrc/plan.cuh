@@ -195,7 +195,14 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int n_cta) {
     const bool listed = pair < n_pairs && nch != 1;
     const int lpos = block_exclusive_scan_1024(listed ? 1 : 0, s_scratch, &s_total) + s_carry_l;
     const int tot_l = s_total;
-    if (listed) p.combine_list[lpos] = pair;
+    if (listed) {
+      CombineEntry ce;
+      ce.pair = pair; ce.nch = nch; ce.part_base = (nch > 1 && part + nch <= p.max_part_slots) ? part : -1;
+      if (in_smem) { ce.q0 = s_q0[r]; ce.m = s_m[r]; }
+      else { ce.q0 = p.q_indptr[r]; ce.m = p.q_indptr[r + 1] - ce.q0; }
+      ce.pad[0] = ce.pad[1] = ce.pad[2] = 0;
+      p.combine_list[lpos] = ce;
+    }
     if (pair < n_pairs) {
       const bool split = nch > 1 && part + nch <= p.max_part_slots;
       if (nch > 1 && !split) s_bad = 2;  // cannot happen: at most n_cta - 1 cuts, two slots each
@@ -220,6 +227,12 @@ __global__ void __launch_bounds__(1024) plan_kernel(AttnParams p, int n_cta) {
     __syncthreads();
     if (tid == 0) { s_carry_p += tot_p; s_carry_l += tot_l; }
     __syncthreads();
+  }
+  // the combine kernel's blocks read their first entry without knowing how long the list is
+  if (tid < kCombineListPad && tid >= s_carry_l) {
+    CombineEntry ce;
+    ce.pair = -1; ce.nch = 1; ce.part_base = -1; ce.q0 = 0; ce.m = 0; ce.pad[0] = ce.pad[1] = ce.pad[2] = 0;
+    p.combine_list[tid] = ce;
   }
   if (tid == 0) {
     const bool bad = overflow || s_bad == 2;
@@ -247,18 +260,24 @@ template <typename T>
 __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) {
   SPX_TL_SCOPE(kTlCombine);
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the attention kernel's partials (no-op without PDL)
-  const int n_list = p.hdr->n_combine;
-  const bool overflow = p.hdr->overflow != 0;
+  const int n_list = p.hdr->n_combine;   // needed from the second entry of a block on: in flight beside the first entry
+  // every request's "bad page id" flag is looked at by one block (the attention kernel sets it while
+  // it runs, so the planner's list cannot know): fetched here, used after the list
+  const int bid = blockIdx.y * gridDim.x + blockIdx.x, n_blocks = gridDim.x * gridDim.y;
+  const int bad_first = bid < p.batch ? p.req_bad[bid] : 0;
   T *out = reinterpret_cast<T *>(p.out);
   const int D = p.D, G = p.G;
   const int vecs = D / 4;
-  for (int li = blockIdx.x; li < n_list; li += gridDim.x) {
-    const int pair = p.combine_list[li];
+  static_assert(sizeof(CombineEntry) == 32, "read as two 16-byte vectors");
+  for (int li = blockIdx.x; li < kCombineListPad || li < n_list; li += gridDim.x) {
+    if (li >= kCombineListPad && li >= n_list) break;
+    const int4 e0 = *reinterpret_cast<const int4 *>(p.combine_list + li);
+    const int pair = e0.x, nch = e0.y, part_base = e0.z, q0 = e0.w;
+    if (pair < 0) break;   // past the end of the list
+    int m = reinterpret_cast<const int32_t *>(p.combine_list + li)[4];
     const int r = pair / p.Hkv, g = pair % p.Hkv;
-    const int nch = p.pair_nchunks[pair];
-    const int q0 = p.q_indptr[r];
-    int m = p.q_indptr[r + 1] - q0;
-    if (nch == 0 || overflow || p.req_bad[r]) {
+    const int bad = p.req_bad[r];   // set by the attention kernel (a page id out of range); on its way beside the partials
+    if (nch == 0) {
       // invalid request (or unusable plan): zero rows, NaN lse; clamp the row range to the tensor
       if (m < 0) m = 0;
       if (m > p.max_q_len) m = p.max_q_len;
@@ -272,7 +291,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) 
       continue;
     }
     if (nch == 1) continue;  // written directly by the attention kernel (not listed; kept for safety)
-    const int64_t slot_base = (int64_t)p.pair_part_base[pair] * p.rows_cap;
+    const int64_t slot_base = (int64_t)part_base * p.rows_cap;
     const int64_t slot_step = p.rows_cap;
     for (int item = blockIdx.y * blockDim.x + threadIdx.x; item < m * G * vecs; item += gridDim.y * blockDim.x) {
       const int row = item / vecs, dv = item % vecs;
@@ -319,15 +338,31 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) 
           }
         }
       }
-      const float inv = 1.f / lstar;
+      // a request the attention kernel found a bad page id in gets the sentinel rows instead
+      const float inv = bad ? 0.f : 1.f / lstar;
       const int j = row / G, hg = row % G;
       const int64_t o_idx = ((int64_t)(q0 + j) * p.Hq + g * G + hg) * D + dv * 4;
-      st_from_float(out, o_idx + 0, acc.x * inv);
-      st_from_float(out, o_idx + 1, acc.y * inv);
-      st_from_float(out, o_idx + 2, acc.z * inv);
-      st_from_float(out, o_idx + 3, acc.w * inv);
-      if (dv == 0 && p.lse) p.lse[(int64_t)(q0 + j) * p.Hq + g * G + hg] = (mstar + log2f(lstar)) * kLn2;
+      st_from_float(out, o_idx + 0, bad ? 0.f : acc.x * inv);
+      st_from_float(out, o_idx + 1, bad ? 0.f : acc.y * inv);
+      st_from_float(out, o_idx + 2, bad ? 0.f : acc.z * inv);
+      st_from_float(out, o_idx + 3, bad ? 0.f : acc.w * inv);
+      if (dv == 0 && p.lse)
+        p.lse[(int64_t)(q0 + j) * p.Hq + g * G + hg] = bad ? __int_as_float(0x7fc00000) : (mstar + log2f(lstar)) * kLn2;
     }
+  }
+  // sentinel rows (zero output, NaN lse) for every head of a request with a bad page id, whichever
+  // of its pairs were split
+  for (int r = bid; r < p.batch; r += n_blocks) {
+    if (!(r == bid ? bad_first : p.req_bad[r])) continue;
+    const int q0 = p.q_indptr[r];
+    int m = p.q_indptr[r + 1] - q0;
+    if (m < 0) m = 0;
+    if (m > p.max_q_len) m = p.max_q_len;
+    if (q0 < 0 || q0 + m > p.total_q) continue;
+    const int64_t n = (int64_t)m * p.Hq * D, base = (int64_t)q0 * p.Hq * D;
+    for (int64_t i = threadIdx.x; i < n; i += blockDim.x) st_from_float(out, base + i, 0.f);
+    if (p.lse)
+      for (int i = threadIdx.x; i < m * p.Hq; i += blockDim.x) p.lse[(int64_t)q0 * p.Hq + i] = __int_as_float(0x7fc00000);
   }
 }
 

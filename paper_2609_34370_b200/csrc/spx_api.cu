@@ -134,7 +134,7 @@ static AttnWs attn_ws_layout(const spx_attn_args_t *a) {
   w.hdr = off; off = align_up(off + sizeof(PlanHeader), 256);
   w.nchunks = off; off = align_up(off + sizeof(int32_t) * pairs, 256);
   w.part_base = off; off = align_up(off + sizeof(int32_t) * pairs, 256);
-  w.combine_list = off; off = align_up(off + sizeof(int32_t) * pairs, 256);
+  w.combine_list = off; off = align_up(off + sizeof(CombineEntry) * (pairs > (size_t)kCombineListPad ? pairs : (size_t)kCombineListPad), 256);
   w.tile_prefix = off; off = align_up(off + sizeof(int32_t) * ((size_t)a->batch + 1), 256);
   w.valid_prefix = off; off = align_up(off + sizeof(int32_t) * ((size_t)a->batch + 1), 256);
   w.cost_prefix = off; off = align_up(off + sizeof(int32_t) * ((size_t)a->batch + 1), 256);
@@ -330,7 +330,7 @@ static spx_status_t launch_attention(const spx_attn_args_t *a, unsigned char *ws
   p.hdr = reinterpret_cast<PlanHeader *>(ws + w.hdr);
   p.pair_nchunks = reinterpret_cast<int32_t *>(ws + w.nchunks);
   p.pair_part_base = reinterpret_cast<int32_t *>(ws + w.part_base);
-  p.combine_list = reinterpret_cast<int32_t *>(ws + w.combine_list);
+  p.combine_list = reinterpret_cast<CombineEntry *>(ws + w.combine_list);
   p.tile_prefix = reinterpret_cast<int32_t *>(ws + w.tile_prefix);
   p.valid_prefix = reinterpret_cast<int32_t *>(ws + w.valid_prefix);
   p.cost_prefix = reinterpret_cast<int32_t *>(ws + w.cost_prefix);

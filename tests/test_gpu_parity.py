@@ -235,6 +235,8 @@ def test_device_side_faults_are_reported_not_fatal():
     out, lse, ws = gpu_attention(bad.to(DEV))
     assert int(ws.status.item()) & spx.DEV_BAD_PAGE
     check_attention(b_cpu, out, lse, ref_o, ref_l, reqs=[0, 1, 3])
+    q0, q1 = int(b_cpu.q_indptr[2]), int(b_cpu.q_indptr[3])
+    assert (out[q0:q1] == 0).all() and torch.isnan(lse[q0:q1]).all()      # sentinel rows, split pair or not
     # draft id out of range for request 0 -> BAD_TOKEN, that request emits n = 0 and -1s
     bad = b_cpu.clone()
     bad.draft_ids[0] = spec.vocab
