@@ -38,9 +38,8 @@ struct SampleParams {
   float *diag_ratio;
   // workspace
   float2 *seg_stats;   // [(TQ+TD)][nsub]  per sub-segment (max in log2 domain, sum)
-  float *seg_resid;    // [B][nseg]        residual mass of each segment of row n (units of 1)
+  float *seg_resid;    // [B][nseg]        residual mass of each segment of row n (units of 1); kMassPending until its block has written it
   float4 *req_norm;    // [B]  (Mt, 1/St, Md, 1/Sd) of row n, log2 domain maxima; Md = NaN => bonus
-  int32_t *req_done;   // [B]  residual-mass blocks of the request that have written their sum (zeroed by the accept kernel)
   int32_t *dev_status;
   // verification variants (both NULL: temperature 1 everywhere)
   const float *temperature;  // [B]  > 0: sample at that temperature; 0: greedy (NULL with filters: 1)
@@ -1377,6 +1376,10 @@ __device__ __forceinline__ void greedy_request(const SampleParams &p, int r) {
   }
 }
 
+// A segment mass that its block has not written yet: a NaN with a payload no arithmetic produces.  The
+// accept kernel fills a request's masses with it, the draw kernel waits for it to go away.
+constexpr uint32_t kMassPending = 0x7fc0dead;
+
 // One warp per request, lane = row (lanes 0..k: target rows, lanes k+1..2k: draft rows).  Each lane
 // merges its row's segment pairs (fp32 exponentials, float64 sum); the accept ratios of all
 // drafts are evaluated in parallel in float64 and the first failure fixes n.  Writes
@@ -1391,7 +1394,7 @@ __global__ void __launch_bounds__(128) accept_kernel(SampleParams p, int accept_
   const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (r >= p.batch) return;
-  if (lane == 0) p.req_done[r] = 0;   // counted up by the residual-mass blocks of this call
+  for (int i = lane; i < p.nseg; i += 32) p.seg_resid[(int64_t)r * p.nseg + i] = __uint_as_float(kMassPending);
   const int t0 = p.q_indptr[r];
   const int k = p.q_indptr[r + 1] - t0 - 1;
   const int d0 = t0 - r;
@@ -1566,7 +1569,7 @@ constexpr int kResidStageBytes = 2 * kSegElems * 2;  // bf16 logits: the block's
 template <typename T, bool kScaled, bool kFiltered>
 __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 6 : 1) resid_mass_kernel(SampleParams p) {
   SPX_TL_SCOPE(kTlResidMass);
-  // the draw kernel may start once every block of this one runs: it waits per request, on req_done
+  // the draw kernel may start once every block of this one runs: it waits for its own request's masses
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int seg_mine = blockIdx.x, r = blockIdx.y;
   ResidCtx<T, kScaled, kFiltered> c;
@@ -1637,14 +1640,13 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 6 : 1) resid_m
   if (threadIdx.x == 0) {
     float tot = 0.f;
     for (int w = 0; w < kResidThreads / 32; ++w) tot += s_w[w];
-    p.seg_resid[(int64_t)r * p.nseg + seg_mine] = tot;
     if (kFiltered) {
       float totp = 0.f;
       for (int w = 0; w < kResidThreads / 32; ++w) totp += s_wp[w];
       p.seg_pmass[(int64_t)r * p.nseg + seg_mine] = totp;
+      __threadfence();   // the draw kernel reads it once it has seen the residual mass below
     }
-    __threadfence();
-    atomicAdd(p.req_done + r, 1);
+    p.seg_resid[(int64_t)r * p.nseg + seg_mine] = tot;
   }
 }
 
@@ -1652,7 +1654,7 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 6 : 1) resid_m
 // token choice by an fp32 scan of the chosen segment (thread t owns tokens [32t, 32t+32) of it).
 // Launched with programmatic stream serialization behind resid_mass_kernel, whose blocks release it
 // as they start: what the accept kernel left is read at once, the masses of the request's own
-// segments after its blocks have counted themselves done.
+// segments as their blocks write them.
 template <typename T, bool kScaled, bool kFiltered>
 __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_pick_kernel(SampleParams p) {
   SPX_TL_SCOPE(kTlResidPick);
@@ -1661,22 +1663,6 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_p
   const bool live = c.init(p, r);
   const float u = p.u_sample[r];
   if (!live) return;
-  // The masses of this request's segments: the draw is launched while the mass blocks still run
-  // (every one of them is resident or done by then, so waiting for them cannot starve them) and
-  // waits for its own request's blocks only, with a limit like every wait of the library.
-  if (c.full_pass()) {
-    if (threadIdx.x == 0) {
-      const long long t_start = clock64();
-      for (;;) {
-        int done;
-        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(done) : "l"(p.req_done + r) : "memory");
-        if (done >= p.nseg) break;
-        if (clock64() - t_start > kWaitLimitCycles) { atomicOr(p.dev_status, SPX_DEV_TIMEOUT); break; }
-        __nanosleep(64);
-      }
-    }
-    __syncthreads();
-  }
   const bool bonus = c.bonus, masked = c.masked;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float2 *tstats = p.seg_stats + (int64_t)(c.t0 + c.n) * p.nsub;
@@ -1708,7 +1694,26 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_p
     return i < kStageSegs ? s_mass[i] : from_target ? target_mass(i) : (double)resid[i];
   };
   bool use_target = bonus && !masked;
-  stage(use_target);
+  if (use_target) {
+    stage(true);
+  } else {
+    // The residual masses of this request's segments.  The draw is launched while the mass blocks
+    // still run (every one of them is resident or done by then, so waiting for them cannot starve
+    // them): each thread waits for one mass to appear - with a limit, like every wait of the
+    // library - and has it in hand when it does, so the masses cost no round trip of their own.
+    for (int i = threadIdx.x; i < p.nseg; i += kResidThreads) {
+      const long long t_start = clock64();
+      uint32_t bits;
+      for (;;) {
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(bits) : "l"(resid + i) : "memory");
+        if (bits != kMassPending) break;
+        if (clock64() - t_start > kWaitLimitCycles) { atomicOr(p.dev_status, SPX_DEV_TIMEOUT); bits = 0u; break; }
+        __nanosleep(32);
+      }
+      if (i < kStageSegs) s_mass[i] = (double)__uint_as_float(bits);
+    }
+    __syncthreads();
+  }
   if (threadIdx.x == 0) {
     double R = 0.0;
     for (int i = 0; i < p.nseg; ++i) R += mass_at(i, use_target);

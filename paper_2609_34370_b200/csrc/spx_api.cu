@@ -149,7 +149,7 @@ static AttnWs attn_ws_layout(const spx_attn_args_t *a) {
 }
 
 struct SampleWs {
-  size_t seg_stats, seg_resid, req_norm, req_done, row_scale, row_req, row_thresh, row_z, req_thresh, seg_pmass, total;
+  size_t seg_stats, seg_resid, req_norm, row_scale, row_req, row_thresh, row_z, req_thresh, seg_pmass, total;
   int32_t nseg, nsub;
 };
 
@@ -178,7 +178,6 @@ static SampleWs sample_ws_layout(const spx_sample_args_t *s) {
   w.seg_stats = off; off = align_up(off + sizeof(float2) * rows * w.nsub, 256);
   w.seg_resid = off; off = align_up(off + sizeof(float) * (size_t)s->batch * w.nseg, 256);
   w.req_norm = off; off = align_up(off + sizeof(float4) * (size_t)s->batch, 256);
-  w.req_done = off; off = align_up(off + sizeof(int32_t) * (size_t)s->batch, 256);
   w.row_scale = off;
   const bool filtered = s->top_k || s->top_p;
   if (s->temperature || filtered) off = align_up(off + sizeof(float) * rows, 256);
@@ -485,7 +484,6 @@ static spx_status_t launch_sampler(const spx_sample_args_t *s, unsigned char *ws
   p.seg_stats = reinterpret_cast<float2 *>(ws + w.seg_stats);
   p.seg_resid = reinterpret_cast<float *>(ws + w.seg_resid);
   p.req_norm = reinterpret_cast<float4 *>(ws + w.req_norm);
-  p.req_done = reinterpret_cast<int32_t *>(ws + w.req_done);
   p.dev_status = dev_status;
   if (s->top_k || s->top_p) {
     p.temperature = s->temperature; p.top_k = s->top_k; p.top_p = s->top_p;
