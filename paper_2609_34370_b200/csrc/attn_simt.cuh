@@ -35,6 +35,9 @@ struct SimtSmem {
 template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads) attn_simt_kernel(AttnParams p) {
   SPX_TL_SCOPE(kTlAttention);
+  // the combine kernel may take its places now (it reads the planner's list, then waits for this
+  // kernel to end): its launch then costs nothing behind the last CTA
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ int s_item;
   const SimtSmem lay(p.rows_cap, D);

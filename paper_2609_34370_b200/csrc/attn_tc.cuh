@@ -163,6 +163,9 @@ template <int D, int QROWS>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, AttnParams p) {
   SPX_TL_SCOPE(kTlAttention);
+  // the combine kernel may take its places now (it reads the planner's list, then waits for this
+  // kernel to end): its launch then costs nothing behind the last CTA
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   using Cfg = TcCfg<D, QROWS>;
   using namespace tc;
   extern __shared__ unsigned char smem_dyn[];

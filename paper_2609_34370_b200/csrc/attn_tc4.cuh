@@ -94,6 +94,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 attn_tc4_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
                 const __grid_constant__ CUtensorMap qmap, AttnParams p) {
   SPX_TL_SCOPE(kTlAttention);
+  // the combine kernel may take its places now (it reads the planner's list, then waits for this
+  // kernel to end): its launch then costs nothing behind the last CTA
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   using Cfg = Tc4Cfg<D, MROWS>;
   using namespace tc;
   constexpr int kSplit = Cfg::kSplit, TPT = Cfg::kTokPerThread;

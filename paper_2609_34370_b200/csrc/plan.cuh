@@ -259,8 +259,15 @@ constexpr int kCombineThreads = 256;
 template <typename T>
 __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) {
   SPX_TL_SCOPE(kTlCombine);
-  asm volatile("griddepcontrol.wait;" ::: "memory");  // the attention kernel's partials (no-op without PDL)
-  const int n_list = p.hdr->n_combine;   // needed from the second entry of a block on: in flight beside the first entry
+  // The attention kernel releases this one as its CTAs start, so the blocks are in place, with what
+  // the planner left for them in registers, when the attention kernel ends: the length of the list
+  // and the block's first entry are read before the wait, the attention kernel's own outputs (the
+  // partials, the "bad page id" flags) after it.
+  static_assert(sizeof(CombineEntry) == 32, "read as two 16-byte vectors");
+  const int n_list = p.hdr->n_combine;
+  const int4 first_a = *reinterpret_cast<const int4 *>(p.combine_list + blockIdx.x);   // blockIdx.x < kCombineListPad: always written
+  const int first_m = reinterpret_cast<const int32_t *>(p.combine_list + blockIdx.x)[4];
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // (no-op without programmatic launch)
   // every request's "bad page id" flag is looked at by one block (the attention kernel sets it while
   // it runs, so the planner's list cannot know): fetched here, used after the list
   const int bid = blockIdx.y * gridDim.x + blockIdx.x, n_blocks = gridDim.x * gridDim.y;
@@ -268,13 +275,13 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) 
   T *out = reinterpret_cast<T *>(p.out);
   const int D = p.D, G = p.G;
   const int vecs = D / 4;
-  static_assert(sizeof(CombineEntry) == 32, "read as two 16-byte vectors");
   for (int li = blockIdx.x; li < kCombineListPad || li < n_list; li += gridDim.x) {
     if (li >= kCombineListPad && li >= n_list) break;
-    const int4 e0 = *reinterpret_cast<const int4 *>(p.combine_list + li);
+    const bool first = li == (int)blockIdx.x;
+    const int4 e0 = first ? first_a : *reinterpret_cast<const int4 *>(p.combine_list + li);
     const int pair = e0.x, nch = e0.y, part_base = e0.z, q0 = e0.w;
     if (pair < 0) break;   // past the end of the list
-    int m = reinterpret_cast<const int32_t *>(p.combine_list + li)[4];
+    int m = first ? first_m : reinterpret_cast<const int32_t *>(p.combine_list + li)[4];
     const int r = pair / p.Hkv, g = pair % p.Hkv;
     const int bad = p.req_bad[r];   // set by the attention kernel (a page id out of range); on its way beside the partials
     if (nch == 0) {

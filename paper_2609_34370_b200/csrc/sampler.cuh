@@ -1714,7 +1714,39 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_p
     }
     __syncthreads();
   }
-  if (threadIdx.x == 0) {
+  // Total mass R, target u * R, first segment whose inclusive sum exceeds it (float64).  Up to 32
+  // segments (a vocabulary of 262144) are scanned by warp 0 with shuffles - a thread that walks
+  // them alone pays a shared-memory latency and a float64 add per segment, three times over, on
+  // the step's critical path; more segments are walked by one thread.
+  const bool by_warp = p.nseg <= 32;
+  auto warp_pick = [&](bool from_target) -> double {   // warp 0; returns R, leaves s_seg / s_target
+    const double m = lane < p.nseg ? s_mass[lane] : 0.0;
+    double incl = m;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const double nb = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += nb;
+    }
+    const double R = __shfl_sync(0xffffffffu, incl, 31);
+    const double target = (double)u * R;
+    const uint32_t over = __ballot_sync(0xffffffffu, lane < p.nseg && incl > target);
+    const uint32_t pos = __ballot_sync(0xffffffffu, m > 0.0);
+    // rounding can leave the target unreached at the end: the last segment with mass takes it
+    const int seg = over ? __ffs(over) - 1 : pos ? 31 - __clz(pos) : -1;
+    if (lane == (seg < 0 ? 0 : seg)) {
+      s_seg = seg;
+      s_target = (float)(target - (incl - m));
+      s_tok = 0x7fffffff;
+    }
+    (void)from_target;
+    return R;
+  };
+  if (by_warp) {
+    if (warp == 0) {
+      const double R = warp_pick(use_target);
+      if (lane == 0) s_degenerate = !use_target && !(R > 0.0);
+    }
+  } else if (threadIdx.x == 0) {
     double R = 0.0;
     for (int i = 0; i < p.nseg; ++i) R += mass_at(i, use_target);
     s_degenerate = !use_target && !(R > 0.0);
@@ -1723,28 +1755,33 @@ __global__ void __launch_bounds__(kResidThreads, sizeof(T) == 2 ? 4 : 1) resid_p
   if (s_degenerate) {  // the residual is identically zero: draw from the target row instead
     use_target = true;
     stage(true);
-  }
-  if (threadIdx.x == 0) {
-    // segment masses (float64), total R, target s*R, first segment whose inclusive sum exceeds it
-    double R = 0.0;
-    for (int i = 0; i < p.nseg; ++i) R += mass_at(i, use_target);
-    const double target = (double)u * R;
-    double cum = 0.0;
-    int seg = -1, last_pos = -1;
-    double before = 0.0, last_before = 0.0;
-    for (int i = 0; i < p.nseg; ++i) {
-      const double mass = mass_at(i, use_target);
-      if (mass > 0.0) { last_pos = i; last_before = cum; }
-      if (cum + mass > target) { seg = i; before = cum; break; }
-      cum += mass;
+    if (threadIdx.x == 0) atomicOr(p.dev_status, SPX_DEV_DEGENERATE);
+    if (by_warp) {
+      if (warp == 0) warp_pick(true);
+      __syncthreads();
     }
-    if (seg < 0) { seg = last_pos; before = last_before; }
-    s_seg = seg;
-    s_target = (float)(target - before);
-    s_tok = 0x7fffffff;
-    if (s_degenerate) atomicOr(p.dev_status, SPX_DEV_DEGENERATE);
   }
-  __syncthreads();
+  if (!by_warp) {
+    if (threadIdx.x == 0) {
+      double R = 0.0;
+      for (int i = 0; i < p.nseg; ++i) R += mass_at(i, use_target);
+      const double target = (double)u * R;
+      double cum = 0.0;
+      int seg = -1, last_pos = -1;
+      double before = 0.0, last_before = 0.0;
+      for (int i = 0; i < p.nseg; ++i) {
+        const double mass = mass_at(i, use_target);
+        if (mass > 0.0) { last_pos = i; last_before = cum; }
+        if (cum + mass > target) { seg = i; before = cum; break; }
+        cum += mass;
+      }
+      if (seg < 0) { seg = last_pos; before = last_before; }
+      s_seg = seg;
+      s_target = (float)(target - before);
+      s_tok = 0x7fffffff;
+    }
+    __syncthreads();
+  }
   const int seg = s_seg;
   if (seg < 0) {  // no mass anywhere (cannot happen for finite logits)
     if (threadIdx.x == 0) p.out_tokens[c.t0 + c.n] = -1;
