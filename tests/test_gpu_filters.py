@@ -340,15 +340,16 @@ def test_ragged_vocabulary_and_unusual_rows(V):
     assert int(tok.max()) < V
 
 
-def test_full_size_filtered():
-    spec = W.CONFIGS[1]
+@pytest.mark.parametrize("idx", [1, 2])
+def test_full_size_filtered(idx):
+    spec = W.CONFIGS[idx]
     b_cpu = W.generate(spec)
     tau, tk, tp = _params(b_cpu.batch, spec.vocab)
     b_cpu = _redraft(b_cpu, tau, tk, tp, seed=11)
     acc, tok, _, ws = _run(b_cpu, tau, tk, tp)
     assert int(ws.status.item()) & ~spx.DEV_DEGENERATE == 0
     rep = check_sampling(b_cpu, acc, tok, temperature=tau, top_k=tk, top_p=tp)
-    _report("llama3-8b, mixed filters", rep)
+    _report(f"{spec.name}, mixed filters", rep)
     assert not rep.hard_mismatch, rep
     # repeated launches agree bit for bit (integer atomics: no dependence on the order of arrival)
     for _ in range(2):
